@@ -1,0 +1,163 @@
+/*
+ * moa.h -- C ABI of libmoa: single-query decode attention over a KV cache on one
+ * NVIDIA B200 (sm_100a), with GQA/MQA head grouping and the O(d_k+d_v) cache append.
+ *
+ * What is computed (per batch item b and query head g, fp32, row-major):
+ *     g_kv   = g / (h_q / h_kv)                         GQA psi-selection (section 6.1)
+ *     s[l]   = scale * sum_j q[b,g,j] * K[b,g_kv,l,j]   Step I,   eq. (1)
+ *     a[l]   = exp(s[l]-max s) / sum_l exp(s[l]-max s)  Step II,  eq. (2)
+ *     out[b,g,d] = sum_l a[l] * V[b,g_kv,l,d]           Step III, eq. (3)  (Algorithm 1)
+ * and the append  K[b,h,pos_b,:] <- k_new[b,h,:],  V likewise      eqs. (4),(5).
+ *
+ * Conventions
+ *  - Unless a parameter says HOST, every pointer is a DEVICE pointer on the current
+ *    device, owned by the caller; the library never frees or retains it.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls
+ *    enqueue work on it and return without synchronising, unless stated otherwise.
+ *  - Every step runs in CUDA kernels of this library.  There is no CPU fallback: on a
+ *    machine without a usable GPU the compute entry points return MOA_ERR_CUDA.
+ *  - Arguments are validated on the host before anything is launched; on a non-zero
+ *    return nothing has been written.
+ *  - Results are deterministic: no floating-point atomics, fixed merge order.
+ */
+#ifndef MOA_H
+#define MOA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- return codes ---------------------------------------------------------------- */
+#define MOA_OK               0
+#define MOA_ERR_INVALID      1  /* null pointer, dimension < 1, h_q % h_kv != 0, non-finite scale */
+#define MOA_ERR_UNSUPPORTED  2  /* d_k or d_v above the compiled maximum (MOA_MAX_DK / MOA_MAX_DV) */
+#define MOA_ERR_ALIGN        3  /* a float pointer that is not 4-byte aligned */
+#define MOA_ERR_CAPACITY     4  /* a size beyond a fixed capacity known on the host */
+#define MOA_ERR_WORKSPACE    5  /* workspace missing or smaller than moa_workspace_bytes() */
+#define MOA_ERR_CUDA         6  /* a CUDA runtime call failed (no device, launch error, ...) */
+
+#define MOA_MAX_DK 1024
+#define MOA_MAX_DV 512
+
+/* ---- device status bits (see moa_device_status) ----------------------------------- */
+#define MOA_STATUS_APPEND_RANGE  1  /* append: pos[b] outside [0,n_max); that row was skipped */
+#define MOA_STATUS_SEQLEN_RANGE  2  /* decode: seq_lens[b] outside [1,n_max]; that item's out untouched */
+#define MOA_STATUS_WAIT_TIMEOUT  4  /* a bounded in-kernel wait expired; results of that call are invalid */
+
+/*
+ * Decode attention over a dense cache (problem statement of section 2; batch/head
+ * lifting of section 2 "Formal Inputs"; GQA of section 6).
+ *   q   [batch, h_q,  d_k]       K [batch, h_kv, n, d_k]
+ *   out [batch, h_q,  d_v]       V [batch, h_kv, n, d_v]
+ * n >= 1 cached tokens.  `scale` is applied once, to the dot product (any finite value).
+ * Scratch for split-sequence partial results comes from a per-device buffer owned by
+ * the library (allocated on first use, outside any stream capture; grown on demand;
+ * released by moa_release).  Calls that may overlap on one device must instead use
+ * moa_decode_attn_varlen with their own workspace.
+ */
+int moa_decode_attn(const float *q, const float *K, const float *V, float *out,
+                    int batch, int h_q, int h_kv, int n, int d_k, int d_v,
+                    float scale, void *stream);
+
+/*
+ * Decode attention over a pre-allocated cache with per-sequence lengths (the cache of
+ * section 5.3 lifted over a batch): K [batch,h_kv,n_max,d_k], V [batch,h_kv,n_max,d_v];
+ * sequence b attends over rows [0, seq_lens[b]).  seq_lens is a device int32[batch]
+ * read by the kernels at execution time (so a captured graph can be replayed while the
+ * lengths advance) and never modified.  seq_lens == NULL means every length is n_max.
+ * A length outside [1, n_max] sets MOA_STATUS_SEQLEN_RANGE and leaves that item's rows
+ * of `out` untouched.
+ * `workspace`: device memory, 256-byte aligned, at least moa_workspace_bytes(...) bytes,
+ * owned by the caller, contents undefined on entry and exit; it must not be shared by
+ * calls that can overlap on the GPU.  The call allocates nothing.
+ */
+int moa_decode_attn_varlen(const float *q, const float *K, const float *V, float *out,
+                           int batch, int h_q, int h_kv, const int32_t *seq_lens,
+                           int n_max, int d_k, int d_v, float scale,
+                           void *workspace, size_t workspace_bytes, void *stream);
+
+/* Workspace size in bytes that moa_decode_attn_varlen needs for these dimensions on the
+ * current device (0 on invalid dimensions).  Host-only arithmetic plus one device
+ * attribute query. */
+size_t moa_workspace_bytes(int batch, int h_q, int h_kv, int n_max, int d_k, int d_v);
+
+/*
+ * Cache append (eqs. (4),(5); Proposition 2): for every (b, h) copy the 32-bit patterns
+ * of k_new[b,h,:] into K[b,h,pos[b],:] and of v_new[b,h,:] into V[b,h,pos[b],:].
+ * Exactly (d_k+d_v)*4 bytes are read and written per (b,h); no other element changes.
+ *   K [batch,h_kv,n_max,d_k]  V [batch,h_kv,n_max,d_v]
+ *   k_new [batch,h_kv,d_k]    v_new [batch,h_kv,d_v]      pos: device int32[batch]
+ * pos[b] outside [0,n_max) sets MOA_STATUS_APPEND_RANGE and skips item b.
+ * pos is not modified (the caller owns the lengths; see moa_lens_add).
+ */
+int moa_kv_append(float *K, float *V, const float *k_new, const float *v_new,
+                  const int32_t *pos, int batch, int h_kv, int n_max, int d_k, int d_v,
+                  void *stream);
+
+/* lens[b] += delta for b < batch, on the stream (the length counter of the cache of
+ * section 5.3, kept on the device so that a decode loop needs no host round trip). */
+int moa_lens_add(int32_t *lens, int batch, int delta, void *stream);
+
+/*
+ * One autoregressive step (the append-then-attend order of section 5.3's decode loop;
+ * per-step cost M_step of section 5.2) in a single call:
+ *   append (k_new, v_new) at row lens[b], then attend q over rows [0, lens[b]+1),
+ *   then lens[b] += 1.
+ * lens is a device int32[batch] that the call updates; all other arguments as above.
+ * Requires lens[b] in [0, n_max-1]; otherwise the status bits above are set, the item
+ * is skipped and its length is left unchanged.
+ */
+int moa_decode_step(const float *q, float *K, float *V, const float *k_new,
+                    const float *v_new, float *out, int32_t *lens,
+                    int batch, int h_q, int h_kv, int n_max, int d_k, int d_v, float scale,
+                    void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Host-buffer convenience call: q, K, V, out are HOST pointers (pinned memory gives
+ * full copy bandwidth).  Copies the inputs to library-owned device staging buffers,
+ * runs moa_decode_attn and copies `out` back; synchronises before returning.
+ * Staging buffers are grown on demand and kept until moa_release.
+ */
+int moa_decode_attn_host(const float *q, const float *K, const float *V, float *out,
+                         int batch, int h_q, int h_kv, int n, int d_k, int d_v,
+                         float scale);
+
+/* Synchronise `stream`, copy the device status word to *status_out (HOST int) and
+ * clear it.  Zero means no kernel of this library reported a problem since the last
+ * call. */
+int moa_device_status(void *stream, int *status_out);
+
+/* The paper's DRAM-traffic model (Proposition 1, with the h_kv/h_q factor of section 6
+ * and lifted over the batch):  batch*(h_kv*n*(d_k+d_v) + h_q*(d_k+d_v))*4 bytes.
+ * Host-only. */
+long long moa_min_bytes(int batch, int h_q, int h_kv, long long n, int d_k, int d_v);
+
+/* Free every library-owned device buffer on the current device (synchronises). */
+int moa_release(void);
+
+/* Text for a return code.  Host-only; the string is static. */
+const char *moa_strerror(int code);
+
+/*
+ * Tuning and test hooks (host-only state, per process).
+ *   MOA_OPT_FORCE_PATH : 0 = automatic, otherwise one of the MOA_PATH_* values below;
+ *                        a forced path that cannot handle the shape returns
+ *                        MOA_ERR_UNSUPPORTED.
+ *   MOA_OPT_NUM_CTAS   : 0 = one streaming CTA per SM, otherwise that many.
+ * moa_last_path() reports which kernel family the last successful decode call used.
+ */
+#define MOA_OPT_FORCE_PATH 1
+#define MOA_OPT_NUM_CTAS   2
+#define MOA_PATH_GENERIC   1   /* any d_k, d_v, alignment: one CTA per (batch, query head) */
+#define MOA_PATH_STREAM    2   /* split-sequence streaming kernel, g_s <= 8, d in {64,128} */
+#define MOA_PATH_GROUPED   3   /* tensor-core kernel for large groups (g_s >= 16) */
+int moa_set_option(int option, int value);
+int moa_last_path(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOA_H */

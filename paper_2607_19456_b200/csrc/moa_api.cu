@@ -1,0 +1,437 @@
+// moa_api.cu -- the extern "C" boundary of libmoa: argument validation, kernel
+// selection, workspace management and launches.  See include/moa.h for the contract.
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+#include <type_traits>
+
+#include "moa.h"
+#include "moa_device.cuh"
+#include "moa_generic.cuh"
+#include "moa_stream.cuh"
+
+namespace moa {
+
+constexpr int kMaxDevices = 64;
+constexpr float kLog2e = 1.4426950408889634f;
+
+struct DeviceState {
+    int sm_count = 0;
+    void *ws = nullptr;          // library-owned workspace (moa_decode_attn)
+    size_t ws_bytes = 0;
+    void *stage[4] = {nullptr, nullptr, nullptr, nullptr};   // host-API staging: q K V out
+    size_t stage_bytes[4] = {0, 0, 0, 0};
+    cudaStream_t host_stream = nullptr;
+};
+static DeviceState g_dev[kMaxDevices];
+static int g_force_path = 0;
+static int g_num_ctas = 0;
+static int g_last_path = 0;
+
+static int current_device(DeviceState **st)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        cudaGetLastError();
+        return MOA_ERR_CUDA;
+    }
+    DeviceState &s = g_dev[dev];
+    if (s.sm_count == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) {
+            cudaGetLastError();
+            return MOA_ERR_CUDA;
+        }
+        s.sm_count = n;
+    }
+    *st = &s;
+    return MOA_OK;
+}
+
+static bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+static int validate_dims(int batch, int h_q, int h_kv, int n, int d_k, int d_v)
+{
+    if (batch < 1 || h_q < 1 || h_kv < 1 || n < 1 || d_k < 1 || d_v < 1) return MOA_ERR_INVALID;
+    if (h_q % h_kv != 0) return MOA_ERR_INVALID;
+    if (d_k > MOA_MAX_DK || d_v > MOA_MAX_DV) return MOA_ERR_UNSUPPORTED;
+    return MOA_OK;
+}
+
+// ---- streaming-kernel plan -------------------------------------------------------------
+struct StreamPlan {
+    bool ok = false;
+    int D = 0;       // feature size
+    int G = 0;       // heads per (virtual) kv head handled by one CTA pass
+    int share = 1;   // virtual kv heads per physical kv head (g_s = share * G when g_s > 8)
+    int R = 0;       // rows per block of the chosen configuration
+};
+
+static int stream_group(int g_s, int *share)
+{
+    if (g_s <= 8) {                      // pad to a power of two
+        int G = 1;
+        while (G < g_s) G <<= 1;
+        *share = 1;
+        return G;
+    }
+    int G = 8;                           // largest power of two <= 8 dividing g_s
+    while (g_s % G != 0) G >>= 1;
+    *share = g_s / G;
+    return G;
+}
+
+static int rows_per_block(int D, int G)
+{
+    if (D == 128) return (G == 8) ? 4 : 8;
+    return (G == 1 || G == 2) ? 16 : (G == 4 ? 8 : 4);
+}
+
+static StreamPlan plan_stream(int g_s, int d_k, int d_v)
+{
+    StreamPlan p;
+    if (d_k != d_v || (d_k != 64 && d_k != 128)) return p;
+    p.D = d_k;
+    p.G = stream_group(g_s, &p.share);
+    p.R = rows_per_block(p.D, p.G);
+    p.ok = true;
+    return p;
+}
+
+static int stream_num_ctas(const DeviceState &s) { return g_num_ctas > 0 ? g_num_ctas : s.sm_count; }
+
+static size_t stream_ws_bytes(const StreamPlan &p, int num_ctas)
+{
+    return (size_t)num_ctas * 2 * p.G * (p.D + 4) * sizeof(float);
+}
+
+template <class C>
+static cudaError_t launch_stream_cfg(const DecodeArgs &a, int num_ctas, cudaStream_t st)
+{
+    static bool attr_set[kMaxDevices] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (!attr_set[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(stream_decode_kernel<C>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)C::SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        attr_set[dev] = true;
+    }
+    stream_decode_kernel<C><<<num_ctas, C::THREADS, C::SMEM_BYTES, st>>>(a);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const long long warps = (long long)a.batch * a.h_q;
+    const int blocks = (int)((warps + 3) / 4);
+    stream_combine_kernel<C::D, C::R><<<blocks, 128, 0, st>>>(a, num_ctas, C::G);
+    return cudaGetLastError();
+}
+
+static cudaError_t launch_stream(const StreamPlan &p, const DecodeArgs &a, int num_ctas,
+                                 cudaStream_t st)
+{
+    //                                   D    G  RV  S  W
+    if (p.D == 128) {
+        switch (p.G) {
+        case 1: return launch_stream_cfg<StreamCfg<128, 1, 8, 3, 8>>(a, num_ctas, st);
+        case 2: return launch_stream_cfg<StreamCfg<128, 2, 8, 3, 8>>(a, num_ctas, st);
+        case 4: return launch_stream_cfg<StreamCfg<128, 4, 8, 3, 8>>(a, num_ctas, st);
+        default: return launch_stream_cfg<StreamCfg<128, 8, 4, 5, 8>>(a, num_ctas, st);
+        }
+    }
+    switch (p.G) {
+    case 1: return launch_stream_cfg<StreamCfg<64, 1, 8, 3, 8>>(a, num_ctas, st);
+    case 2: return launch_stream_cfg<StreamCfg<64, 2, 8, 3, 8>>(a, num_ctas, st);
+    case 4: return launch_stream_cfg<StreamCfg<64, 4, 4, 6, 8>>(a, num_ctas, st);
+    default: return launch_stream_cfg<StreamCfg<64, 8, 2, 8, 8>>(a, num_ctas, st);
+    }
+}
+
+static cudaError_t launch_generic(const DecodeArgs &a, cudaStream_t st)
+{
+    const size_t smem = sizeof(float) * ((size_t)a.d_k + (size_t)kGenericWarps * a.d_v + 2 * kGenericWarps);
+    if (a.seq_lens != nullptr) {
+        check_lens_kernel<<<(a.batch + 127) / 128, 128, 0, st>>>(a.seq_lens, a.len_bias, a.batch, a.n_max);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    generic_decode_kernel<<<a.batch * a.h_q, kGenericWarps * 32, smem, st>>>(a);
+    return cudaGetLastError();
+}
+
+// Shared implementation of the decode entry points.  `ws` may be null when the chosen
+// path needs none.
+static int decode_impl(const float *q, const float *K, const float *V, float *out, int batch,
+                       int h_q, int h_kv, const int32_t *seq_lens, int len_bias, int n_max,
+                       int d_k, int d_v, float scale, void *ws, size_t ws_bytes,
+                       bool library_ws, cudaStream_t st)
+{
+    if (!q || !K || !V || !out) return MOA_ERR_INVALID;
+    int rc = validate_dims(batch, h_q, h_kv, n_max, d_k, d_v);
+    if (rc != MOA_OK) return rc;
+    if (!isfinite(scale)) return MOA_ERR_INVALID;
+    if (!aligned(q, 4) || !aligned(K, 4) || !aligned(V, 4) || !aligned(out, 4)) return MOA_ERR_ALIGN;
+    if (seq_lens && !aligned(seq_lens, 4)) return MOA_ERR_ALIGN;
+    if ((long long)batch * h_q > 0x7fffffffLL) return MOA_ERR_CAPACITY;
+
+    DeviceState *dev = nullptr;
+    rc = current_device(&dev);
+    if (rc != MOA_OK) return rc;
+
+    const int g_s = h_q / h_kv;
+    StreamPlan plan = plan_stream(g_s, d_k, d_v);
+    const bool fast_ok = plan.ok && aligned(q, 16) && aligned(K, 16) && aligned(V, 16) && aligned(out, 16);
+    int path = fast_ok ? MOA_PATH_STREAM : MOA_PATH_GENERIC;
+    if (g_force_path == MOA_PATH_GENERIC) path = MOA_PATH_GENERIC;
+    else if (g_force_path == MOA_PATH_STREAM) {
+        if (!fast_ok) return MOA_ERR_UNSUPPORTED;
+    } else if (g_force_path != 0) return MOA_ERR_UNSUPPORTED;
+
+    DecodeArgs a;
+    a.q = q; a.K = K; a.V = V; a.out = out; a.ws = nullptr;
+    a.seq_lens = seq_lens; a.len_bias = len_bias;
+    a.batch = batch; a.h_q = h_q; a.h_kv = h_kv; a.g_s = g_s; a.kv_share = 1;
+    a.n_max = n_max; a.d_k = d_k; a.d_v = d_v;
+    a.qscale = scale * kLog2e;
+
+    cudaError_t e;
+    if (path == MOA_PATH_STREAM) {
+        const int num_ctas = stream_num_ctas(*dev);
+        const size_t need = stream_ws_bytes(plan, num_ctas);
+        if (library_ws) {
+            if (dev->ws_bytes < need) {
+                if (dev->ws) { cudaDeviceSynchronize(); cudaFree(dev->ws); dev->ws = nullptr; dev->ws_bytes = 0; }
+                if (cudaMalloc(&dev->ws, need) != cudaSuccess) { cudaGetLastError(); return MOA_ERR_CUDA; }
+                dev->ws_bytes = need;
+            }
+            ws = dev->ws;
+        } else {
+            if (!ws || ws_bytes < need) return MOA_ERR_WORKSPACE;
+            if (!aligned(ws, 256)) return MOA_ERR_ALIGN;
+        }
+        a.ws = static_cast<float *>(ws);
+        a.h_kv = h_kv * plan.share;        // virtual kv heads of plan.G query heads each
+        a.g_s = (plan.share > 1) ? plan.G : g_s;
+        a.kv_share = plan.share;
+        e = launch_stream(plan, a, num_ctas, st);
+    } else {
+        e = launch_generic(a, st);
+    }
+    if (e != cudaSuccess) return MOA_ERR_CUDA;
+    g_last_path = path;
+    return MOA_OK;
+}
+
+}  // namespace moa
+
+using namespace moa;
+
+extern "C" {
+
+int moa_decode_attn(const float *q, const float *K, const float *V, float *out, int batch,
+                    int h_q, int h_kv, int n, int d_k, int d_v, float scale, void *stream)
+{
+    return decode_impl(q, K, V, out, batch, h_q, h_kv, nullptr, 0, n, d_k, d_v, scale, nullptr, 0,
+                       true, static_cast<cudaStream_t>(stream));
+}
+
+int moa_decode_attn_varlen(const float *q, const float *K, const float *V, float *out, int batch,
+                           int h_q, int h_kv, const int32_t *seq_lens, int n_max, int d_k,
+                           int d_v, float scale, void *workspace, size_t workspace_bytes,
+                           void *stream)
+{
+    return decode_impl(q, K, V, out, batch, h_q, h_kv, seq_lens, 0, n_max, d_k, d_v, scale,
+                       workspace, workspace_bytes, false, static_cast<cudaStream_t>(stream));
+}
+
+size_t moa_workspace_bytes(int batch, int h_q, int h_kv, int n_max, int d_k, int d_v)
+{
+    if (validate_dims(batch, h_q, h_kv, n_max, d_k, d_v) != MOA_OK) return 0;
+    StreamPlan plan = plan_stream(h_q / h_kv, d_k, d_v);
+    if (!plan.ok) return 256;              // generic path: no scratch; keep the result non-zero
+    DeviceState *dev = nullptr;
+    int ctas = g_num_ctas;
+    if (ctas <= 0) ctas = (current_device(&dev) == MOA_OK) ? dev->sm_count : 256;
+    const size_t need = stream_ws_bytes(plan, ctas);
+    return (need + 255) / 256 * 256;
+}
+
+int moa_kv_append(float *K, float *V, const float *k_new, const float *v_new, const int32_t *pos,
+                  int batch, int h_kv, int n_max, int d_k, int d_v, void *stream)
+{
+    if (!K || !V || !k_new || !v_new || !pos) return MOA_ERR_INVALID;
+    if (batch < 1 || h_kv < 1 || n_max < 1 || d_k < 1 || d_v < 1) return MOA_ERR_INVALID;
+    if (!aligned(K, 4) || !aligned(V, 4) || !aligned(k_new, 4) || !aligned(v_new, 4) || !aligned(pos, 4))
+        return MOA_ERR_ALIGN;
+    DeviceState *dev = nullptr;
+    int rc = current_device(&dev);
+    if (rc != MOA_OK) return rc;
+    const long long words = (long long)batch * h_kv * ((long long)d_k + d_v);
+    const long long blocks = (words + 255) / 256;
+    if (blocks > 0x7fffffffLL) return MOA_ERR_CAPACITY;
+    kv_append_kernel<<<(int)blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        reinterpret_cast<uint32_t *>(K), reinterpret_cast<uint32_t *>(V),
+        reinterpret_cast<const uint32_t *>(k_new), reinterpret_cast<const uint32_t *>(v_new), pos,
+        batch, h_kv, n_max, d_k, d_v);
+    return cudaGetLastError() == cudaSuccess ? MOA_OK : MOA_ERR_CUDA;
+}
+
+int moa_lens_add(int32_t *lens, int batch, int delta, void *stream)
+{
+    if (!lens || batch < 1) return MOA_ERR_INVALID;
+    if (!aligned(lens, 4)) return MOA_ERR_ALIGN;
+    DeviceState *dev = nullptr;
+    int rc = current_device(&dev);
+    if (rc != MOA_OK) return rc;
+    lens_add_kernel<<<(batch + 127) / 128, 128, 0, static_cast<cudaStream_t>(stream)>>>(lens, batch, delta, 0);
+    return cudaGetLastError() == cudaSuccess ? MOA_OK : MOA_ERR_CUDA;
+}
+
+int moa_decode_step(const float *q, float *K, float *V, const float *k_new, const float *v_new,
+                    float *out, int32_t *lens, int batch, int h_q, int h_kv, int n_max, int d_k,
+                    int d_v, float scale, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!q || !K || !V || !k_new || !v_new || !out || !lens) return MOA_ERR_INVALID;
+    int rc = validate_dims(batch, h_q, h_kv, n_max, d_k, d_v);
+    if (rc != MOA_OK) return rc;
+    if (!isfinite(scale)) return MOA_ERR_INVALID;
+    // Dry validation of the decode arguments first, so that nothing is appended when the
+    // attention call would be rejected.
+    if (!aligned(q, 4) || !aligned(K, 4) || !aligned(V, 4) || !aligned(out, 4) || !aligned(lens, 4) ||
+        !aligned(k_new, 4) || !aligned(v_new, 4))
+        return MOA_ERR_ALIGN;
+    const size_t need = moa_workspace_bytes(batch, h_q, h_kv, n_max, d_k, d_v);
+    StreamPlan plan = plan_stream(h_q / h_kv, d_k, d_v);
+    const bool fast_ok = plan.ok && aligned(q, 16) && aligned(K, 16) && aligned(V, 16) && aligned(out, 16);
+    if (fast_ok && g_force_path != MOA_PATH_GENERIC) {
+        if (!workspace || workspace_bytes < need) return MOA_ERR_WORKSPACE;
+        if (!aligned(workspace, 256)) return MOA_ERR_ALIGN;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    rc = moa_kv_append(K, V, k_new, v_new, lens, batch, h_kv, n_max, d_k, d_v, stream);
+    if (rc != MOA_OK) return rc;
+    rc = decode_impl(q, K, V, out, batch, h_q, h_kv, lens, 1, n_max, d_k, d_v, scale, workspace,
+                     workspace_bytes, false, st);
+    if (rc != MOA_OK) return rc;
+    lens_add_kernel<<<(batch + 127) / 128, 128, 0, st>>>(lens, batch, 1, n_max);
+    return cudaGetLastError() == cudaSuccess ? MOA_OK : MOA_ERR_CUDA;
+}
+
+int moa_decode_attn_host(const float *q, const float *K, const float *V, float *out, int batch,
+                         int h_q, int h_kv, int n, int d_k, int d_v, float scale)
+{
+    if (!q || !K || !V || !out) return MOA_ERR_INVALID;
+    int rc = validate_dims(batch, h_q, h_kv, n, d_k, d_v);
+    if (rc != MOA_OK) return rc;
+    if (!isfinite(scale)) return MOA_ERR_INVALID;
+    DeviceState *dev = nullptr;
+    rc = current_device(&dev);
+    if (rc != MOA_OK) return rc;
+    if (!dev->host_stream &&
+        cudaStreamCreateWithFlags(&dev->host_stream, cudaStreamNonBlocking) != cudaSuccess) {
+        cudaGetLastError();
+        return MOA_ERR_CUDA;
+    }
+    const size_t bytes[4] = {sizeof(float) * (size_t)batch * h_q * d_k,
+                             sizeof(float) * (size_t)batch * h_kv * n * d_k,
+                             sizeof(float) * (size_t)batch * h_kv * n * d_v,
+                             sizeof(float) * (size_t)batch * h_q * d_v};
+    for (int i = 0; i < 4; ++i) {
+        if (dev->stage_bytes[i] < bytes[i]) {
+            if (dev->stage[i]) { cudaDeviceSynchronize(); cudaFree(dev->stage[i]); dev->stage[i] = nullptr; dev->stage_bytes[i] = 0; }
+            if (cudaMalloc(&dev->stage[i], bytes[i]) != cudaSuccess) { cudaGetLastError(); return MOA_ERR_CUDA; }
+            dev->stage_bytes[i] = bytes[i];
+        }
+    }
+    cudaStream_t st = dev->host_stream;
+    const void *src[3] = {q, K, V};
+    for (int i = 0; i < 3; ++i)
+        if (cudaMemcpyAsync(dev->stage[i], src[i], bytes[i], cudaMemcpyHostToDevice, st) != cudaSuccess) {
+            cudaGetLastError();
+            return MOA_ERR_CUDA;
+        }
+    rc = decode_impl(static_cast<float *>(dev->stage[0]), static_cast<float *>(dev->stage[1]),
+                     static_cast<float *>(dev->stage[2]), static_cast<float *>(dev->stage[3]), batch,
+                     h_q, h_kv, nullptr, 0, n, d_k, d_v, scale, nullptr, 0, true, st);
+    if (rc != MOA_OK) return rc;
+    if (cudaMemcpyAsync(out, dev->stage[3], bytes[3], cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+        cudaGetLastError();
+        return MOA_ERR_CUDA;
+    }
+    return MOA_OK;
+}
+
+int moa_device_status(void *stream, int *status_out)
+{
+    if (!status_out) return MOA_ERR_INVALID;
+    DeviceState *dev = nullptr;
+    int rc = current_device(&dev);
+    if (rc != MOA_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int v = 0;
+    const int zero = 0;
+    if (cudaMemcpyFromSymbolAsync(&v, g_status_word, sizeof(int), 0, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaMemcpyToSymbolAsync(g_status_word, &zero, sizeof(int), 0, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+        cudaGetLastError();
+        return MOA_ERR_CUDA;
+    }
+    *status_out = v;
+    return MOA_OK;
+}
+
+long long moa_min_bytes(int batch, int h_q, int h_kv, long long n, int d_k, int d_v)
+{
+    const long long row_pair = (long long)d_k + (long long)d_v;
+    return 4LL * batch * (h_kv * n * row_pair + h_q * row_pair);
+}
+
+int moa_release(void)
+{
+    DeviceState *dev = nullptr;
+    int rc = current_device(&dev);
+    if (rc != MOA_OK) return rc;
+    cudaDeviceSynchronize();
+    if (dev->ws) cudaFree(dev->ws);
+    dev->ws = nullptr; dev->ws_bytes = 0;
+    for (int i = 0; i < 4; ++i) {
+        if (dev->stage[i]) cudaFree(dev->stage[i]);
+        dev->stage[i] = nullptr; dev->stage_bytes[i] = 0;
+    }
+    if (dev->host_stream) { cudaStreamDestroy(dev->host_stream); dev->host_stream = nullptr; }
+    return cudaGetLastError() == cudaSuccess ? MOA_OK : MOA_ERR_CUDA;
+}
+
+const char *moa_strerror(int code)
+{
+    switch (code) {
+    case MOA_OK: return "ok";
+    case MOA_ERR_INVALID: return "invalid argument";
+    case MOA_ERR_UNSUPPORTED: return "unsupported dimensions or forced path";
+    case MOA_ERR_ALIGN: return "misaligned pointer";
+    case MOA_ERR_CAPACITY: return "size beyond a fixed capacity";
+    case MOA_ERR_WORKSPACE: return "workspace missing or too small";
+    case MOA_ERR_CUDA: return "CUDA runtime error";
+    default: return "unknown error code";
+    }
+}
+
+int moa_set_option(int option, int value)
+{
+    if (option == MOA_OPT_FORCE_PATH) {
+        if (value < 0 || value > MOA_PATH_GROUPED) return MOA_ERR_INVALID;
+        g_force_path = value;
+        return MOA_OK;
+    }
+    if (option == MOA_OPT_NUM_CTAS) {
+        if (value < 0 || value > 65535) return MOA_ERR_INVALID;
+        g_num_ctas = value;
+        return MOA_OK;
+    }
+    return MOA_ERR_INVALID;
+}
+
+int moa_last_path(void) { return g_last_path; }
+
+}  // extern "C"

@@ -1,0 +1,200 @@
+// moa_device.cuh -- small device-side building blocks shared by the kernels of libmoa:
+// mbarrier + bulk-async-copy wrappers (inline PTX, sm_100a), bounded waits, the device
+// status word and the work cursor that maps a flat row-block index to (batch, kv head,
+// first row).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "moa.h"
+
+namespace moa {
+
+// One status word per device, OR-ed into by kernels, read and cleared by
+// moa_device_status().
+__device__ int g_status_word;
+
+__device__ __forceinline__ void raise_status(int bits) { atomicOr(&g_status_word, bits); }
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p)
+{
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+// ---- mbarrier -------------------------------------------------------------------------
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+
+__device__ __forceinline__ void mbar_fence_init()
+{
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+                 : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// Every spin in this library is bounded: after kWaitLimit unsuccessful polls the caller
+// gives up, raises MOA_STATUS_WAIT_TIMEOUT and leaves without touching the data.
+constexpr uint32_t kWaitLimit = 1u << 22;
+
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
+{
+    for (uint32_t it = 0; it < kWaitLimit; ++it)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+
+// ---- bulk asynchronous copy global -> shared (TMA engine, 1-D) --------------------------
+// dst and src 16-byte aligned, bytes a positive multiple of 16.  Completion is signalled
+// on the mbarrier as `bytes` transaction bytes.  No multicast: every CTA fetches its own
+// tile.
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes,
+                                         uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+        : "memory");
+}
+
+__device__ __forceinline__ float fast_exp2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// exp2(a - b) that is 0 when a is -inf (an empty partial), whatever b is.
+__device__ __forceinline__ float exp2_diff(float a, float b)
+{
+    return (a == -INFINITY) ? 0.0f : fast_exp2(a - b);
+}
+
+// ---- problem description passed to the decode kernels ----------------------------------
+struct DecodeArgs {
+    const float *q;           // [batch, h_q, d_k]
+    const float *K;           // [batch, h_kv, n_max, d_k]
+    const float *V;           // [batch, h_kv, n_max, d_v]
+    float *out;               // [batch, h_q, d_v]
+    float *ws;                // partial slots (streaming kernels) or nullptr
+    const int32_t *seq_lens;  // device [batch] or nullptr (= every length is n_max)
+    int32_t len_bias;         // added to every seq_lens[b] (fused step: attend over len+1)
+    int batch, h_q;
+    int h_kv;                 // kv heads as the kernels count them (virtual heads, see kv_share)
+    int g_s;                  // query heads per (virtual) kv head
+    int kv_share;             // consecutive virtual kv heads that read the same stored K/V head
+    int n_max;                // row capacity = stride between heads
+    int d_k, d_v;
+    float qscale;             // scale * log2(e): scores live in the log2 domain
+};
+
+// Length of sequence b as the kernels see it; 0 for an out-of-range length (the item is
+// then skipped by construction: it owns no row blocks).
+__device__ __forceinline__ int seq_len_of(const DecodeArgs &a, int b)
+{
+    if (a.seq_lens == nullptr) return a.n_max;
+    const int len = a.seq_lens[b] + a.len_bias;
+    return (len >= 1 && len <= a.n_max) ? len : 0;
+}
+
+// ---- work cursor -----------------------------------------------------------------------
+// The sequence axis of every (batch b, kv head h) "unit" is cut into row blocks of R
+// rows; blocks are numbered unit by unit (b major, h minor).  A cursor remembers the unit
+// that contains a block index and can only move forward.
+struct Cursor {
+    int b, h;          // current unit
+    int len;           // rows in this unit's sequence
+    int ub;            // row blocks in this unit
+    long long first;   // flat index of the unit's first block
+};
+
+template <int R>
+__device__ __forceinline__ int blocks_of(int len) { return (len + R - 1) / R; }
+
+// Total number of row blocks (warp-collective; every lane gets the result).
+template <int R>
+__device__ __forceinline__ long long total_blocks(const DecodeArgs &a, int lane)
+{
+    if (a.seq_lens == nullptr) return (long long)a.batch * a.h_kv * blocks_of<R>(a.n_max);
+    long long tot = 0;
+    for (int base = 0; base < a.batch; base += 32) {
+        const int b = base + lane;
+        int nb = (b < a.batch) ? blocks_of<R>(seq_len_of(a, b)) : 0;
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) nb += __shfl_xor_sync(0xffffffffu, nb, off);
+        tot += (long long)nb * a.h_kv;
+    }
+    return tot;
+}
+
+// Position a cursor on the unit containing block j (0 <= j < total).  Warp-uniform.
+template <int R>
+__device__ __forceinline__ Cursor cursor_at(const DecodeArgs &a, long long j)
+{
+    Cursor c;
+    if (a.seq_lens == nullptr) {
+        const int ub = blocks_of<R>(a.n_max);
+        const long long u = j / ub;
+        c.b = (int)(u / a.h_kv);
+        c.h = (int)(u % a.h_kv);
+        c.len = a.n_max;
+        c.ub = ub;
+        c.first = u * ub;
+        return c;
+    }
+    long long first = 0;
+    int b = 0;
+    for (; b < a.batch; ++b) {
+        const int len = seq_len_of(a, b);
+        const int ub = blocks_of<R>(len);
+        const long long span = (long long)ub * a.h_kv;
+        if (j < first + span) {
+            c.b = b;
+            c.h = (int)((j - first) / ub);
+            c.len = len;
+            c.ub = ub;
+            c.first = first + (long long)c.h * ub;
+            return c;
+        }
+        first += span;
+    }
+    c.b = a.batch; c.h = 0; c.len = 0; c.ub = 0; c.first = first;   // past the end
+    return c;
+}
+
+// Move to the next unit that owns at least one block (or past the end: b == batch).
+template <int R>
+__device__ __forceinline__ void cursor_next_unit(const DecodeArgs &a, Cursor &c)
+{
+    c.first += c.ub;
+    for (;;) {
+        if (++c.h == a.h_kv) {
+            c.h = 0;
+            if (++c.b >= a.batch) { c.b = a.batch; c.len = 0; c.ub = 0; return; }
+            c.len = seq_len_of(a, c.b);
+            c.ub = blocks_of<R>(c.len);
+        }
+        if (c.ub > 0) return;
+    }
+}
+
+}  // namespace moa

@@ -1,0 +1,277 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the
+same seeded inputs.  Bar: max abs error <= 5e-6 for fp32 outputs; append bit-exact."""
+import math
+
+import numpy as np
+import pytest
+
+import moa_inputs as mi
+import oracle
+import paper_2607_19456_b200 as moa
+from gpu_util import TOL, Guarded, gpu_decode, max_err, workspace_for
+
+pytestmark = pytest.mark.gpu
+torch = pytest.importorskip("torch")
+
+
+def make(seed, B, hq, hkv, n, dk, dv, v_dist="normal"):
+    w = mi.Workload("t", seed, B, hq, hkv, n, dk, dv, v_dist=v_dist)
+    return w.q(), w.K(), w.V(), w.scale
+
+
+# ---------------------------------------------------------------------------------------
+# the paper's worked example and verification shapes
+# ---------------------------------------------------------------------------------------
+def test_worked_example_on_gpu():
+    q = np.array([[[1, 0]]], np.float32)
+    K = np.array([[[[1, 0], [0, 1]]]], np.float32)
+    V = np.array([[[[2, 4], [6, 8]]]], np.float32)
+    out = gpu_decode(q, K, V, 1 / math.sqrt(2), expect_path=moa.PATH_GENERIC)
+    assert max_err(out, oracle.decode(q, K, V, 1 / math.sqrt(2))) <= TOL
+    assert abs(out[0, 0, 0] - 3.32) < 6e-3 and abs(out[0, 0, 1] - 5.32) < 6e-3
+
+
+@pytest.mark.parametrize("n", [4, 64, 256, 1024, 4096])
+def test_paper_decode_shapes_d64(n):
+    q, K, V, s = make(10 + n, 1, 1, 1, n, 64, 64)
+    ref = oracle.decode(q, K, V, s)
+    assert max_err(gpu_decode(q, K, V, s, expect_path=moa.PATH_STREAM), ref) <= TOL
+    assert max_err(gpu_decode(q, K, V, s, path=moa.PATH_GENERIC), ref) <= TOL
+
+
+@pytest.mark.parametrize("hkv", [8, 4, 2, 1])
+def test_paper_gqa_shapes_d32(hkv):
+    q, K, V, s = make(20 + hkv, 1, 8, hkv, 64, 32, 32)
+    assert max_err(gpu_decode(q, K, V, s), oracle.decode(q, K, V, s)) <= TOL
+
+
+# ---------------------------------------------------------------------------------------
+# streaming kernel: every compiled (D, G) variant, ragged tails, several tiles, splits
+# ---------------------------------------------------------------------------------------
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("gs", [1, 2, 3, 4, 5, 8, 12, 16, 64])
+def test_stream_kernel_group_sizes(D, gs):
+    hkv = 2
+    for n in (1, 7, 130, 1037):
+        q, K, V, s = make(1000 * D + 10 * gs + n, 2, gs * hkv, hkv, n, D, D)
+        out = gpu_decode(q, K, V, s, expect_path=moa.PATH_STREAM)
+        assert max_err(out, oracle.decode(q, K, V, s)) <= TOL, (D, gs, n)
+
+
+@pytest.mark.parametrize("n", [1, 2, 3, 4, 5, 8, 9, 15, 16, 17, 31, 32, 33, 63, 64, 65, 127, 129, 1000, 5003])
+def test_stream_kernel_every_tail_length(n):
+    q, K, V, s = make(300 + n, 3, 8, 2, n, 128, 128)
+    assert max_err(gpu_decode(q, K, V, s, expect_path=moa.PATH_STREAM), oracle.decode(q, K, V, s)) <= TOL
+    q, K, V, s = make(400 + n, 2, 2, 2, n, 64, 64)
+    assert max_err(gpu_decode(q, K, V, s, expect_path=moa.PATH_STREAM), oracle.decode(q, K, V, s)) <= TOL
+
+
+@pytest.mark.parametrize("ctas", [1, 2, 3, 7, 37, 148, 500, 4000])
+def test_stream_kernel_any_cta_count_gives_the_same_answer(ctas):
+    # units split across CTAs at arbitrary places, CTAs spanning several units, idle CTAs
+    q, K, V, s = make(77, 3, 8, 2, 2500, 128, 128)
+    ref = oracle.decode(q, K, V, s)
+    assert max_err(gpu_decode(q, K, V, s, num_ctas=ctas, expect_path=moa.PATH_STREAM), ref) <= TOL
+
+
+def test_results_are_deterministic():
+    q, K, V, s = make(78, 2, 32, 8, 3000, 128, 128)
+    a = gpu_decode(q, K, V, s)
+    b = gpu_decode(q, K, V, s)
+    assert np.array_equal(a.view(np.uint32), b.view(np.uint32))
+
+
+def test_large_scores_and_uniform_values():
+    q, K, V, s = make(79, 2, 8, 2, 700, 128, 128, v_dist="uniform")
+    q, K = 4 * q, 4 * K                      # scores of order +-70: exercises the running max
+    # (fp32 scores carry an absolute rounding error of about |s| * 2^-23, which the softmax
+    # turns into the same relative error of the weights; +-70 keeps that inside the bar)
+    ref = oracle.decode(q, K, V, s)
+    assert max_err(gpu_decode(q, K, V, s), ref) <= TOL
+    assert max_err(gpu_decode(q, K, V, s, path=moa.PATH_GENERIC), ref) <= TOL
+
+
+def test_invariants_on_gpu():
+    q, K, V, s = make(80, 2, 4, 2, 1, 128, 128)                 # n = 1 -> out = v_0
+    out = gpu_decode(q, K, V, s)
+    assert np.array_equal(out, np.repeat(V[:, :, 0, :], 2, axis=1))
+    q, K, V, s = make(81, 1, 4, 1, 999, 128, 128)               # identical keys -> mean of V
+    K[:] = K[:, :, :1, :]
+    out = gpu_decode(q, K, V, s)
+    mean = V[0, 0].astype(np.float64).mean(axis=0)
+    assert np.max(np.abs(out[0] - mean)) <= TOL
+
+
+# ---------------------------------------------------------------------------------------
+# generic kernel: odd sizes, d_k != d_v, pointers that are only 4-byte aligned
+# ---------------------------------------------------------------------------------------
+@pytest.mark.parametrize("B,hq,hkv,n,dk,dv", [(1, 1, 1, 3, 2, 2), (2, 4, 2, 9, 3, 5), (1, 6, 3, 100, 40, 72),
+                                               (2, 2, 1, 517, 256, 130), (1, 3, 1, 33, 1024, 512),
+                                               (3, 8, 8, 64, 8, 8), (1, 2, 2, 2000, 96, 96)])
+def test_generic_kernel_shapes(B, hq, hkv, n, dk, dv):
+    q, K, V, s = make(500 + n, B, hq, hkv, n, dk, dv)
+    assert max_err(gpu_decode(q, K, V, s, expect_path=moa.PATH_GENERIC), oracle.decode(q, K, V, s)) <= TOL
+
+
+def test_unaligned_pointers_take_the_generic_kernel():
+    q, K, V, s = make(600, 2, 8, 2, 300, 128, 128)
+    out = gpu_decode(q, K, V, s, misalign=1, expect_path=moa.PATH_GENERIC)
+    assert max_err(out, oracle.decode(q, K, V, s)) <= TOL
+
+
+# ---------------------------------------------------------------------------------------
+# ragged lengths over a pre-allocated cache
+# ---------------------------------------------------------------------------------------
+@pytest.mark.parametrize("D,hq,hkv", [(128, 8, 2), (64, 4, 4), (128, 16, 1), (32, 4, 2)])
+def test_varlen_matches_oracle(D, hq, hkv):
+    B, n_max = 5, 700
+    q, K, V, s = make(700 + D, B, hq, hkv, n_max, D, D)
+    lens = np.array([1, 700, 8, 333, 9], np.int32)
+    ref = oracle.decode_varlen(q, K, V, lens, s)
+    assert max_err(gpu_decode(q, K, V, s, seq_lens=lens), ref) <= TOL
+    assert max_err(gpu_decode(q, K, V, s, seq_lens=lens, num_ctas=5), ref) <= TOL
+    assert max_err(gpu_decode(q, K, V, s, seq_lens=lens, path=moa.PATH_GENERIC), ref) <= TOL
+
+
+@pytest.mark.parametrize("path", [moa.PATH_AUTO, moa.PATH_GENERIC])
+def test_out_of_range_length_sets_status_and_skips_the_item(path):
+    B, hq, hkv, n_max, D = 3, 4, 2, 64, 128
+    q, K, V, s = make(800, B, hq, hkv, n_max, D, D)
+    lens = np.array([10, 0, 65], np.int32)
+    gq, gK, gV = Guarded(q), Guarded(K), Guarded(V)
+    gout = Guarded(shape=(B, hq, D), fill=-7.0)
+    glens = Guarded(lens)
+    gws, nbytes = workspace_for(B, hq, hkv, n_max, D, D)
+    moa.moa_set_option(moa.OPT_FORCE_PATH, path)
+    try:
+        moa.moa_decode_attn_varlen(gq.ptr, gK.ptr, gV.ptr, gout.ptr, B, hq, hkv, glens.ptr, n_max, D, D,
+                                   s, gws.ptr, nbytes)
+    finally:
+        moa.moa_set_option(moa.OPT_FORCE_PATH, 0)
+    assert moa.moa_device_status() == moa.STATUS_SEQLEN_RANGE
+    assert moa.moa_device_status() == 0                       # reading clears it
+    out = gout.host()
+    assert np.all(out[1] == -7.0) and np.all(out[2] == -7.0)
+    ref = oracle.decode_varlen(q[:1], K[:1], V[:1], lens[:1], s)
+    assert max_err(out[:1], ref) <= TOL
+    assert gout.guards_intact() and gws.guards_intact()
+
+
+# ---------------------------------------------------------------------------------------
+# cache append: bit-exact, nothing else touched
+# ---------------------------------------------------------------------------------------
+@pytest.mark.parametrize("B,hkv,n_max,dk,dv", [(1, 1, 3, 3, 1), (4, 8, 50, 128, 128), (3, 2, 7, 5, 9)])
+def test_append_is_bit_exact(B, hkv, n_max, dk, dv):
+    K, V = mi.normal(900, 2, (B, hkv, n_max, dk)), mi.normal(900, 3, (B, hkv, n_max, dv))
+    k_new, v_new = mi.normal(900, 4, (B, hkv, dk)), mi.normal(900, 5, (B, hkv, dv))
+    kb, vb = k_new.view(np.uint32), v_new.view(np.uint32)
+    kb[0, 0, 0] = 0x80000000            # -0.0
+    kb[-1, -1, -1] = 0x7FC12345         # NaN with a payload
+    vb[0, 0, 0] = 0x00000001            # denormal
+    vb[-1, -1, -1] = 0xFF800000         # -inf
+    pos = mi.integers(900, 6, B, 0, n_max - 1)
+    Kr, Vr = K.copy(), V.copy()
+    oracle.kv_append(Kr, Vr, k_new, v_new, pos)
+    gK, gV, gk, gv, gp = Guarded(K), Guarded(V), Guarded(k_new), Guarded(v_new), Guarded(pos)
+    moa.moa_kv_append(gK.ptr, gV.ptr, gk.ptr, gv.ptr, gp.ptr, B, hkv, n_max, dk, dv)
+    assert moa.moa_device_status() == 0
+    assert np.array_equal(gK.host().view(np.uint32), Kr.view(np.uint32))
+    assert np.array_equal(gV.host().view(np.uint32), Vr.view(np.uint32))
+    for g in (gK, gV, gk, gv, gp):
+        assert g.guards_intact()
+    assert np.array_equal(gp.host(), pos)                     # the library never advances pos
+
+
+def test_append_out_of_range_position_is_skipped_and_reported():
+    B, hkv, n_max, d = 3, 2, 4, 8
+    K, V = mi.normal(901, 2, (B, hkv, n_max, d)), mi.normal(901, 3, (B, hkv, n_max, d))
+    k_new, v_new = mi.normal(901, 4, (B, hkv, d)), mi.normal(901, 5, (B, hkv, d))
+    pos = np.array([4, 1, -1], np.int32)
+    gK, gV, gk, gv, gp = Guarded(K), Guarded(V), Guarded(k_new), Guarded(v_new), Guarded(pos)
+    moa.moa_kv_append(gK.ptr, gV.ptr, gk.ptr, gv.ptr, gp.ptr, B, hkv, n_max, d, d)
+    assert moa.moa_device_status() == moa.STATUS_APPEND_RANGE
+    Kr, Vr = K.copy(), V.copy()
+    oracle.kv_append(Kr[1:2], Vr[1:2], k_new[1:2], v_new[1:2], pos[1:2])
+    assert np.array_equal(gK.host().view(np.uint32), Kr.view(np.uint32))
+    assert np.array_equal(gV.host().view(np.uint32), Vr.view(np.uint32))
+    assert gK.guards_intact() and gV.guards_intact()
+
+
+# ---------------------------------------------------------------------------------------
+# multi-step decode: append then attend, token by token
+# ---------------------------------------------------------------------------------------
+@pytest.mark.parametrize("fused", [True, False])
+@pytest.mark.parametrize("D,hq,hkv", [(128, 8, 2), (64, 2, 1), (16, 4, 4)])
+def test_multistep_small(fused, D, hq, hkv):
+    w = mi.Workload("ms", 950 + D, 4, hq, hkv, 80, D, D, steps=40, len_lo=1, len_hi=40)
+    B, n_max = w.batch, w.n
+    lens = w.start_lens()
+    K, V = w.K(), w.V()
+    for b in range(B):
+        K[b, :, lens[b]:] = 0
+        V[b, :, lens[b]:] = 0
+    gK, gV, glens = Guarded(K), Guarded(V), Guarded(lens)
+    gws, nbytes = workspace_for(B, hq, hkv, n_max, D, D)
+    gout = Guarded(shape=(B, hq, D))
+    for t in range(w.steps):
+        kn, vn, qt = w.k_new(t), w.v_new(t), w.q_step(t)
+        gk, gv, gq = Guarded(kn), Guarded(vn), Guarded(qt)
+        if fused:
+            moa.moa_decode_step(gq.ptr, gK.ptr, gV.ptr, gk.ptr, gv.ptr, gout.ptr, glens.ptr, B, hq, hkv,
+                                n_max, D, D, w.scale, gws.ptr, nbytes)
+        else:
+            moa.moa_kv_append(gK.ptr, gV.ptr, gk.ptr, gv.ptr, glens.ptr, B, hkv, n_max, D, D)
+            moa.moa_lens_add(glens.ptr, B, 1)
+            moa.moa_decode_attn_varlen(gq.ptr, gK.ptr, gV.ptr, gout.ptr, B, hq, hkv, glens.ptr, n_max,
+                                       D, D, w.scale, gws.ptr, nbytes)
+        oracle.kv_append(K, V, kn, vn, lens)
+        lens = lens + 1
+        ref = oracle.decode_varlen(qt, K, V, lens, w.scale)
+        assert max_err(gout.host(), ref) <= TOL, t
+        assert np.array_equal(glens.host(), lens)
+    assert moa.moa_device_status() == 0
+    assert np.array_equal(gK.host().view(np.uint32), K.view(np.uint32))
+    assert np.array_equal(gV.host().view(np.uint32), V.view(np.uint32))
+    for g in (gK, gV, glens, gws, gout):
+        assert g.guards_intact()
+
+
+def test_fused_step_at_capacity_skips_and_keeps_length():
+    B, hq, hkv, n_max, D = 2, 4, 2, 8, 128
+    q, K, V, s = make(960, B, hq, hkv, n_max, D, D)
+    lens = np.array([8, 3], np.int32)                       # item 0 is full
+    kn, vn = mi.normal(960, 4, (B, hkv, D)), mi.normal(960, 5, (B, hkv, D))
+    gq, gK, gV, gk, gv, glens = Guarded(q), Guarded(K), Guarded(V), Guarded(kn), Guarded(vn), Guarded(lens)
+    gout = Guarded(shape=(B, hq, D), fill=-7.0)
+    gws, nbytes = workspace_for(B, hq, hkv, n_max, D, D)
+    moa.moa_decode_step(gq.ptr, gK.ptr, gV.ptr, gk.ptr, gv.ptr, gout.ptr, glens.ptr, B, hq, hkv, n_max,
+                        D, D, s, gws.ptr, nbytes)
+    st = moa.moa_device_status()
+    assert st == (moa.STATUS_APPEND_RANGE | moa.STATUS_SEQLEN_RANGE)
+    assert list(glens.host()) == [8, 4]
+    assert np.all(gout.host()[0] == -7.0)
+    assert np.array_equal(gK.host()[0].view(np.uint32), K[0].view(np.uint32))
+    oracle.kv_append(K[1:], V[1:], kn[1:], vn[1:], lens[1:])
+    ref = oracle.decode_varlen(q[1:], K[1:], V[1:], np.array([4], np.int32), s)
+    assert max_err(gout.host()[1:], ref) <= TOL
+
+
+# ---------------------------------------------------------------------------------------
+# argument errors never launch anything
+# ---------------------------------------------------------------------------------------
+def test_argument_errors():
+    q, K, V, s = make(970, 1, 4, 2, 16, 128, 128)
+    gq, gK, gV = Guarded(q), Guarded(K), Guarded(V)
+    gout = Guarded(shape=(1, 4, 128), fill=-7.0)
+    L = moa.lib()
+    st = torch.cuda.current_stream().cuda_stream
+    assert L.moa_decode_attn(None, gK.ptr, gV.ptr, gout.ptr, 1, 4, 2, 16, 128, 128, s, st) == moa.ERR_INVALID
+    assert L.moa_decode_attn(gq.ptr, gK.ptr, gV.ptr, gout.ptr, 1, 4, 3, 16, 128, 128, s, st) == moa.ERR_INVALID
+    assert L.moa_decode_attn(gq.ptr, gK.ptr, gV.ptr, gout.ptr, 1, 4, 2, 0, 128, 128, s, st) == moa.ERR_INVALID
+    assert L.moa_decode_attn(gq.ptr, gK.ptr, gV.ptr, gout.ptr, 1, 4, 2, 16, 128, 128, float("nan"), st) == moa.ERR_INVALID
+    assert L.moa_decode_attn(gq.ptr, gK.ptr, gV.ptr, gout.ptr, 1, 4, 2, 16, 2048, 128, s, st) == moa.ERR_UNSUPPORTED
+    assert L.moa_decode_attn(gq.ptr + 2, gK.ptr, gV.ptr, gout.ptr, 1, 4, 2, 16, 128, 128, s, st) == moa.ERR_ALIGN
+    assert L.moa_decode_attn_varlen(gq.ptr, gK.ptr, gV.ptr, gout.ptr, 1, 4, 2, None, 16, 128, 128, s,
+                                    None, 0, st) == moa.ERR_WORKSPACE
+    torch.cuda.synchronize()
+    assert np.all(gout.host() == -7.0)
