@@ -157,6 +157,22 @@ const char *moa_strerror(int code);
 int moa_set_option(int option, int value);
 int moa_last_path(void);
 
+/*
+ * Launch accounting for benchmarks (host-only state plus CUDA events; off by default).
+ * moa_profile(1) clears the counters and starts counting every kernel the library
+ * launches; while on, each launch of the dominant decode kernel (streaming, grouped or
+ * generic) is also bracketed by a pair of CUDA events on the caller's stream (at most
+ * MOA_PROFILE_MAX_EVENTS pairs are kept; later launches are counted but not timed).
+ * moa_profile_read synchronises the device and reports the summed event time of the
+ * timed decode-kernel launches in milliseconds, how many of them were timed, and the
+ * total number of kernels launched since moa_profile(1).  Any pointer may be NULL.
+ * moa_profile(0) stops counting.
+ */
+#define MOA_PROFILE_MAX_EVENTS 8192
+int moa_profile(int enable);
+int moa_profile_read(double *decode_kernel_ms, long long *decode_kernel_launches,
+                     long long *all_kernel_launches);
+
 #ifdef __cplusplus
 }
 #endif

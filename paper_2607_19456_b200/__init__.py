@@ -52,6 +52,9 @@ def lib():
         L.moa_strerror.argtypes = [i]
         L.moa_strerror.restype = C.c_char_p
         L.moa_set_option.argtypes = [i, i]
+        L.moa_profile.argtypes = [i]
+        L.moa_profile_read.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_longlong),
+                                       C.POINTER(C.c_longlong)]
         _lib = L
     return _lib
 
@@ -151,3 +154,14 @@ def moa_set_option(option: int, value: int):
 
 def moa_last_path() -> int:
     return int(lib().moa_last_path())
+
+
+def moa_profile(enable: int):
+    _check(lib().moa_profile(int(enable)), "moa_profile")
+
+
+def moa_profile_read():
+    """-> (decode_kernel_ms, decode_kernel_launches_timed, all_kernel_launches)."""
+    ms, n, a = C.c_double(0), C.c_longlong(0), C.c_longlong(0)
+    _check(lib().moa_profile_read(C.byref(ms), C.byref(n), C.byref(a)), "moa_profile_read")
+    return ms.value, n.value, a.value

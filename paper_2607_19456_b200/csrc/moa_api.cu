@@ -28,6 +28,35 @@ static int g_force_path = 0;
 static int g_num_ctas = 0;
 static int g_last_path = 0;
 
+// ---- launch accounting (moa_profile) ----------------------------------------------------
+static bool g_prof_on = false;
+static long long g_prof_all = 0;          // kernels launched while profiling
+static long long g_prof_timed = 0;        // decode-kernel launches bracketed by events
+static cudaEvent_t *g_prof_ev = nullptr;  // 2 * MOA_PROFILE_MAX_EVENTS events, created lazily
+
+struct TimedLaunch {                      // RAII: event before / after the dominant kernel
+    cudaStream_t st;
+    long long slot = -1;
+    explicit TimedLaunch(cudaStream_t s) : st(s)
+    {
+        if (!g_prof_on || g_prof_timed >= MOA_PROFILE_MAX_EVENTS) return;
+        if (!g_prof_ev) {
+            g_prof_ev = new cudaEvent_t[2 * MOA_PROFILE_MAX_EVENTS]();
+            for (int i = 0; i < 2 * MOA_PROFILE_MAX_EVENTS; ++i)
+                if (cudaEventCreate(&g_prof_ev[i]) != cudaSuccess) { cudaGetLastError(); g_prof_ev[i] = nullptr; }
+        }
+        slot = g_prof_timed;
+        if (g_prof_ev[2 * slot]) cudaEventRecord(g_prof_ev[2 * slot], st);
+    }
+    ~TimedLaunch()
+    {
+        if (slot < 0) return;
+        if (g_prof_ev[2 * slot + 1]) cudaEventRecord(g_prof_ev[2 * slot + 1], st);
+        ++g_prof_timed;
+    }
+};
+static inline void count_launch(int n = 1) { if (g_prof_on) g_prof_all += n; }
+
 static int current_device(DeviceState **st)
 {
     int dev = -1;
@@ -118,7 +147,11 @@ static cudaError_t launch_stream_cfg(const DecodeArgs &a, int num_ctas, cudaStre
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
-    stream_decode_kernel<C><<<num_ctas, C::THREADS, C::SMEM_BYTES, st>>>(a);
+    {
+        TimedLaunch t(st);
+        stream_decode_kernel<C><<<num_ctas, C::THREADS, C::SMEM_BYTES, st>>>(a);
+    }
+    count_launch(2);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     const long long warps = (long long)a.batch * a.h_q;
@@ -152,10 +185,15 @@ static cudaError_t launch_generic(const DecodeArgs &a, cudaStream_t st)
     const size_t smem = sizeof(float) * ((size_t)a.d_k + (size_t)kGenericWarps * a.d_v + 2 * kGenericWarps);
     if (a.seq_lens != nullptr) {
         check_lens_kernel<<<(a.batch + 127) / 128, 128, 0, st>>>(a.seq_lens, a.len_bias, a.batch, a.n_max);
+        count_launch();
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
-    generic_decode_kernel<<<a.batch * a.h_q, kGenericWarps * 32, smem, st>>>(a);
+    {
+        TimedLaunch t(st);
+        generic_decode_kernel<<<a.batch * a.h_q, kGenericWarps * 32, smem, st>>>(a);
+    }
+    count_launch();
     return cudaGetLastError();
 }
 
@@ -273,6 +311,7 @@ int moa_kv_append(float *K, float *V, const float *k_new, const float *v_new, co
         reinterpret_cast<uint32_t *>(K), reinterpret_cast<uint32_t *>(V),
         reinterpret_cast<const uint32_t *>(k_new), reinterpret_cast<const uint32_t *>(v_new), pos,
         batch, h_kv, n_max, d_k, d_v);
+    count_launch();
     return cudaGetLastError() == cudaSuccess ? MOA_OK : MOA_ERR_CUDA;
 }
 
@@ -284,6 +323,7 @@ int moa_lens_add(int32_t *lens, int batch, int delta, void *stream)
     int rc = current_device(&dev);
     if (rc != MOA_OK) return rc;
     lens_add_kernel<<<(batch + 127) / 128, 128, 0, static_cast<cudaStream_t>(stream)>>>(lens, batch, delta, 0);
+    count_launch();
     return cudaGetLastError() == cudaSuccess ? MOA_OK : MOA_ERR_CUDA;
 }
 
@@ -314,6 +354,7 @@ int moa_decode_step(const float *q, float *K, float *V, const float *k_new, cons
                      workspace_bytes, false, st);
     if (rc != MOA_OK) return rc;
     lens_add_kernel<<<(batch + 127) / 128, 128, 0, st>>>(lens, batch, 1, n_max);
+    count_launch();
     return cudaGetLastError() == cudaSuccess ? MOA_OK : MOA_ERR_CUDA;
 }
 
@@ -433,5 +474,34 @@ int moa_set_option(int option, int value)
 }
 
 int moa_last_path(void) { return g_last_path; }
+
+int moa_profile(int enable)
+{
+    g_prof_on = enable != 0;
+    if (g_prof_on) { g_prof_all = 0; g_prof_timed = 0; }
+    return MOA_OK;
+}
+
+int moa_profile_read(double *decode_kernel_ms, long long *decode_kernel_launches,
+                     long long *all_kernel_launches)
+{
+    if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return MOA_ERR_CUDA; }
+    double ms = 0.0;
+    long long timed = 0;
+    for (long long i = 0; i < g_prof_timed; ++i) {
+        float t = 0.f;
+        if (g_prof_ev && g_prof_ev[2 * i] && g_prof_ev[2 * i + 1] &&
+            cudaEventElapsedTime(&t, g_prof_ev[2 * i], g_prof_ev[2 * i + 1]) == cudaSuccess) {
+            ms += t;
+            ++timed;
+        } else {
+            cudaGetLastError();
+        }
+    }
+    if (decode_kernel_ms) *decode_kernel_ms = ms;
+    if (decode_kernel_launches) *decode_kernel_launches = timed;
+    if (all_kernel_launches) *all_kernel_launches = g_prof_all;
+    return MOA_OK;
+}
 
 }  // extern "C"
