@@ -125,6 +125,41 @@ int moa_decode_attn_host(const float *q, const float *K, const float *V, float *
                          int batch, int h_q, int h_kv, int n, int d_k, int d_v,
                          float scale);
 
+/*
+ * Decode attention for callers that must not allocate device memory.  (The paper has no
+ * counterpart to this entry point; it exists for deployment reasons only.)
+ *
+ * Who needs it: code that runs after a process has handed all of its device memory to
+ * a framework's pooling allocator (a cudaMalloc issued then fails or fragments the pool),
+ * code inside a latency-critical serving loop where the implicit device-wide
+ * synchronisation of cudaMalloc/cudaFree would stall every other stream, and plug-in
+ * callbacks whose host framework forbids allocation calls while its own work is in
+ * flight.  moa_decode_attn may call cudaMalloc on its first use (or when a larger problem
+ * arrives) and moa_decode_attn_varlen pushes the scratch buffer onto the caller; this
+ * variant does neither.
+ *
+ * Same arguments, layouts, results and return codes as moa_decode_attn.  The scratch for
+ * the split-sequence partial results lives in a fixed array of
+ * MOA_NOALLOC_SCRATCH_BYTES bytes that is part of the library image: every GPU that
+ * loads the library holds that much memory until the process exits.  The call issues no
+ * cudaMalloc, cudaFree or other allocating routine.
+ *  - A problem whose scratch need exceeds MOA_NOALLOC_SCRATCH_BYTES (only possible when
+ *    MOA_OPT_NUM_CTAS was raised far above the SM count) is rejected with
+ *    MOA_ERR_CAPACITY before anything is launched.
+ *  - The first call on each device looks up the device address of the array (one
+ *    cudaGetSymbolAddress with that device current) and keeps it; make that first call
+ *    before starting any stream capture on that device.
+ *  - The array is shared by every call on the device and keeps whatever the previous call
+ *    left in it.  Nothing in it has to start at zero: each call writes every slot it later
+ *    reads.  Two calls that can overlap on the GPU (different streams, no dependency
+ *    between them) would race on it; order them, or give one of them its own workspace
+ *    through moa_decode_attn_varlen.
+ */
+#define MOA_NOALLOC_SCRATCH_BYTES (2u << 20)
+int moa_decode_attn_noalloc(const float *q, const float *K, const float *V, float *out,
+                            int batch, int h_q, int h_kv, int n, int d_k, int d_v,
+                            float scale, void *stream);
+
 /* Synchronise `stream`, copy the device status word to *status_out (HOST int) and
  * clear it.  Zero means no kernel of this library reported a problem since the last
  * call. */

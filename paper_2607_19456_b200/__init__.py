@@ -18,6 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libmoa.so")
 OK, ERR_INVALID, ERR_UNSUPPORTED, ERR_ALIGN, ERR_CAPACITY, ERR_WORKSPACE, ERR_CUDA = range(7)
 STATUS_APPEND_RANGE, STATUS_SEQLEN_RANGE, STATUS_WAIT_TIMEOUT = 1, 2, 4
 OPT_FORCE_PATH, OPT_NUM_CTAS = 1, 2
+NOALLOC_SCRATCH_BYTES = 2 << 20
 PATH_AUTO, PATH_GENERIC, PATH_STREAM, PATH_GROUPED = 0, 1, 2, 3
 
 _lib = None
@@ -39,6 +40,7 @@ def lib():
         L = C.CDLL(LIB_PATH)
         p, i, f, sz = C.c_void_p, C.c_int, C.c_float, C.c_size_t
         L.moa_decode_attn.argtypes = [p, p, p, p, i, i, i, i, i, i, f, p]
+        L.moa_decode_attn_noalloc.argtypes = [p, p, p, p, i, i, i, i, i, i, f, p]
         L.moa_decode_attn_varlen.argtypes = [p, p, p, p, i, i, i, p, i, i, i, f, p, sz, p]
         L.moa_workspace_bytes.argtypes = [i, i, i, i, i, i]
         L.moa_workspace_bytes.restype = sz
@@ -93,6 +95,13 @@ def strerror(code: int) -> str:
 def moa_decode_attn(q, K, V, out, batch, h_q, h_kv, n, d_k, d_v, scale, stream=None):
     _check(lib().moa_decode_attn(_ptr(q), _ptr(K), _ptr(V), _ptr(out), batch, h_q, h_kv, n, d_k,
                                  d_v, scale, _stream(stream)), "moa_decode_attn")
+
+
+def moa_decode_attn_noalloc(q, K, V, out, batch, h_q, h_kv, n, d_k, d_v, scale, stream=None):
+    """Same as :func:`moa_decode_attn`, for callers that may not allocate device memory:
+    scratch comes from a fixed array inside the library (see ``include/moa.h``)."""
+    _check(lib().moa_decode_attn_noalloc(_ptr(q), _ptr(K), _ptr(V), _ptr(out), batch, h_q, h_kv, n,
+                                         d_k, d_v, scale, _stream(stream)), "moa_decode_attn_noalloc")
 
 
 def moa_decode_attn_varlen(q, K, V, out, batch, h_q, h_kv, seq_lens, n_max, d_k, d_v, scale,

@@ -260,6 +260,12 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
     return MOA_OK;
 }
 
+// ---- fixed scratch for the allocation-free entry point ---------------------------------
+// Lives in the library image; the host-side name below is only a handle for
+// cudaGetSymbolAddress, never a pointer a kernel may be given.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[MOA_NOALLOC_SCRATCH_BYTES];
+static void *g_noalloc_scratch_dev[kMaxDevices] = {};   // resolved device address, per device
+
 }  // namespace moa
 
 using namespace moa;
@@ -271,6 +277,43 @@ int moa_decode_attn(const float *q, const float *K, const float *V, float *out, 
 {
     return decode_impl(q, K, V, out, batch, h_q, h_kv, nullptr, 0, n, d_k, d_v, scale, nullptr, 0,
                        true, static_cast<cudaStream_t>(stream));
+}
+
+int moa_decode_attn_noalloc(const float *q, const float *K, const float *V, float *out, int batch,
+                            int h_q, int h_kv, int n, int d_k, int d_v, float scale, void *stream)
+{
+    // Argument errors first, exactly as the allocating entry point reports them.
+    if (!q || !K || !V || !out) return MOA_ERR_INVALID;
+    int rc = validate_dims(batch, h_q, h_kv, n, d_k, d_v);
+    if (rc != MOA_OK) return rc;
+    DeviceState *dev = nullptr;
+    rc = current_device(&dev);
+    if (rc != MOA_OK) return rc;
+    int device = 0;
+    if (cudaGetDevice(&device) != cudaSuccess) { cudaGetLastError(); return MOA_ERR_CUDA; }
+    // One-time set-up on this device (it is the current one): turn the array's host-side
+    // handle into the address kernels can use.
+    if (g_noalloc_scratch_dev[device] == nullptr) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || p == nullptr) {
+            cudaGetLastError();
+            return MOA_ERR_CUDA;
+        }
+        g_noalloc_scratch_dev[device] = p;
+    }
+    // Refuse problems whose partial-result slots would not fit the fixed array.
+    const StreamPlan plan = plan_stream(h_q / h_kv, d_k, d_v);
+    if (plan.ok && stream_ws_bytes(plan, stream_num_ctas(*dev)) > (size_t)MOA_NOALLOC_SCRATCH_BYTES)
+        return MOA_ERR_CAPACITY;
+    // The launch-accounting hooks create their CUDA events lazily; keep that (an
+    // allocation of driver objects) out of this call if it has not happened yet.
+    const bool prof_saved = g_prof_on;
+    if (g_prof_ev == nullptr) g_prof_on = false;
+    rc = decode_impl(q, K, V, out, batch, h_q, h_kv, nullptr, 0, n, d_k, d_v, scale,
+                     g_noalloc_scratch_dev[device], (size_t)MOA_NOALLOC_SCRATCH_BYTES, false,
+                     static_cast<cudaStream_t>(stream));
+    g_prof_on = prof_saved;
+    return rc;
 }
 
 int moa_decode_attn_varlen(const float *q, const float *K, const float *V, float *out, int batch,
