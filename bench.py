@@ -69,7 +69,10 @@ class ClockSampler:
                0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown",
                0x100: "display_clock_setting"}
 
-    def __init__(self, index):
+    def __init__(self, index, interval=0.02):
+        # NVML queries go through the driver; polling them every couple of milliseconds
+        # measurably slows the kernels being timed, so sample sparsely.
+        self.interval = interval
         self.samples, self.reasons, self.max_mhz = [], set(), None
         self._stop = threading.Event()
         self._thr = None
@@ -105,7 +108,7 @@ class ClockSampler:
                         self.reasons.add(name)
             except Exception:
                 pass
-            self._stop.wait(0.002)
+            self._stop.wait(self.interval)
 
     def start(self):
         if self.nv is not None:
@@ -171,16 +174,21 @@ class DenseRun:
         self.out = torch.zeros((S, B, hq, dv), device=device)
         self.pos = torch.full((B,), n - 1, dtype=torch.int32, device=device)
         self.i = 0
+        # raw addresses, so that the timed loop does no tensor indexing on the host
+        self.ptrs = [(self.q[s].data_ptr(), self.K[s].data_ptr(), self.V[s].data_ptr(),
+                      self.out[s].data_ptr()) for s in range(S)]
+        self.aux = (self.k_new.data_ptr(), self.v_new.data_ptr(), self.pos.data_ptr())
+        self.stream = torch.cuda.current_stream().cuda_stream
         self.l2_note = ("inputs larger than L2 (%.0f MB per step)" % (one / 1e6)) if S == 1 else \
             ("rotating over %d buffer sets (%.0f MB total, larger than L2)" % (S, S * one / 1e6))
 
     def step(self):
-        w, m, s = self.w, self.moa, self.i % self.nsets
+        w, m = self.w, self.moa
+        q, K, V, out = self.ptrs[self.i % self.nsets]
+        kn, vn, pos = self.aux
         self.i += 1
-        m.moa_kv_append(self.K[s], self.V[s], self.k_new, self.v_new, self.pos, w.batch, w.h_kv, w.n,
-                        w.d_k, w.d_v)
-        m.moa_decode_attn(self.q[s], self.K[s], self.V[s], self.out[s], w.batch, w.h_q, w.h_kv, w.n,
-                          w.d_k, w.d_v, w.scale)
+        m.moa_kv_append(K, V, kn, vn, pos, w.batch, w.h_kv, w.n, w.d_k, w.d_v, self.stream)
+        m.moa_decode_attn(q, K, V, out, w.batch, w.h_q, w.h_kv, w.n, w.d_k, w.d_v, w.scale, self.stream)
 
     def reset(self):
         self.i = 0
@@ -222,6 +230,11 @@ class MultiStepRun:
         self.wsbuf = torch.empty(self.ws_bytes, dtype=torch.uint8, device=device)
         self.t = 0
         self.nsets = 1
+        self.step_ptrs = [(self.q[t].data_ptr(), self.k_new[t].data_ptr(), self.v_new[t].data_ptr())
+                          for t in range(T)]
+        self.fix_ptrs = (self.K.data_ptr(), self.V.data_ptr(), self.out.data_ptr(), self.lens.data_ptr(),
+                         self.wsbuf.data_ptr())
+        self.stream = torch.cuda.current_stream().cuda_stream
         self.l2_note = "every step streams the whole live cache (about 400 MB, larger than L2)"
 
     def bytes_for_steps(self, t0, t1):
@@ -237,8 +250,10 @@ class MultiStepRun:
         w, m, t = self.w, self.moa, self.t
         if t >= w.steps:
             raise RuntimeError("multi_step: warmup + steps must not exceed %d" % w.steps)
-        m.moa_decode_step(self.q[t], self.K, self.V, self.k_new[t], self.v_new[t], self.out, self.lens,
-                          w.batch, w.h_q, w.h_kv, w.n, w.d_k, w.d_v, w.scale, self.wsbuf, self.ws_bytes)
+        q, kn, vn = self.step_ptrs[t]
+        K, V, out, lens, wsb = self.fix_ptrs
+        m.moa_decode_step(q, K, V, kn, vn, out, lens, w.batch, w.h_q, w.h_kv, w.n, w.d_k, w.d_v, w.scale,
+                          wsb, self.ws_bytes, self.stream)
         self.t += 1
 
     def reset(self):
@@ -363,13 +378,15 @@ def run_reference(args, wname):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=list(mi.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-others", action="store_true", help="skip the timing-only lines of the other workloads")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling on a small case)")
+    ap.add_argument("--n", type=int, default=0, help="override the workload's cached tokens (profiling on a small case)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -393,6 +410,10 @@ def main():
     moa.lib()                                           # fail loudly if the library is missing
 
     w = mi.WORKLOADS[wname]
+    if args.batch > 0:
+        w = mi.small_like(w, batch=args.batch)
+    if args.n > 0 and wname != "multi_step":
+        w = mi.small_like(w, n=args.n)
     if wname == "multi_step":
         args.steps = min(args.steps, w.steps - args.warmup)
         run = MultiStepRun(w, seed_shift=rank)
