@@ -294,18 +294,15 @@ _DIST = {"on": False}
 
 def barrier():
     if _DIST["on"]:
-        import torch.distributed as dist
-        dist.barrier()
+        from paper_2607_19456_b200 import shard
+        shard.barrier()
 
 
 def max_over_ranks(x):
     if not _DIST["on"]:
         return x
-    import torch
-    import torch.distributed as dist
-    t = torch.tensor([x], dtype=torch.float64, device="cuda")
-    dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    return float(t.item())
+    from paper_2607_19456_b200 import shard
+    return shard.reduce_step_time(x, device="cuda")
 
 
 # --------------------------------------------------------------------------------------
