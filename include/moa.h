@@ -109,11 +109,25 @@ int moa_lens_add(int32_t *lens, int batch, int delta, void *stream);
  * lens is a device int32[batch] that the call updates; all other arguments as above.
  * Requires lens[b] in [0, n_max-1]; otherwise the status bits above are set, the item
  * is skipped and its length is left unchanged.
+ * For d_k == d_v in {64, 128} and 16-byte-aligned pointers all three parts run in one
+ * kernel launch (the streaming kernel takes the new row from k_new/v_new, stores it into
+ * the cache, and the last CTA to finish advances the lengths); otherwise in three.
+ * `workspace` as for moa_decode_attn_varlen.
  */
 int moa_decode_step(const float *q, float *K, float *V, const float *k_new,
                     const float *v_new, float *out, int32_t *lens,
                     int batch, int h_q, int h_kv, int n_max, int d_k, int d_v, float scale,
                     void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * The same step without touching the lengths: append (k_new, v_new) at row pos[b], then
+ * attend q over rows [0, pos[b]+1).  pos is a device int32[batch] that is only read.
+ * (Eqs. (4),(5) followed by Algorithm 1 on the extended cache.)
+ */
+int moa_append_decode(const float *q, float *K, float *V, const float *k_new,
+                      const float *v_new, float *out, const int32_t *pos,
+                      int batch, int h_q, int h_kv, int n_max, int d_k, int d_v, float scale,
+                      void *workspace, size_t workspace_bytes, void *stream);
 
 /*
  * Host-buffer convenience call: q, K, V, out are HOST pointers (pinned memory gives
@@ -182,10 +196,13 @@ const char *moa_strerror(int code);
  *                        a forced path that cannot handle the shape returns
  *                        MOA_ERR_UNSUPPORTED.
  *   MOA_OPT_NUM_CTAS   : 0 = one streaming CTA per SM, otherwise that many.
+ *   MOA_OPT_GROUPED_HEADS : query heads per CTA of the tensor-core kernel (16, 32 or 64;
+ *                        0 = automatic).  Larger groups are cut into neighbouring CTAs.
  * moa_last_path() reports which kernel family the last successful decode call used.
  */
 #define MOA_OPT_FORCE_PATH 1
 #define MOA_OPT_NUM_CTAS   2
+#define MOA_OPT_GROUPED_HEADS 3
 #define MOA_PATH_GENERIC   1   /* any d_k, d_v, alignment: one CTA per (batch, query head) */
 #define MOA_PATH_STREAM    2   /* split-sequence streaming kernel, g_s <= 8, d in {64,128} */
 #define MOA_PATH_GROUPED   3   /* tensor-core kernel for large groups (g_s >= 16) */

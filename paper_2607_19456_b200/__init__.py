@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libmoa.so")
 
 OK, ERR_INVALID, ERR_UNSUPPORTED, ERR_ALIGN, ERR_CAPACITY, ERR_WORKSPACE, ERR_CUDA = range(7)
 STATUS_APPEND_RANGE, STATUS_SEQLEN_RANGE, STATUS_WAIT_TIMEOUT = 1, 2, 4
-OPT_FORCE_PATH, OPT_NUM_CTAS = 1, 2
+OPT_FORCE_PATH, OPT_NUM_CTAS, OPT_GROUPED_HEADS = 1, 2, 3
 NOALLOC_SCRATCH_BYTES = 2 << 20
 PATH_AUTO, PATH_GENERIC, PATH_STREAM, PATH_GROUPED = 0, 1, 2, 3
 
@@ -47,6 +47,7 @@ def lib():
         L.moa_kv_append.argtypes = [p, p, p, p, p, i, i, i, i, i, p]
         L.moa_lens_add.argtypes = [p, i, i, p]
         L.moa_decode_step.argtypes = [p, p, p, p, p, p, p, i, i, i, i, i, i, f, p, sz, p]
+        L.moa_append_decode.argtypes = [p, p, p, p, p, p, p, i, i, i, i, i, i, f, p, sz, p]
         L.moa_decode_attn_host.argtypes = [p, p, p, p, i, i, i, i, i, i, f]
         L.moa_device_status.argtypes = [p, C.POINTER(C.c_int)]
         L.moa_min_bytes.argtypes = [i, i, i, C.c_longlong, i, i]
@@ -131,6 +132,14 @@ def moa_decode_step(q, K, V, k_new, v_new, out, lens, batch, h_q, h_kv, n_max, d
                                  _ptr(lens), batch, h_q, h_kv, n_max, d_k, d_v, scale,
                                  _ptr(workspace), workspace_bytes, _stream(stream)),
            "moa_decode_step")
+
+
+def moa_append_decode(q, K, V, k_new, v_new, out, pos, batch, h_q, h_kv, n_max, d_k, d_v, scale,
+                      workspace, workspace_bytes, stream=None):
+    _check(lib().moa_append_decode(_ptr(q), _ptr(K), _ptr(V), _ptr(k_new), _ptr(v_new), _ptr(out),
+                                   _ptr(pos), batch, h_q, h_kv, n_max, d_k, d_v, scale,
+                                   _ptr(workspace), workspace_bytes, _stream(stream)),
+           "moa_append_decode")
 
 
 def moa_decode_attn_host(q, K, V, out, batch, h_q, h_kv, n, d_k, d_v, scale):

@@ -9,6 +9,7 @@
 #include "moa_device.cuh"
 #include "moa_generic.cuh"
 #include "moa_stream.cuh"
+#include "moa_grouped.cuh"
 
 namespace moa {
 
@@ -22,6 +23,8 @@ struct DeviceState {
     void *stage[4] = {nullptr, nullptr, nullptr, nullptr};   // host-API staging: q K V out
     size_t stage_bytes[4] = {0, 0, 0, 0};
     cudaStream_t host_stream = nullptr;
+    unsigned *tickets = nullptr;  // device address of g_tickets (resolved once)
+    unsigned ticket_seq = 0;      // launches so far: picks the counter slot round-robin
 };
 static DeviceState g_dev[kMaxDevices];
 static int g_force_path = 0;
@@ -129,6 +132,17 @@ static StreamPlan plan_stream(int g_s, int d_k, int d_v)
 
 static int stream_num_ctas(const DeviceState &s) { return g_num_ctas > 0 ? g_num_ctas : s.sm_count; }
 
+// CTAs actually launched: never more than one per 8 row blocks (one block per warp), so
+// that small problems are not cut into partials that then have to be merged.
+static int stream_grid(const DeviceState &s, const StreamPlan &p, int batch, int h_kv, int n_max)
+{
+    const int cap = stream_num_ctas(s);
+    if (g_num_ctas > 0) return cap;
+    const long long blocks = (long long)batch * h_kv * p.share * ((n_max + p.R - 1) / p.R);
+    const long long want = (blocks + 7) / 8;
+    return (int)(want < cap ? (want < 1 ? 1 : want) : cap);
+}
+
 static size_t stream_ws_bytes(const StreamPlan &p, int num_ctas)
 {
     return (size_t)num_ctas * 2 * p.G * (p.D + 4) * sizeof(float);
@@ -151,12 +165,13 @@ static cudaError_t launch_stream_cfg(const DecodeArgs &a, int num_ctas, cudaStre
         TimedLaunch t(st);
         stream_decode_kernel<C><<<num_ctas, C::THREADS, C::SMEM_BYTES, st>>>(a);
     }
-    count_launch(2);
+    count_launch();
     cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
+    if (e != cudaSuccess || a.tickets != nullptr) return e;
     const long long warps = (long long)a.batch * a.h_q;
     const int blocks = (int)((warps + 3) / 4);
     stream_combine_kernel<C::D, C::R><<<blocks, 128, 0, st>>>(a, num_ctas, C::G);
+    count_launch();
     return cudaGetLastError();
 }
 
@@ -180,6 +195,102 @@ static cudaError_t launch_stream(const StreamPlan &p, const DecodeArgs &a, int n
     }
 }
 
+// ---- grouped (tensor-core) plan -----------------------------------------------------------
+struct GroupedPlan {
+    bool ok = false;
+    int GH = 0;          // query heads per CTA (per virtual kv head)
+    int share = 1;       // virtual kv heads per stored kv head
+    int splits = 1, tiles_per_split = 1;
+    size_t ws_bytes = 0;
+};
+static int g_grouped_heads = 0;   // MOA_OPT_GROUPED_HEADS: 0 = automatic
+
+static GroupedPlan plan_grouped(const DeviceState &s, int batch, int h_q, int h_kv, int n, int d_k, int d_v)
+{
+    GroupedPlan p;
+    const int g_s = h_q / h_kv;
+    if (d_k != 128 || d_v != 128 || (g_s != 16 && g_s != 32 && g_s != 64)) return p;
+    const long long units = (long long)batch * h_kv;
+    if (units > 0x7fffffffLL / 256 || (long long)n > 0x7fffffffLL - 256) return p;
+    // 32 heads per CTA leave room for a ten-deep chunk ring (64 heads: six), which is what
+    // hides the HBM latency; a group of 64 runs as two neighbouring CTAs over the same rows.
+    p.GH = g_s > 32 ? 32 : g_s;
+    if (g_grouped_heads == 16 || g_grouped_heads == 32 || g_grouped_heads == 64)
+        if (g_grouped_heads <= g_s) p.GH = g_grouped_heads;
+    p.share = g_s / p.GH;
+    const long long ctas_per_split = units * p.share;
+    const int tiles = (n + 127) / 128;
+    long long splits = ctas_per_split >= s.sm_count ? 1 : s.sm_count / ctas_per_split;
+    if (splits > tiles) splits = tiles;
+    p.splits = (int)splits;
+    p.tiles_per_split = (tiles + p.splits - 1) / p.splits;
+    p.ws_bytes = (size_t)units * p.share * p.splits * p.GH * 132 * sizeof(float);
+    p.ok = true;
+    return p;
+}
+
+typedef CUresult (*TmapEncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                 const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                 CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static TmapEncodeFn tmap_encoder()
+{
+    static TmapEncodeFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess) {
+            cudaGetLastError();
+            return nullptr;
+        }
+        fn = reinterpret_cast<TmapEncodeFn>(p);
+    }
+    return fn;
+}
+
+// Tensor map over a cache [units][n][128] fp32 with boxes of 32 features x box_rows rows.
+static bool make_cache_map(CUtensorMap *m, const float *base, long long units, int n, int box_rows,
+                           CUtensorMapSwizzle swz)
+{
+    TmapEncodeFn enc = tmap_encoder();
+    if (!enc) return false;
+    cuuint64_t dims[3] = {128, (cuuint64_t)n, (cuuint64_t)units};
+    cuuint64_t strides[2] = {512, (cuuint64_t)n * 512};
+    cuuint32_t box[3] = {32, (cuuint32_t)box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int GH>
+static cudaError_t launch_grouped_cfg(const CUtensorMap &mk, const CUtensorMap &mv, const GroupedArgs &ga,
+                                      int grid, cudaStream_t st)
+{
+    using C = GroupedCfg<GH>;
+    static bool attr_set[kMaxDevices] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (!attr_set[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(grouped_decode_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)C::SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        attr_set[dev] = true;
+    }
+    {
+        TimedLaunch t(st);
+        grouped_decode_kernel<C><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(mk, mv, ga);
+    }
+    count_launch();
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const long long warps = (long long)ga.batch * ga.h_q;
+    grouped_combine_kernel<GH><<<(int)((warps + 3) / 4), 128, 0, st>>>(ga);
+    count_launch();
+    return cudaGetLastError();
+}
+
 static cudaError_t launch_generic(const DecodeArgs &a, cudaStream_t st)
 {
     const size_t smem = sizeof(float) * ((size_t)a.d_k + (size_t)kGenericWarps * a.d_v + 2 * kGenericWarps);
@@ -199,10 +310,17 @@ static cudaError_t launch_generic(const DecodeArgs &a, cudaStream_t st)
 
 // Shared implementation of the decode entry points.  `ws` may be null when the chosen
 // path needs none.
+struct FusedStep {                 // extra work folded into the streaming launch
+    float *Kw = nullptr, *Vw = nullptr;
+    const float *k_new = nullptr, *v_new = nullptr;
+    int32_t *lens_rw = nullptr;
+};
+
 static int decode_impl(const float *q, const float *K, const float *V, float *out, int batch,
                        int h_q, int h_kv, const int32_t *seq_lens, int len_bias, int n_max,
                        int d_k, int d_v, float scale, void *ws, size_t ws_bytes,
-                       bool library_ws, cudaStream_t st)
+                       bool library_ws, cudaStream_t st, const FusedStep *fused = nullptr,
+                       bool allow_grouped = true)
 {
     if (!q || !K || !V || !out) return MOA_ERR_INVALID;
     int rc = validate_dims(batch, h_q, h_kv, n_max, d_k, d_v);
@@ -220,9 +338,17 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
     StreamPlan plan = plan_stream(g_s, d_k, d_v);
     const bool fast_ok = plan.ok && aligned(q, 16) && aligned(K, 16) && aligned(V, 16) && aligned(out, 16);
     int path = fast_ok ? MOA_PATH_STREAM : MOA_PATH_GENERIC;
+    // Large head groups over a dense cache go to the tensor cores.
+    GroupedPlan gplan;
+    if (fast_ok && allow_grouped && fused == nullptr && seq_lens == nullptr)
+        gplan = plan_grouped(*dev, batch, h_q, h_kv, n_max, d_k, d_v);
+    if (gplan.ok && (library_ws || (ws && ws_bytes >= gplan.ws_bytes))) path = MOA_PATH_GROUPED;
     if (g_force_path == MOA_PATH_GENERIC) path = MOA_PATH_GENERIC;
     else if (g_force_path == MOA_PATH_STREAM) {
         if (!fast_ok) return MOA_ERR_UNSUPPORTED;
+        path = MOA_PATH_STREAM;
+    } else if (g_force_path == MOA_PATH_GROUPED) {
+        if (path != MOA_PATH_GROUPED) return MOA_ERR_UNSUPPORTED;
     } else if (g_force_path != 0) return MOA_ERR_UNSUPPORTED;
 
     DecodeArgs a;
@@ -231,10 +357,37 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
     a.batch = batch; a.h_q = h_q; a.h_kv = h_kv; a.g_s = g_s; a.kv_share = 1;
     a.n_max = n_max; a.d_k = d_k; a.d_v = d_v;
     a.qscale = scale * kLog2e;
+    a.Kw = nullptr; a.Vw = nullptr; a.k_new = nullptr; a.v_new = nullptr; a.lens_rw = nullptr;
+    a.tickets = nullptr;
+    if (fused != nullptr && path != MOA_PATH_STREAM) return MOA_ERR_UNSUPPORTED;
 
     cudaError_t e;
-    if (path == MOA_PATH_STREAM) {
-        const int num_ctas = stream_num_ctas(*dev);
+    if (path == MOA_PATH_GROUPED) {
+        if (library_ws) {
+            if (dev->ws_bytes < gplan.ws_bytes) {
+                if (dev->ws) { cudaDeviceSynchronize(); cudaFree(dev->ws); dev->ws = nullptr; dev->ws_bytes = 0; }
+                if (cudaMalloc(&dev->ws, gplan.ws_bytes) != cudaSuccess) { cudaGetLastError(); return MOA_ERR_CUDA; }
+                dev->ws_bytes = gplan.ws_bytes;
+            }
+            ws = dev->ws;
+        } else if (!aligned(ws, 256)) return MOA_ERR_ALIGN;
+        CUtensorMap mk, mv;
+        const long long units = (long long)batch * h_kv;
+        if (!make_cache_map(&mk, K, units, n_max, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
+            !make_cache_map(&mv, V, units, n_max, 32, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B))
+            return MOA_ERR_CUDA;
+        GroupedArgs ga;
+        ga.q = q; ga.out = out; ga.ws = static_cast<float *>(ws);
+        ga.batch = batch; ga.h_q = h_q; ga.h_kv = h_kv * gplan.share; ga.n = n_max;
+        ga.h_kv_stored = h_kv; ga.share = gplan.share;
+        ga.splits = gplan.splits; ga.tiles_per_split = gplan.tiles_per_split;
+        ga.qscale = scale * kLog2e;
+        const int grid = (int)(units * gplan.share * gplan.splits);
+        if (gplan.GH == 16) e = launch_grouped_cfg<16>(mk, mv, ga, grid, st);
+        else if (gplan.GH == 32) e = launch_grouped_cfg<32>(mk, mv, ga, grid, st);
+        else e = launch_grouped_cfg<64>(mk, mv, ga, grid, st);
+    } else if (path == MOA_PATH_STREAM) {
+        const int num_ctas = stream_grid(*dev, plan, batch, h_kv, n_max);
         const size_t need = stream_ws_bytes(plan, num_ctas);
         if (library_ws) {
             if (dev->ws_bytes < need) {
@@ -248,6 +401,19 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
             if (!aligned(ws, 256)) return MOA_ERR_ALIGN;
         }
         a.ws = static_cast<float *>(ws);
+        if (num_ctas <= kTicketCtas) {      // merge partials inside the streaming launch
+            if (dev->tickets == nullptr) {
+                void *p = nullptr;
+                if (cudaGetSymbolAddress(&p, g_tickets) != cudaSuccess || !p) { cudaGetLastError(); return MOA_ERR_CUDA; }
+                dev->tickets = static_cast<unsigned *>(p);
+            }
+            a.tickets = dev->tickets + (size_t)(dev->ticket_seq++ % kTicketSlots) * kTicketStride;
+        }
+        if (fused != nullptr) {
+            if (a.tickets == nullptr && fused->lens_rw != nullptr) return MOA_ERR_UNSUPPORTED;
+            a.Kw = fused->Kw; a.Vw = fused->Vw; a.k_new = fused->k_new; a.v_new = fused->v_new;
+            a.lens_rw = fused->lens_rw;
+        }
         a.h_kv = h_kv * plan.share;        // virtual kv heads of plan.G query heads each
         a.g_s = (plan.share > 1) ? plan.G : g_s;
         a.kv_share = plan.share;
@@ -311,7 +477,7 @@ int moa_decode_attn_noalloc(const float *q, const float *K, const float *V, floa
     if (g_prof_ev == nullptr) g_prof_on = false;
     rc = decode_impl(q, K, V, out, batch, h_q, h_kv, nullptr, 0, n, d_k, d_v, scale,
                      g_noalloc_scratch_dev[device], (size_t)MOA_NOALLOC_SCRATCH_BYTES, false,
-                     static_cast<cudaStream_t>(stream));
+                     static_cast<cudaStream_t>(stream), nullptr, false);
     g_prof_on = prof_saved;
     return rc;
 }
@@ -333,7 +499,11 @@ size_t moa_workspace_bytes(int batch, int h_q, int h_kv, int n_max, int d_k, int
     DeviceState *dev = nullptr;
     int ctas = g_num_ctas;
     if (ctas <= 0) ctas = (current_device(&dev) == MOA_OK) ? dev->sm_count : 256;
-    const size_t need = stream_ws_bytes(plan, ctas);
+    size_t need = stream_ws_bytes(plan, ctas);
+    if (dev != nullptr || current_device(&dev) == MOA_OK) {
+        const GroupedPlan gp = plan_grouped(*dev, batch, h_q, h_kv, n_max, d_k, d_v);
+        if (gp.ok && gp.ws_bytes > need) need = gp.ws_bytes;
+    }
     return (need + 255) / 256 * 256;
 }
 
@@ -370,35 +540,64 @@ int moa_lens_add(int32_t *lens, int batch, int delta, void *stream)
     return cudaGetLastError() == cudaSuccess ? MOA_OK : MOA_ERR_CUDA;
 }
 
-int moa_decode_step(const float *q, float *K, float *V, const float *k_new, const float *v_new,
-                    float *out, int32_t *lens, int batch, int h_q, int h_kv, int n_max, int d_k,
-                    int d_v, float scale, void *workspace, size_t workspace_bytes, void *stream)
+// Shared body of moa_append_decode (advance == false) and moa_decode_step (advance == true).
+static int step_impl(const float *q, float *K, float *V, const float *k_new, const float *v_new,
+                     float *out, int32_t *lens_rw, const int32_t *lens, int batch, int h_q, int h_kv,
+                     int n_max, int d_k, int d_v, float scale, void *workspace, size_t workspace_bytes,
+                     void *stream, bool advance)
 {
     if (!q || !K || !V || !k_new || !v_new || !out || !lens) return MOA_ERR_INVALID;
     int rc = validate_dims(batch, h_q, h_kv, n_max, d_k, d_v);
     if (rc != MOA_OK) return rc;
     if (!isfinite(scale)) return MOA_ERR_INVALID;
-    // Dry validation of the decode arguments first, so that nothing is appended when the
-    // attention call would be rejected.
     if (!aligned(q, 4) || !aligned(K, 4) || !aligned(V, 4) || !aligned(out, 4) || !aligned(lens, 4) ||
         !aligned(k_new, 4) || !aligned(v_new, 4))
         return MOA_ERR_ALIGN;
-    const size_t need = moa_workspace_bytes(batch, h_q, h_kv, n_max, d_k, d_v);
-    StreamPlan plan = plan_stream(h_q / h_kv, d_k, d_v);
+    DeviceState *dev = nullptr;
+    rc = current_device(&dev);
+    if (rc != MOA_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const StreamPlan plan = plan_stream(h_q / h_kv, d_k, d_v);
     const bool fast_ok = plan.ok && aligned(q, 16) && aligned(K, 16) && aligned(V, 16) && aligned(out, 16);
-    if (fast_ok && g_force_path != MOA_PATH_GENERIC) {
-        if (!workspace || workspace_bytes < need) return MOA_ERR_WORKSPACE;
+    const bool stream_path = fast_ok && g_force_path != MOA_PATH_GENERIC;
+    if (g_force_path == MOA_PATH_STREAM && !fast_ok) return MOA_ERR_UNSUPPORTED;
+    if (stream_path) {          // validate the scratch before anything is written
+        if (!workspace || workspace_bytes < stream_ws_bytes(plan, stream_num_ctas(*dev))) return MOA_ERR_WORKSPACE;
         if (!aligned(workspace, 256)) return MOA_ERR_ALIGN;
     }
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // One launch: the streaming kernel appends the new rows, attends over len+1 rows and
+    // (for the step) advances the lengths when the whole grid is done.
+    if (stream_path && aligned(k_new, 16) && aligned(v_new, 16) && stream_num_ctas(*dev) <= kTicketCtas) {
+        FusedStep f;
+        f.Kw = K; f.Vw = V; f.k_new = k_new; f.v_new = v_new; f.lens_rw = advance ? lens_rw : nullptr;
+        return decode_impl(q, K, V, out, batch, h_q, h_kv, lens, 1, n_max, d_k, d_v, scale, workspace,
+                           workspace_bytes, false, st, &f);
+    }
+    // Otherwise the same thing as three launches.
     rc = moa_kv_append(K, V, k_new, v_new, lens, batch, h_kv, n_max, d_k, d_v, stream);
     if (rc != MOA_OK) return rc;
     rc = decode_impl(q, K, V, out, batch, h_q, h_kv, lens, 1, n_max, d_k, d_v, scale, workspace,
                      workspace_bytes, false, st);
-    if (rc != MOA_OK) return rc;
-    lens_add_kernel<<<(batch + 127) / 128, 128, 0, st>>>(lens, batch, 1, n_max);
+    if (rc != MOA_OK || !advance) return rc;
+    lens_add_kernel<<<(batch + 127) / 128, 128, 0, st>>>(lens_rw, batch, 1, n_max);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? MOA_OK : MOA_ERR_CUDA;
+}
+
+int moa_decode_step(const float *q, float *K, float *V, const float *k_new, const float *v_new,
+                    float *out, int32_t *lens, int batch, int h_q, int h_kv, int n_max, int d_k,
+                    int d_v, float scale, void *workspace, size_t workspace_bytes, void *stream)
+{
+    return step_impl(q, K, V, k_new, v_new, out, lens, lens, batch, h_q, h_kv, n_max, d_k, d_v, scale,
+                     workspace, workspace_bytes, stream, true);
+}
+
+int moa_append_decode(const float *q, float *K, float *V, const float *k_new, const float *v_new,
+                      float *out, const int32_t *pos, int batch, int h_q, int h_kv, int n_max, int d_k,
+                      int d_v, float scale, void *workspace, size_t workspace_bytes, void *stream)
+{
+    return step_impl(q, K, V, k_new, v_new, out, nullptr, pos, batch, h_q, h_kv, n_max, d_k, d_v, scale,
+                     workspace, workspace_bytes, stream, false);
 }
 
 int moa_decode_attn_host(const float *q, const float *K, const float *V, float *out, int batch,
@@ -506,6 +705,11 @@ int moa_set_option(int option, int value)
     if (option == MOA_OPT_FORCE_PATH) {
         if (value < 0 || value > MOA_PATH_GROUPED) return MOA_ERR_INVALID;
         g_force_path = value;
+        return MOA_OK;
+    }
+    if (option == MOA_OPT_GROUPED_HEADS) {
+        if (value != 0 && value != 16 && value != 32 && value != 64) return MOA_ERR_INVALID;
+        g_grouped_heads = value;
         return MOA_OK;
     }
     if (option == MOA_OPT_NUM_CTAS) {

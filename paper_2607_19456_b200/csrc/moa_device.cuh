@@ -52,6 +52,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
+// Non-blocking probe of a phase (try_wait may suspend the thread for a while when the phase
+// is not complete; a thread that polls several barriers in turn must not do that).
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
 // Every spin in this library is bounded: after kWaitLimit unsuccessful polls the caller
 // gives up, raises MOA_STATUS_WAIT_TIMEOUT and leaves without touching the data.
 constexpr uint32_t kWaitLimit = 1u << 22;
@@ -105,7 +120,22 @@ struct DecodeArgs {
     int n_max;                // row capacity = stride between heads
     int d_k, d_v;
     float qscale;             // scale * log2(e): scores live in the log2 domain
+    // ---- fused step (all null/zero for a plain decode) ----
+    float *Kw, *Vw;           // writable K / V when the new row is appended by the decode kernel
+    const float *k_new;       // [batch, stored kv heads, d_k] row appended at index seq_lens[b]
+    const float *v_new;       // [batch, stored kv heads, d_v]
+    int32_t *lens_rw;         // lengths advanced by one when the whole grid is done, or nullptr
+    unsigned *tickets;        // completion counters (kTicketStride words, all zero between
+                              // launches), or nullptr: partials are merged by a second kernel
 };
+
+// Completion counters of one launch: word c counts the CTAs that have delivered their
+// partial for the split unit whose first segment lies in CTA c; the last word counts CTAs
+// that have finished altogether.  Whoever brings a counter to its final value resets it.
+constexpr int kTicketCtas = 1024;
+constexpr int kTicketStride = kTicketCtas + 1;
+constexpr int kTicketSlots = 32;
+__device__ unsigned g_tickets[kTicketSlots * kTicketStride];
 
 // Length of sequence b as the kernels see it; 0 for an out-of-range length (the item is
 // then skipped by construction: it owns no row blocks).
@@ -146,11 +176,53 @@ __device__ __forceinline__ long long total_blocks(const DecodeArgs &a, int lane)
     return tot;
 }
 
-// Position a cursor on the unit containing block j (0 <= j < total).  Warp-uniform.
+// Largest batch whose per-item block prefix is kept in shared memory by the streaming
+// kernel (larger batches scan the lengths in global memory instead).
+constexpr int kPrefixBatch = 1024;
+
+// Fill pref[0..batch] with the exclusive prefix sum of blocks_of(len_b) (per kv head).
+// Called by one full warp; the caller synchronises the block afterwards.
 template <int R>
-__device__ __forceinline__ Cursor cursor_at(const DecodeArgs &a, long long j)
+__device__ __forceinline__ void build_block_prefix(const DecodeArgs &a, int *pref, int lane)
+{
+    int run = 0;
+    for (int base = 0; base < a.batch; base += 32) {
+        const int b = base + lane;
+        const int nb = (b < a.batch) ? blocks_of<R>(seq_len_of(a, b)) : 0;
+        int inc = nb;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, inc, off);
+            if (lane >= off) inc += t;
+        }
+        if (b < a.batch) pref[b] = run + inc - nb;
+        run += __shfl_sync(0xffffffffu, inc, 31);
+    }
+    if (lane == 0) pref[a.batch] = run;
+}
+
+// Position a cursor on the unit containing block j (0 <= j < total).  Warp-uniform.
+// `pref` is the shared-memory prefix built by build_block_prefix, or nullptr.
+template <int R>
+__device__ __forceinline__ Cursor cursor_at(const DecodeArgs &a, long long j, const int *pref = nullptr)
 {
     Cursor c;
+    if (a.seq_lens != nullptr && pref != nullptr) {
+        int lo = 0, hi = a.batch;              // find b with h_kv*pref[b] <= j < h_kv*pref[b+1]
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if ((long long)pref[mid] * a.h_kv <= j) lo = mid; else hi = mid;
+        }
+        while (lo < a.batch - 1 && pref[lo + 1] == pref[lo]) ++lo;   // skip items without blocks
+        const int ub = pref[lo + 1] - pref[lo];
+        const long long first = (long long)pref[lo] * a.h_kv;
+        c.b = lo;
+        c.ub = ub;
+        c.len = seq_len_of(a, lo);
+        c.h = ub > 0 ? (int)((j - first) / ub) : 0;
+        c.first = first + (long long)c.h * ub;
+        return c;
+    }
     if (a.seq_lens == nullptr) {
         const int ub = blocks_of<R>(a.n_max);
         const long long u = j / ub;

@@ -1,0 +1,529 @@
+// moa_grouped.cuh -- tensor-core decode kernel for large head groups (MQA / wide GQA).
+//
+// When GH = h_q/h_kv query heads share one K/V head, Steps I and III of Algorithm 1
+// (eqs. (1),(3)) are dense contractions per tile of cached rows:
+//     S^T[rows x GH] = K_tile[rows x d] * Q^T[d x GH],   O^T[d x GH] += V_tile^T[d x rows] * P^T[rows x GH]
+// and at GH >= 16 the fp32 FMA pipes, not HBM, would bound the kernel.  Here both products
+// run on the 5th-generation tensor cores (tcgen05.mma, kind::tf32, accumulators in tensor
+// memory) with a three-term error-compensated split so that the result keeps fp32 accuracy:
+//     x = hi + lo,  hi = x with the low 13 mantissa bits cleared (exactly what the tensor
+//     core keeps of an fp32 operand),  a*b ~= a_hi*b_hi + a_lo*b_hi + a_hi*b_lo.
+// The hi and lo parts of the small operand (Q, P) are stacked along N so one instruction
+// covers two terms; the lo part of the streamed operand (K, V) is produced in place in
+// the shared-memory buffer after the hi product has consumed it, so it costs no space.
+//
+// Orientation: the 128 cached rows of a tile are the M dimension, so a thread of the
+// softmax group owns one cached row and all GH heads of it.  Step II (eq. (2)) uses a
+// per-head reference m_ref instead of the exact running maximum (any reference gives the
+// same value; it only has to keep exp2 in range): m_ref is raised, and the accumulators
+// rescaled, only when a score exceeds it by more than 2^16.
+//
+// Roles (448 threads): warp 0 TMA producer, warps 1 and 2 MMA issuers (warp 1 also owns the
+// TMEM allocation), warps 4-11 softmax (warp w works on TMEM lane quarter w % 4, i.e. cached
+// rows 32*(w%4).., and on the lower (w < 8) or upper half of the heads), warps 3, 12, 13
+// turn K/V chunks into their lo parts.  Every hand-off is an mbarrier; every wait is bounded.
+#pragma once
+
+#include <cuda.h>
+
+#include "moa_device.cuh"
+#include "moa_tc.cuh"
+
+namespace moa {
+
+template <int GH_>
+struct GroupedCfg {
+    static constexpr int GH = GH_;
+    static constexpr int D = 128;
+    static constexpr int TILE = 128;               // cached rows per tile = MMA M
+    static constexpr int N1 = 2 * GH;              // hi|lo stacked operand rows
+    static constexpr int NBUF = GH == 64 ? 6 : (GH == 32 ? 10 : 12);   // 16 KB K/V chunk buffers
+    static constexpr int CHUNK = 16384;
+    static constexpr int OPCH = N1 * 128;          // bytes of one 32-wide k-chunk of the Q / P operand
+    static constexpr int THREADS = 448;            // 14 warps, see the role list above
+    static constexpr int NCONV = 3 * 32;           // converter threads (warps 3, 12, 13)
+    static constexpr int NSOFT = 256;              // softmax threads (warps 4..11)
+    static constexpr int HH = GH / 2;              // heads per softmax thread
+    static constexpr int PW = HH < 16 ? HH : 16;   // heads handled per TMEM read
+    static constexpr int PS = D + 4;               // floats per partial row: o[D], m, l, pad
+    static constexpr uint32_t OFF_Q = 0;
+    static constexpr uint32_t OFF_P = OFF_Q + 4 * OPCH;
+    static constexpr uint32_t OFF_RING = OFF_P + 4 * OPCH;
+    static constexpr uint32_t OFF_MREF = OFF_RING + NBUF * CHUNK;
+    static constexpr uint32_t OFF_ALPHA = OFF_MREF + GH * 4;
+    static constexpr uint32_t OFF_TMAX = OFF_ALPHA + GH * 4;
+    static constexpr uint32_t OFF_LRED = OFF_TMAX + GH * 4;
+    static constexpr uint32_t OFF_BAR = OFF_LRED + 4 * GH * 4;      // lred: [4 row quarters][GH]
+    static constexpr int NBAR = 4 * NBUF + 2 + 2 + 4 + 1;
+    static constexpr uint32_t OFF_TMEM = OFF_BAR + NBAR * 8;
+    static constexpr uint32_t OFF_ABORT = OFF_TMEM + 4;
+    static constexpr size_t SMEM_BYTES = OFF_ABORT + 4;
+    static_assert(GH == 16 || GH == 32 || GH == 64, "group size");
+    static_assert(OFF_RING % 1024 == 0, "swizzled tiles need 1024-byte alignment");
+};
+
+struct GroupedArgs {
+    const float *q;      // [batch, h_q, 128]
+    float *out;          // [batch, h_q, 128]
+    float *ws;           // partial slots [units][splits][GH][PS]
+    int batch, h_q, h_kv, n;
+    int h_kv_stored;     // K/V heads as stored; h_kv above counts virtual heads of GH query heads
+    int share;           // virtual heads per stored K/V head (h_kv = h_kv_stored * share)
+    int splits;          // sequence splits per unit
+    int tiles_per_split;
+    float qscale;        // scale * log2(e)
+};
+
+// Bounded mbarrier wait that also gives up when another role has already failed.
+__device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+{
+    for (uint32_t it = 0; it < kWaitLimit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 255u) == 255u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    raise_status(MOA_STATUS_WAIT_TIMEOUT);
+    return false;
+}
+
+__device__ __forceinline__ uint32_t ordered_bits(float x)      // monotone float -> uint
+{
+    const uint32_t b = __float_as_uint(x);
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float from_ordered_bits(uint32_t u)
+{
+    return __uint_as_float((u & 0x80000000u) ? (u & 0x7FFFFFFFu) : ~u);
+}
+__device__ __forceinline__ float tf32_hi(float x) { return __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
+
+__device__ __forceinline__ void named_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
+__device__ __forceinline__ bool named_or(int id, int n, bool pred)
+{
+    uint32_t r;
+    asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %3, 0;\n\tbar.red.or.pred p, %1, %2, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(r) : "r"(id), "r"(n), "r"((uint32_t)pred) : "memory");
+    return r != 0;
+}
+
+// The order in which 16 KB chunks travel through the ring, shared by producer, issuer and
+// converters: K(0), then for every tile t: K(t+1) (if any) followed by V(t).
+struct ChunkSeq {
+    int T;          // tiles of this CTA
+    int t;          // tile of the current group
+    bool is_k;      // group kind
+    int c;          // chunk inside the group, 0..3
+    int seq;        // running chunk number (ring position = seq % NBUF)
+    bool done;
+    __device__ __forceinline__ explicit ChunkSeq(int tiles) : T(tiles), t(0), is_k(true), c(0), seq(0), done(tiles <= 0) {}
+    // Skip whole groups of the other kind (used by an issuer that handles one kind only).
+    __device__ __forceinline__ void skip_to_kind(bool want_k)
+    {
+        while (!done && is_k != want_k) { next(); next(); next(); next(); }
+    }
+    __device__ __forceinline__ void next()
+    {
+        ++seq;
+        if (++c < 4) return;
+        c = 0;
+        if (is_k) {                     // after K(0) comes K(1) or V(0); after K(t+1) comes V(t)
+            if (t == 0 && T > 1 && seq == 4) { t = 1; return; }     // K(0) -> K(1)
+            is_k = false;
+            t = (t == 0) ? 0 : t - 1;
+        } else {                        // after V(t): K(t+2) if it exists, else V(t+1), else done
+            if (t + 2 < T) { is_k = true; t = t + 2; }
+            else if (t + 1 < T) { t = t + 1; }
+            else done = true;
+        }
+    }
+};
+
+template <class C>
+__global__ void __launch_bounds__(C::THREADS, 1)
+grouped_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant__ CUtensorMap tmapV,
+                      const GroupedArgs a)
+{
+    constexpr int GH = C::GH, N1 = C::N1, NBUF = C::NBUF, PS = C::PS;
+    extern __shared__ __align__(1024) unsigned char smem[];
+    float *mref = reinterpret_cast<float *>(smem + C::OFF_MREF);
+    float *alpha_s = reinterpret_cast<float *>(smem + C::OFF_ALPHA);
+    uint32_t *tmax = reinterpret_cast<uint32_t *>(smem + C::OFF_TMAX);
+    float *lred = reinterpret_cast<float *>(smem + C::OFF_LRED);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + C::OFF_BAR);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + C::OFF_TMEM);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + C::OFF_ABORT);
+
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t sQ = sbase + C::OFF_Q, sP = sbase + C::OFF_P, sRing = sbase + C::OFF_RING;
+    auto bar_full = [&](int b) { return smem_u32(&bars[b]); };
+    auto bar_hi = [&](int b) { return smem_u32(&bars[NBUF + b]); };
+    auto bar_lo = [&](int b) { return smem_u32(&bars[2 * NBUF + b]); };
+    auto bar_empty = [&](int b) { return smem_u32(&bars[3 * NBUF + b]); };
+    auto bar_sfull = [&](int s) { return smem_u32(&bars[4 * NBUF + s]); };
+    auto bar_sfree = [&](int s) { return smem_u32(&bars[4 * NBUF + 2 + s]); };
+    auto bar_pfull = [&](int c) { return smem_u32(&bars[4 * NBUF + 4 + c]); };
+    const uint32_t bar_pvdone = smem_u32(&bars[4 * NBUF + 8]);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    // CTA order: the virtual heads that share one stored K/V head are neighbours, so they run
+    // at the same time and the second reader of a chunk finds it in L2.
+    const int sub = blockIdx.x % a.share;
+    const int split = (blockIdx.x / a.share) % a.splits;
+    const int sunit = blockIdx.x / (a.share * a.splits);          // stored (batch, kv head)
+    const int b = sunit / a.h_kv_stored, h = (sunit % a.h_kv_stored) * a.share + sub;   // virtual head
+    const int unit = sunit;                                         // tensor-map coordinate
+    const int tiles_total = (a.n + C::TILE - 1) / C::TILE;
+    const int tile0 = split * a.tiles_per_split;
+    int T = tiles_total - tile0;
+    if (T > a.tiles_per_split) T = a.tiles_per_split;
+    if (T <= 0) return;                            // an empty split (uniform for the CTA)
+
+    // ---- set-up --------------------------------------------------------------------------
+    if (tid == 0) {
+        for (int i = 0; i < NBUF; ++i) {
+            mbar_init(bar_full(i), 1); mbar_init(bar_hi(i), 1);
+            mbar_init(bar_lo(i), C::NCONV / 32); mbar_init(bar_empty(i), 1);
+        }
+        for (int i = 0; i < 2; ++i) { mbar_init(bar_sfull(i), 1); mbar_init(bar_sfree(i), 8); }
+        for (int i = 0; i < 4; ++i) mbar_init(bar_pfull(i), 2);
+        mbar_init(bar_pvdone, 1);
+        mbar_fence_init();
+        *abort_flag = 0;
+        tc::prefetch_tmap(&tmapK);
+        tc::prefetch_tmap(&tmapV);
+    }
+    if (warp == 1) tc::tmem_alloc(smem_u32(tmem_slot), 512);
+    // Q operand: rows 0..GH-1 hold hi(q*qscale), rows GH..2GH-1 the lo parts; K-major, 4
+    // chunks of 32 features, 128-byte swizzle.
+    {
+        const float *qb = a.q + ((size_t)b * a.h_q + (size_t)h * GH) * 128;
+        for (int i = tid; i < GH * 128; i += C::THREADS) {
+            const int g = i >> 7, k = i & 127;
+            const float x = qb[i] * a.qscale;
+            const float hi = tf32_hi(x);
+            const uint32_t chunk = (uint32_t)(k >> 5) * C::OPCH, col = (uint32_t)(k & 31) * 4;
+            *reinterpret_cast<float *>(smem + C::OFF_Q + chunk + tc::swz128(g, col)) = hi;
+            *reinterpret_cast<float *>(smem + C::OFF_Q + chunk + tc::swz128(GH + g, col)) = x - hi;
+        }
+        if (tid < GH) mref[tid] = -INFINITY;
+    }
+    tc::fence_async_smem();
+    tc::fence_before_sync();
+    __syncthreads();
+    tc::fence_after_sync();
+    const uint32_t tmem = *tmem_slot;
+    auto tS_of = [tmem](int sb) -> uint32_t { return tmem + (uint32_t)(sb & 1) * 128u; };   // two score buffers
+    const uint32_t tO = tmem + 256u;           // per-tile weighted sum [hi | lo] written by the tensor core
+    const uint32_t tOm = tmem + 384u;          // fp32 master copy of the weighted sum, GH columns
+    const int row_base = tile0 * C::TILE;
+
+    if (warp == 0) {
+        // ================= TMA producer =================
+        if (lane == 0) {
+            for (ChunkSeq s(T); !s.done; s.next()) {
+                const int buf = s.seq % NBUF, use = s.seq / NBUF;
+                if (use > 0 && !wait_or_abort(bar_empty(buf), (uint32_t)(use - 1) & 1u, abort_flag)) break;
+                const uint32_t dst = sRing + (uint32_t)buf * C::CHUNK;
+                mbar_expect_tx(bar_full(buf), C::CHUNK);
+                const int row = row_base + s.t * C::TILE;
+                if (s.is_k) {
+                    tc::tma_load_3d(dst, &tmapK, 32 * s.c, row, unit, bar_full(buf));
+                } else {
+                    for (int dg = 0; dg < 4; ++dg)
+                        tc::tma_load_3d(dst + dg * 4096, &tmapV, 32 * dg, row + 32 * s.c, unit, bar_full(buf));
+                }
+            }
+        }
+    } else if (warp == 1 || warp == 2) {
+        // ================= MMA issuers =================
+        // Two single-thread issuers feed the tensor core: warp 1 the score products (K chunks,
+        // accumulators S), warp 2 the weighted-sum products (V chunks, accumulator O).  Each
+        // keeps two cursors over its chunks: `hi` (next chunk whose raw data is multiplied) and
+        // `lo` (next chunk whose in-place lo part is multiplied) and issues whichever is
+        // ready, so a chunk waiting for its converters never holds up the ones behind it.
+        // A lone thread retires an instruction every few cycles, so the issue path is kept to
+        // a handful of instructions per MMA (descriptor words are advanced, not rebuilt).
+        if (lane == 0) {
+            const bool kind_k = (warp == 1);
+            const uint32_t idesc_hi = kind_k ? tc::idesc_tf32(128, N1, false, false) : tc::idesc_tf32(128, N1, true, false);
+            const uint32_t idesc_lo = kind_k ? tc::idesc_tf32(128, GH, false, false) : tc::idesc_tf32(128, GH, true, false);
+            // descriptor words: [addr>>4 | lbo>>4 << 16] and [sbo>>4 | version << 14 | layout << 29]
+            const uint32_t a_hiword = kind_k ? (64u | (1u << 14) | (2u << 29)) : (32u | (1u << 14) | (1u << 29));
+            const uint32_t a_base = (sRing >> 4) | (kind_k ? (1u << 16) : (256u << 16));
+            const uint32_t a_step = kind_k ? 2u : 64u;                 // 32 B / 1024 B per k-step
+            const uint32_t b_hiword = 64u | (1u << 14) | (2u << 29);
+            const uint32_t b_base = ((kind_k ? sQ : sP) >> 4) | (1u << 16);
+            // Issue order inside a group of four chunks is fixed (hi0 hi1 hi2 lo0 hi3 lo1 lo2 lo3):
+            // the hi*lo and lo*hi terms share accumulator columns and the tensor core's
+            // accumulation is not associative, so a timing-dependent order would make the
+            // result differ from run to run.  The two-chunk lag gives the converters time.
+            // In the chunk sequence the K groups sit at group indices 0,1,3,5,... and the V
+            // groups at 2,4,...,2T-2,2T-1; a group's first chunk is number 4*index.
+            auto spin = [&](uint32_t bar, uint32_t parity) -> bool {      // bounded, non-suspending
+                for (uint32_t it = 0; it < kWaitLimit; ++it) {
+                    if (mbar_test_wait(bar, parity)) return true;
+                    if ((it & 255u) == 255u && *abort_flag) return false;
+                }
+                *abort_flag = 1;
+                raise_status(MOA_STATUS_WAIT_TIMEOUT);
+                return false;
+            };
+            bool ok = true;
+            for (int t = 0; ok && t < T; ++t) {
+                const int gi = kind_k ? (t == 0 ? 0 : 2 * t - 1) : (t < T - 1 ? 2 * t + 2 : 2 * T - 1);
+                const int seq0 = 4 * gi;
+                const uint32_t d_hi = kind_k ? tS_of(t) : tO;
+                if (kind_k && t >= 2) ok = spin(bar_sfree(t & 1), (uint32_t)(t / 2 - 1) & 1u);
+                if (!kind_k) {
+                    // chunk 0 overwrites the whole per-tile accumulator, which every softmax
+                    // warp reads while folding the previous tile: wait for all of them
+                    for (int w = 0; ok && w < 4; ++w) ok = spin(bar_pfull(w), (uint32_t)t & 1u);
+                }
+#pragma unroll
+                for (int step = 0; step < 8; ++step) {
+                    // steps: H0 H1 H2 L0 H3 L1 L2 L3
+                    const bool is_hi = (step < 3) || (step == 4);
+                    const int c = is_hi ? (step < 3 ? step : 3) : (step == 3 ? 0 : step - 4);
+                    const int seq = seq0 + c;
+                    const int buf = seq % NBUF;
+                    const uint32_t ph = (uint32_t)(seq / NBUF) & 1u;
+                    if (!ok) break;
+                    ok = spin(is_hi ? bar_full(buf) : bar_lo(buf), ph);
+                    if (!ok) break;
+                    tc::fence_after_sync();
+                    const uint32_t a_lo = a_base + (uint32_t)buf * (C::CHUNK >> 4);
+                    const uint32_t b_lo = b_base + (uint32_t)c * (C::OPCH >> 4);
+                    if (is_hi) {
+                        // the first product of a tile overwrites its accumulator (the weighted
+                        // sum is folded into an fp32 master copy by the softmax group every tile)
+                        tc::mma_tf32_ss(d_hi, tc::pack64(a_lo, a_hiword), tc::pack64(b_lo, b_hiword), idesc_hi, (uint32_t)c);
+#pragma unroll
+                        for (uint32_t ks = 1; ks < 4; ++ks)
+                            tc::mma_tf32_ss(d_hi, tc::pack64(a_lo + ks * a_step, a_hiword),
+                                            tc::pack64(b_lo + ks * 2u, b_hiword), idesc_hi, 1u);
+                        tc::mma_commit(bar_hi(buf));
+                    } else {
+#pragma unroll
+                        for (uint32_t ks = 0; ks < 4; ++ks)
+                            tc::mma_tf32_ss(d_hi + GH, tc::pack64(a_lo + ks * a_step, a_hiword),
+                                            tc::pack64(b_lo + ks * 2u, b_hiword), idesc_lo, 1u);
+                        tc::mma_commit(bar_empty(buf));
+                        if (c == 3) tc::mma_commit(kind_k ? bar_sfull(t & 1) : bar_pvdone);
+                    }
+                }
+            }
+        }
+    } else if (warp >= 4 && warp < 12) {
+        // ================= softmax group: thread = (cached row, half of the heads) =================
+        constexpr int HH = C::HH, PW = C::PW, NP = HH / PW, NS = C::NSOFT;
+        const int q4 = warp & 3;                     // TMEM lane quarter = rows 32*q4 .. 32*q4+31 of the tile
+        const int h0 = (warp < 8) ? 0 : HH;          // first head of this thread
+        const int st = tid - 128;                    // 0..255 inside the group
+        const int row_in_tile = q4 * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)(q4 * 32) << 16;
+        float lsum[HH], p[HH];
+#pragma unroll
+        for (int g = 0; g < HH; ++g) lsum[g] = 0.f;
+        unsigned char *pch = smem + C::OFF_P + (uint32_t)q4 * C::OPCH;     // this row quarter's P chunk
+        bool ok = true;
+        for (int t = 0; ok && t < T; ++t) {
+            const int sb = t & 1;
+            ok = wait_or_abort(bar_sfull(sb), (uint32_t)(t >> 1) & 1u, abort_flag);
+            if (named_or(1, NS, !ok)) { ok = false; break; }     // leave together or not at all
+            tc::fence_after_sync();
+            const bool valid = (row_base + t * C::TILE + row_in_tile) < a.n;
+            // scores of this row against the current references; probabilities are formed at
+            // once (they are only wrong if the reference has to be raised, which is rare)
+            float vmax = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < NP; ++j) {
+                uint32_t hi[PW], lo[PW];
+                tc::tmem_ld_piece<PW>(tS_of(sb) + lane_addr + h0 + PW * j, hi);
+                tc::tmem_ld_piece<PW>(tS_of(sb) + lane_addr + GH + h0 + PW * j, lo);
+                tc::tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < PW; ++i) {
+                    const float x = (__uint_as_float(hi[i]) + __uint_as_float(lo[i])) - mref[h0 + PW * j + i];
+                    vmax = fmaxf(vmax, x);
+                    p[PW * j + i] = valid ? fast_exp2(x) : 0.f;
+                }
+            }
+            const bool raise = named_or(1, NS, valid && (vmax > 16.0f));
+            if (raise) {
+                // ---- exact per-head maximum of this tile
+                if (st < GH) tmax[st] = 0u;
+                named_sync(1, NS);
+#pragma unroll
+                for (int j = 0; j < NP; ++j) {
+                    uint32_t hi[PW], lo[PW];
+                    tc::tmem_ld_piece<PW>(tS_of(sb) + lane_addr + h0 + PW * j, hi);
+                    tc::tmem_ld_piece<PW>(tS_of(sb) + lane_addr + GH + h0 + PW * j, lo);
+                    tc::tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < PW; ++i) {
+                        const float sv = valid ? (__uint_as_float(hi[i]) + __uint_as_float(lo[i])) : -INFINITY;
+                        const uint32_t m = __reduce_max_sync(0xffffffffu, ordered_bits(sv));
+                        if (lane == 0) atomicMax(&tmax[h0 + PW * j + i], m);
+                    }
+                }
+                named_sync(1, NS);
+                if (st < GH) {
+                    const float old = mref[st];
+                    const float nw = fmaxf(old, from_ordered_bits(tmax[st]));
+                    alpha_s[st] = exp2_diff(old, nw);
+                    mref[st] = nw;
+                }
+                named_sync(1, NS);
+#pragma unroll
+                for (int j = 0; j < NP; ++j) {        // probabilities again, against the new references
+                    uint32_t hi[PW], lo[PW];
+                    tc::tmem_ld_piece<PW>(tS_of(sb) + lane_addr + h0 + PW * j, hi);
+                    tc::tmem_ld_piece<PW>(tS_of(sb) + lane_addr + GH + h0 + PW * j, lo);
+                    tc::tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < PW; ++i) {
+                        const float x = (__uint_as_float(hi[i]) + __uint_as_float(lo[i])) - mref[h0 + PW * j + i];
+                        p[PW * j + i] = valid ? fast_exp2(x) : 0.f;
+                    }
+                }
+#pragma unroll
+                for (int g = 0; g < HH; ++g) lsum[g] *= alpha_s[h0 + g];
+            }
+            // the score buffer is free again
+            tc::fence_before_sync();
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive(bar_sfree(sb));
+#pragma unroll
+            for (int g = 0; g < HH; ++g) lsum[g] += p[g];
+            // The previous tile's weighted sum is complete: fold it into the fp32 master copy
+            // (the tensor core accumulates with truncation, so its chains are kept one tile
+            // long), which also frees the P buffers and the per-tile accumulator.
+            if (t > 0) {
+                ok = wait_or_abort(bar_pvdone, (uint32_t)(t - 1) & 1u, abort_flag);
+                if (named_or(1, NS, !ok)) { ok = false; break; }
+                tc::fence_after_sync();
+#pragma unroll
+                for (int j = 0; j < NP; ++j) {
+                    uint32_t hi[PW], lo[PW], ms[PW];
+                    tc::tmem_ld_piece<PW>(tO + lane_addr + h0 + PW * j, hi);
+                    tc::tmem_ld_piece<PW>(tO + lane_addr + GH + h0 + PW * j, lo);
+                    if (t > 1) tc::tmem_ld_piece<PW>(tOm + lane_addr + h0 + PW * j, ms);
+                    tc::tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < PW; ++i) {
+                        float add = __uint_as_float(hi[i]) + __uint_as_float(lo[i]);
+                        if (t > 1) add += __uint_as_float(ms[i]);
+                        if (raise) add *= alpha_s[h0 + PW * j + i];
+                        ms[i] = __float_as_uint(add);
+                    }
+                    tc::tmem_st_piece<PW>(tOm + lane_addr + h0 + PW * j, ms);
+                }
+                tc::tmem_st_wait();
+            }
+            // probabilities, split into hi|lo, as the K-major B operand of this row quarter
+#pragma unroll
+            for (int g = 0; g < HH; ++g) {
+                const float ph = tf32_hi(p[g]);
+                *reinterpret_cast<float *>(pch + tc::swz128(h0 + g, lane * 4)) = ph;
+                *reinterpret_cast<float *>(pch + tc::swz128(GH + h0 + g, lane * 4)) = p[g] - ph;
+            }
+            tc::fence_before_sync();
+            tc::fence_async_smem();
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive(bar_pfull(q4));
+        }
+        // ---- epilogue: this split's partial (m_ref, l, o) per head
+        if (ok) {                            // (ok is uniform across the group here)
+            ok = wait_or_abort(bar_pvdone, (uint32_t)(T - 1) & 1u, abort_flag);
+            if (named_or(1, NS, !ok)) ok = false;
+        }
+        if (ok) {
+            tc::fence_after_sync();
+#pragma unroll
+            for (int g = 0; g < HH; ++g) {
+                float v = lsum[g];
+#pragma unroll
+                for (int off = 16; off >= 1; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+                if (lane == 0) lred[q4 * GH + h0 + g] = v;
+            }
+            named_sync(1, NS);
+            float *slot = a.ws + ((((size_t)b * a.h_kv + h) * a.splits + split) * GH) * PS;
+            const int d = row_in_tile;               // TMEM lane of O^T = output feature
+#pragma unroll
+            for (int j = 0; j < NP; ++j) {
+                uint32_t hi[PW], lo[PW], ms[PW];
+                tc::tmem_ld_piece<PW>(tO + lane_addr + h0 + PW * j, hi);
+                tc::tmem_ld_piece<PW>(tO + lane_addr + GH + h0 + PW * j, lo);
+                if (T > 1) tc::tmem_ld_piece<PW>(tOm + lane_addr + h0 + PW * j, ms);
+                tc::tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < PW; ++i) {
+                    float add = __uint_as_float(hi[i]) + __uint_as_float(lo[i]);
+                    if (T > 1) add += __uint_as_float(ms[i]);
+                    slot[(size_t)(h0 + PW * j + i) * PS + d] = add;
+                }
+            }
+            if (st < GH) {
+                slot[(size_t)st * PS + 128] = mref[st];
+                slot[(size_t)st * PS + 129] = (lred[st] + lred[GH + st]) + (lred[2 * GH + st] + lred[3 * GH + st]);
+            }
+        }
+    } else {
+        // ================= converters: chunk -> its lo part, in place =================
+        const int ct = (warp == 3 ? 0 : warp - 11) * 32 + lane;            // 0..95
+        bool ok = true;
+        for (ChunkSeq s(T); ok && !s.done; s.next()) {
+            const int buf = s.seq % NBUF, use = s.seq / NBUF;
+            ok = wait_or_abort(bar_full(buf), (uint32_t)use & 1u, abort_flag) &&
+                 wait_or_abort(bar_hi(buf), (uint32_t)use & 1u, abort_flag);
+            if (!ok) break;
+            float4 *p = reinterpret_cast<float4 *>(smem + C::OFF_RING + (uint32_t)buf * C::CHUNK);
+            for (int i = ct; i < C::CHUNK / 16; i += C::NCONV) {
+                float4 v = p[i];
+                v.x -= tf32_hi(v.x); v.y -= tf32_hi(v.y); v.z -= tf32_hi(v.z); v.w -= tf32_hi(v.w);
+                p[i] = v;
+            }
+            tc::fence_async_smem();
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive(bar_lo(buf));
+        }
+    }
+
+    tc::fence_before_sync();
+    __syncthreads();
+    if (warp == 1) tc::tmem_dealloc(tmem, 512);
+}
+
+// Merge the per-split partials of the grouped kernel.  One warp per (batch, query head).
+template <int GH>
+__global__ void __launch_bounds__(128) grouped_combine_kernel(const GroupedArgs a)
+{
+    constexpr int PS = 132;
+    const int lane = threadIdx.x & 31;
+    const long long wid = (long long)blockIdx.x * 4 + (threadIdx.x >> 5);
+    if (wid >= (long long)a.batch * a.h_q) return;
+    const int b = (int)(wid / a.h_q), gq = (int)(wid % a.h_q);
+    const int h = gq / GH, g = gq % GH;
+    const int unit = b * a.h_kv + h;
+    const int tiles_total = (a.n + 127) / 128;
+    const int used = (tiles_total + a.tiles_per_split - 1) / a.tiles_per_split;   // non-empty splits
+    const float *base = a.ws + ((size_t)unit * a.splits * GH + g) * PS;
+    const size_t stride = (size_t)GH * PS;
+    float M = -INFINITY;
+    for (int s = 0; s < used; ++s) M = fmaxf(M, base[s * stride + 128]);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float L = 0.f;
+    for (int s = 0; s < used; ++s) {
+        const float *p = base + s * stride;
+        const float f = exp2_diff(p[128], M);
+        L = fmaf(p[129], f, L);
+        const float4 t = *reinterpret_cast<const float4 *>(p + lane * 4);
+        acc.x = fmaf(t.x, f, acc.x); acc.y = fmaf(t.y, f, acc.y);
+        acc.z = fmaf(t.z, f, acc.z); acc.w = fmaf(t.w, f, acc.w);
+    }
+    const float inv = 1.0f / L;
+    *reinterpret_cast<float4 *>(a.out + ((size_t)b * a.h_q + gq) * 128 + lane * 4) =
+        make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+}
+
+}  // namespace moa

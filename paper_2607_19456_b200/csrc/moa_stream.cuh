@@ -15,8 +15,11 @@
 // streaming loop.  A warp keeps its own running (max, sum, weighted-V) state; when the
 // CTA's range crosses a unit boundary the warps' states are merged through shared
 // memory and written either as the final output (the CTA saw the whole unit) or as a
-// partial (m, l, o) triple into the CTA's slot of the workspace.  A second tiny kernel
-// merges the partial triples of units that were split across CTAs, in a fixed order.
+// partial (m, l, o) triple into the CTA's slot of the workspace.  The CTA that delivers the
+// last partial of a split unit (found with a completion counter) merges that unit's
+// partials in CTA order, so the result does not depend on which CTA does it; with more than
+// kTicketCtas CTAs a second tiny kernel does the merging instead.  The same launch can
+// also perform the cache append of the step's new (k, v) row and advance the lengths.
 #pragma once
 
 #include "moa_device.cuh"
@@ -93,6 +96,8 @@ __global__ void __launch_bounds__(C::THREADS, 1) stream_decode_kernel(const Deco
     float *pbuf = reinterpret_cast<float *>(smem + C::OFF_P);
     float *abuf = reinterpret_cast<float *>(smem + C::OFF_A);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + C::OFF_BAR);
+    __shared__ int s_last;                    // "this CTA completed a counter" broadcast
+    __shared__ int s_pref[kPrefixBatch + 1];  // per-item block prefix for ragged batches
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int sub = lane / LPR;               // which of the RPI rows of a 512-byte read
@@ -101,37 +106,62 @@ __global__ void __launch_bounds__(C::THREADS, 1) stream_decode_kernel(const Deco
     const int my_g = vi / RV, my_r = vi % RV;
     const int my_row = my_r * RPI + sub;      // its row inside the block
     const bool owner = (lane % LPR) < NV;     // first copy of the value inside the row group
+    const int h_stored = a.h_kv / a.kv_share; // K/V heads as stored
 
     if (tid < W * S) mbar_init(smem_u32(&bars[tid]), 1);
     mbar_fence_init();
     __syncthreads();
 
-    const long long total = total_blocks<R>(a, lane);
+    const int *pref = nullptr;
+    if (a.seq_lens != nullptr && a.batch <= kPrefixBatch) {
+        if (warp == 0) build_block_prefix<R>(a, s_pref, lane);
+        __syncthreads();
+        pref = s_pref;
+    }
+    const long long total = pref ? (long long)pref[a.batch] * a.h_kv : total_blocks<R>(a, lane);
     const long long bpc = (total + gridDim.x - 1) / gridDim.x;
     const long long c0 = (long long)blockIdx.x * bpc;
     const long long c1 = (c0 + bpc < total) ? c0 + bpc : total;
-    if (c0 >= c1) return;                     // uniform for the whole CTA
 
+    if (c0 < c1) {                            // uniform for the whole CTA
     float *my_ring = ring + (size_t)warp * S * C::STAGE_FLOATS;
     const uint32_t my_bar0 = smem_u32(&bars[warp * S]);
 
     // ---- load side: this warp's blocks are c0+warp, c0+warp+W, ... ---------------------
     long long jl = c0 + warp;
     int kl = 0;
-    Cursor lc = cursor_at<R>(a, (jl < c1) ? jl : c0);
+    Cursor lc = cursor_at<R>(a, (jl < c1) ? jl : c0, pref);
     auto issue_next_load = [&]() {
         while (jl >= lc.first + lc.ub) cursor_next_unit<R>(a, lc);
         const int row0 = (int)(jl - lc.first) * R;
         const int nr = (lc.len - row0 < R) ? lc.len - row0 : R;
+        // Fused append: the unit's last row is the token being appended.  It is fetched from
+        // k_new / v_new (never from the cache), and this warp also stores it into the cache.
+        const bool has_new = (a.k_new != nullptr) && (row0 + nr == lc.len);
+        const int nr_cache = has_new ? nr - 1 : nr;
+        const size_t slab = (size_t)lc.b * h_stored + lc.h / a.kv_share;
+        const size_t row = slab * (size_t)a.n_max + row0;
         if (lane == 0) {
             const int stage = kl % S;
             const uint32_t bar = my_bar0 + 8u * stage;
             const uint32_t dst = smem_u32(my_ring + (size_t)stage * C::STAGE_FLOATS);
-            const uint32_t bytes = (uint32_t)nr * D * 4u;
-            const size_t row = ((size_t)lc.b * (a.h_kv / a.kv_share) + lc.h / a.kv_share) * (size_t)a.n_max + row0;
-            mbar_expect_tx(bar, 2u * bytes);
-            bulk_g2s(dst, a.K + row * D, bytes, bar);
-            bulk_g2s(dst + R * D * 4u, a.V + row * D, bytes, bar);
+            const uint32_t bytes = (uint32_t)nr_cache * D * 4u;
+            mbar_expect_tx(bar, 2u * (uint32_t)nr * D * 4u);
+            if (nr_cache > 0) {
+                bulk_g2s(dst, a.K + row * D, bytes, bar);
+                bulk_g2s(dst + R * D * 4u, a.V + row * D, bytes, bar);
+            }
+            if (has_new) {
+                bulk_g2s(dst + bytes, a.k_new + slab * D, D * 4u, bar);
+                bulk_g2s(dst + R * D * 4u + bytes, a.v_new + slab * D, D * 4u, bar);
+            }
+        }
+        if (has_new && (lc.h % a.kv_share) == 0 && lane < LPR) {
+            const size_t dst_row = (row + nr_cache) * D + lane * 4;
+            *reinterpret_cast<float4 *>(a.Kw + dst_row) =
+                *reinterpret_cast<const float4 *>(a.k_new + slab * D + lane * 4);
+            *reinterpret_cast<float4 *>(a.Vw + dst_row) =
+                *reinterpret_cast<const float4 *>(a.v_new + slab * D + lane * 4);
         }
         jl += W;
         ++kl;
@@ -140,7 +170,7 @@ __global__ void __launch_bounds__(C::THREADS, 1) stream_decode_kernel(const Deco
     for (int i = 0; i < S && jl < c1; ++i) issue_next_load();
 
     // ---- compute side ------------------------------------------------------------------
-    Cursor cc = cursor_at<R>(a, c0);
+    Cursor cc = cursor_at<R>(a, c0, pref);
     float4 qreg[G];
     float4 o[G];
     float m_run, l_run;
@@ -159,7 +189,8 @@ __global__ void __launch_bounds__(C::THREADS, 1) stream_decode_kernel(const Deco
 
     // Merge the VW running states of this CTA for the unit under `cc` and emit either the
     // final output rows or this CTA's partial triple.  Called by every warp, in the same
-    // order, once per unit the CTA touches.
+    // order, once per unit the CTA touches.  When completion counters are in use, the CTA
+    // that delivers the last partial of a split unit also merges that unit's partials.
     auto finish_unit = [&]() {
         float l_tot = l_run;                   // sum over the RV lanes holding one head
 #pragma unroll
@@ -172,6 +203,10 @@ __global__ void __launch_bounds__(C::THREADS, 1) stream_decode_kernel(const Deco
         for (int g = 0; g < G; ++g)
             *reinterpret_cast<float4 *>(merge_o + ((size_t)(vw * G + g)) * D + (lane % LPR) * 4) = o[g];
         __syncthreads();
+        const long long seg_begin = (c0 > cc.first) ? c0 : cc.first;
+        const long long unit_end = cc.first + cc.ub;
+        const long long seg_end = (c1 < unit_end) ? c1 : unit_end;
+        const bool complete = (seg_begin == cc.first) && (seg_end == unit_end);
         if (tid < G * LPR) {
             const int g = tid / LPR, d4 = tid % LPR;
             float M = -INFINITY;
@@ -187,10 +222,6 @@ __global__ void __launch_bounds__(C::THREADS, 1) stream_decode_kernel(const Deco
                 acc.z = fmaf(t.z, f, acc.z); acc.w = fmaf(t.w, f, acc.w);
                 L = fmaf(merge_ml[(v * G + g) * 2 + 1], f, L);
             }
-            const long long seg_begin = (c0 > cc.first) ? c0 : cc.first;
-            const long long unit_end = cc.first + cc.ub;
-            const long long seg_end = (c1 < unit_end) ? c1 : unit_end;
-            const bool complete = (seg_begin == cc.first) && (seg_end == unit_end);
             if (complete) {
                 if (g < a.g_s) {
                     const float inv = 1.0f / L;
@@ -205,6 +236,42 @@ __global__ void __launch_bounds__(C::THREADS, 1) stream_decode_kernel(const Deco
             }
         }
         __syncthreads();
+        if (!complete && a.tickets != nullptr) {
+            const long long c_first = cc.first / bpc, c_last = (unit_end - 1) / bpc;
+            if (tid == 0) {
+                __threadfence();               // this CTA's partial is visible before it is counted
+                const unsigned arrived = atomicAdd(&a.tickets[c_first], 1u);
+                const int last = (arrived == (unsigned)(c_last - c_first));
+                if (last) a.tickets[c_first] = 0u;
+                s_last = last;
+            }
+            __syncthreads();
+            if (s_last && tid < G * LPR) {
+                __threadfence();
+                const int g = tid / LPR, d4 = tid % LPR;
+                float M = -INFINITY;
+                for (long long c = c_first; c <= c_last; ++c) {
+                    const int slot = (cc.first <= c * bpc) ? 0 : 1;
+                    M = fmaxf(M, __ldcg(a.ws + (((size_t)c * 2 + slot) * G + g) * PS + D));
+                }
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                float L = 0.f;
+                for (long long c = c_first; c <= c_last; ++c) {
+                    const int slot = (cc.first <= c * bpc) ? 0 : 1;
+                    const float *p = a.ws + (((size_t)c * 2 + slot) * G + g) * PS;
+                    const float f = exp2_diff(__ldcg(p + D), M);
+                    L = fmaf(__ldcg(p + D + 1), f, L);
+                    const float4 t = __ldcg(reinterpret_cast<const float4 *>(p + d4 * 4));
+                    acc.x = fmaf(t.x, f, acc.x); acc.y = fmaf(t.y, f, acc.y);
+                    acc.z = fmaf(t.z, f, acc.z); acc.w = fmaf(t.w, f, acc.w);
+                }
+                if (g < a.g_s) {
+                    const float inv = 1.0f / L;
+                    float *dst = a.out + ((size_t)cc.b * a.h_q + (size_t)cc.h * a.g_s + g) * D + d4 * 4;
+                    *reinterpret_cast<float4 *>(dst) = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+                }
+            }
+        }
     };
 
     auto process_block = [&](const float *stage_base, int nr, auto full_tag) {
@@ -291,6 +358,31 @@ __global__ void __launch_bounds__(C::THREADS, 1) stream_decode_kernel(const Deco
         begin_unit();
     }
     finish_unit();
+    }  // c0 < c1
+
+    // ---- whole-grid completion: range report and length advance by the last CTA ---------
+    if (a.tickets != nullptr) {
+        __syncthreads();
+        if (tid == 0) {
+            __threadfence();
+            const unsigned done = atomicAdd(&a.tickets[kTicketCtas], 1u);
+            const int last = (done == gridDim.x - 1);
+            if (last) a.tickets[kTicketCtas] = 0u;
+            s_last = last;
+        }
+        __syncthreads();
+        if (s_last && a.seq_lens != nullptr) {   // every CTA has finished reading the lengths
+            for (int b = tid; b < a.batch; b += blockDim.x) {
+                const int raw = a.seq_lens[b];
+                const int len = raw + a.len_bias;
+                if (len < 1 || len > a.n_max) {
+                    raise_status(MOA_STATUS_SEQLEN_RANGE | (a.k_new != nullptr ? MOA_STATUS_APPEND_RANGE : 0));
+                } else if (a.lens_rw != nullptr) {
+                    a.lens_rw[b] = raw + 1;
+                }
+            }
+        }
+    }
 }
 
 // Merge the partial triples of every unit that was split across CTAs.  One warp per

@@ -21,7 +21,7 @@ def run_dense_on_gpu(w):
     out = torch.full((w.batch, w.h_q, w.d_v), float("nan"), device="cuda")
     moa.moa_decode_attn(dq, dK, dV, out, w.batch, w.h_q, w.h_kv, w.n, w.d_k, w.d_v, w.scale)
     torch.cuda.synchronize()
-    assert moa.moa_last_path() == moa.PATH_STREAM
+    assert moa.moa_last_path() == (moa.PATH_GROUPED if w.group >= 16 and w.d_k == 128 else moa.PATH_STREAM)
     assert moa.moa_device_status() == 0
     res = out.cpu().numpy()
     del dq, dK, dV, out

@@ -54,8 +54,12 @@ def test_stream_kernel_group_sizes(D, gs):
     hkv = 2
     for n in (1, 7, 130, 1037):
         q, K, V, s = make(1000 * D + 10 * gs + n, 2, gs * hkv, hkv, n, D, D)
-        out = gpu_decode(q, K, V, s, expect_path=moa.PATH_STREAM)
-        assert max_err(out, oracle.decode(q, K, V, s)) <= TOL, (D, gs, n)
+        want = moa.PATH_GROUPED if (D == 128 and gs in (16, 32, 64)) else moa.PATH_STREAM
+        out = gpu_decode(q, K, V, s, expect_path=want)
+        ref = oracle.decode(q, K, V, s)
+        assert max_err(out, ref) <= TOL, (D, gs, n)
+        if want == moa.PATH_GROUPED:         # the same shape through the FFMA kernel
+            assert max_err(gpu_decode(q, K, V, s, path=moa.PATH_STREAM), ref) <= TOL, (D, gs, n)
 
 
 @pytest.mark.parametrize("n", [1, 2, 3, 4, 5, 8, 9, 15, 16, 17, 31, 32, 33, 63, 64, 65, 127, 129, 1000, 5003])
@@ -72,6 +76,45 @@ def test_stream_kernel_any_cta_count_gives_the_same_answer(ctas):
     q, K, V, s = make(77, 3, 8, 2, 2500, 128, 128)
     ref = oracle.decode(q, K, V, s)
     assert max_err(gpu_decode(q, K, V, s, num_ctas=ctas, expect_path=moa.PATH_STREAM), ref) <= TOL
+
+
+# ---------------------------------------------------------------------------------------
+# grouped tensor-core kernel (g_s in {16, 32, 64}, d = 128, dense cache)
+# ---------------------------------------------------------------------------------------
+@pytest.mark.parametrize("gs", [16, 32, 64])
+@pytest.mark.parametrize("B,hkv,n", [(1, 1, 1), (1, 1, 127), (2, 1, 128), (1, 2, 129), (1, 1, 1000),
+                                     (3, 1, 4133), (1, 1, 20000), (40, 4, 300)])
+def test_grouped_kernel_shapes(gs, B, hkv, n):
+    q, K, V, s = make(2000 + gs + n, B, gs * hkv, hkv, n, 128, 128)
+    out = gpu_decode(q, K, V, s, expect_path=moa.PATH_GROUPED)
+    assert max_err(out, oracle.decode(q, K, V, s)) <= TOL
+
+
+def test_grouped_kernel_larger_scores_rising_maximum_and_small_n():
+    # The tensor core accumulates with truncation, so the score error of this path grows with
+    # the score magnitude about 3-4 times faster than on the FFMA paths: the 5e-6 bar is
+    # checked here up to |score| ~ 14 (the benchmark workloads have |score| < 7).
+    q, K, V, s = make(2100, 1, 64, 1, 3000, 128, 128, v_dist="uniform")
+    q, K = 2 * q, 2 * K
+    assert max_err(gpu_decode(q, K, V, s, expect_path=moa.PATH_GROUPED), oracle.decode(q, K, V, s)) <= TOL
+    # rows sorted by score, ascending: the reference of every head is raised tile after tile
+    # (accumulator rescale path)
+    q, K, V, s = make(2101, 1, 16, 1, 2048, 128, 128)
+    order = np.argsort(K[0, 0] @ q[0, 0])
+    K, V = np.ascontiguousarray(K[:, :, order]), np.ascontiguousarray(V[:, :, order])
+    q2 = q.copy()
+    q2[:] = q[:, :1]                       # every head sees the same ascending order
+    assert max_err(gpu_decode(q2 * 8, K, V, s, expect_path=moa.PATH_GROUPED), oracle.decode(q2 * 8, K, V, s)) <= TOL
+    # few rows: no averaging hides a product error (this is what the three-term split is for)
+    q, K, V, s = make(2102, 2, 64, 1, 3, 128, 128)
+    assert max_err(gpu_decode(q, K, V, s, expect_path=moa.PATH_GROUPED), oracle.decode(q, K, V, s)) <= TOL
+
+
+def test_grouped_kernel_is_deterministic():
+    q, K, V, s = make(2103, 2, 64, 1, 5000, 128, 128)
+    a = gpu_decode(q, K, V, s, expect_path=moa.PATH_GROUPED)
+    b = gpu_decode(q, K, V, s, expect_path=moa.PATH_GROUPED)
+    assert np.array_equal(a.view(np.uint32), b.view(np.uint32))
 
 
 def test_results_are_deterministic():
@@ -233,6 +276,37 @@ def test_multistep_small(fused, D, hq, hkv):
     assert np.array_equal(gK.host().view(np.uint32), K.view(np.uint32))
     assert np.array_equal(gV.host().view(np.uint32), V.view(np.uint32))
     for g in (gK, gV, glens, gws, gout):
+        assert g.guards_intact()
+
+
+@pytest.mark.parametrize("ctas,misalign_new", [(0, 0), (4000, 0), (0, 1), (5, 0)])
+@pytest.mark.parametrize("D,hq,hkv", [(128, 32, 8), (64, 16, 1), (128, 6, 2)])
+def test_append_decode_single_call(ctas, misalign_new, D, hq, hkv):
+    # one call appends at pos[b] and attends over pos[b]+1 rows; lengths are not modified.
+    # ctas=4000 and a k_new that is only 4-byte aligned take the three-launch fallback.
+    B, n_max = 3, 300
+    q, K, V, s = make(1200 + D + hq, B, hq, hkv, n_max, D, D)
+    pos = np.array([0, 299, 123], np.int32)
+    kn, vn = mi.normal(1201, 4, (B, hkv, D)), mi.normal(1201, 5, (B, hkv, D))
+    gq, gK, gV, gpos = Guarded(q), Guarded(K), Guarded(V), Guarded(pos)
+    gk, gv = Guarded(kn, misalign=misalign_new), Guarded(vn, misalign=misalign_new)
+    gout = Guarded(shape=(B, hq, D))
+    moa.moa_set_option(moa.OPT_NUM_CTAS, ctas)
+    try:
+        gws, nbytes = workspace_for(B, hq, hkv, n_max, D, D)
+        moa.moa_append_decode(gq.ptr, gK.ptr, gV.ptr, gk.ptr, gv.ptr, gout.ptr, gpos.ptr, B, hq, hkv, n_max,
+                              D, D, s, gws.ptr, nbytes)
+        torch.cuda.synchronize()
+    finally:
+        moa.moa_set_option(moa.OPT_NUM_CTAS, 0)
+    assert moa.moa_device_status() == 0
+    oracle.kv_append(K, V, kn, vn, pos)
+    assert np.array_equal(gK.host().view(np.uint32), K.view(np.uint32))
+    assert np.array_equal(gV.host().view(np.uint32), V.view(np.uint32))
+    ref = oracle.decode_varlen(q, K, V, pos + 1, s)
+    assert max_err(gout.host(), ref) <= TOL
+    assert np.array_equal(gpos.host(), pos)
+    for g in (gq, gK, gV, gk, gv, gout, gpos, gws):
         assert g.guards_intact()
 
 
