@@ -212,9 +212,9 @@ static GroupedPlan plan_grouped(const DeviceState &s, int batch, int h_q, int h_
     if (d_k != 128 || d_v != 128 || (g_s != 16 && g_s != 32 && g_s != 64)) return p;
     const long long units = (long long)batch * h_kv;
     if (units > 0x7fffffffLL / 256 || (long long)n > 0x7fffffffLL - 256) return p;
-    // 32 heads per CTA leave room for a ten-deep chunk ring (64 heads: six), which is what
-    // hides the HBM latency; a group of 64 runs as two neighbouring CTAs over the same rows.
-    p.GH = g_s > 32 ? 32 : g_s;
+    // One CTA takes the whole group (measured faster than cutting a group of 64 into two
+    // neighbouring CTAs of 32 heads that read the same rows through L2).
+    p.GH = g_s;
     if (g_grouped_heads == 16 || g_grouped_heads == 32 || g_grouped_heads == 64)
         if (g_grouped_heads <= g_s) p.GH = g_grouped_heads;
     p.share = g_s / p.GH;

@@ -18,10 +18,12 @@
 // same value; it only has to keep exp2 in range): m_ref is raised, and the accumulators
 // rescaled, only when a score exceeds it by more than 2^16.
 //
-// Roles (448 threads): warp 0 TMA producer, warps 1 and 2 MMA issuers (warp 1 also owns the
+// Roles (512 threads): warp 0 TMA producer, warps 1 and 2 MMA issuers (warp 1 also owns the
 // TMEM allocation), warps 4-11 softmax (warp w works on TMEM lane quarter w % 4, i.e. cached
-// rows 32*(w%4).., and on the lower (w < 8) or upper half of the heads), warps 3, 12, 13
-// turn K/V chunks into their lo parts.  Every hand-off is an mbarrier; every wait is bounded.
+// rows 32*(w%4).., and on the lower (w < 8) or upper half of the heads), warps 3 and 12-15
+// turn K chunks into their lo parts.  V chunks are turned into their lo parts by the
+// softmax warps themselves: they would otherwise idle exactly while the weighted-sum
+// products of the previous tile wait for that conversion.  Every hand-off is an mbarrier; every wait is bounded.
 #pragma once
 
 #include <cuda.h>
@@ -40,8 +42,9 @@ struct GroupedCfg {
     static constexpr int NBUF = GH == 64 ? 6 : (GH == 32 ? 10 : 12);   // 16 KB K/V chunk buffers
     static constexpr int CHUNK = 16384;
     static constexpr int OPCH = N1 * 128;          // bytes of one 32-wide k-chunk of the Q / P operand
-    static constexpr int THREADS = 448;            // 14 warps, see the role list above
-    static constexpr int NCONV = 3 * 32;           // converter threads (warps 3, 12, 13)
+    static constexpr int THREADS = 512;            // 16 warps, see the role list above
+    static constexpr int KCONV_WARPS = 5;          // warps 3, 12..15 convert K chunks
+    static constexpr int VCONV_WARPS = 8;          // the softmax warps convert V chunks
     static constexpr int NSOFT = 256;              // softmax threads (warps 4..11)
     static constexpr int HH = GH / 2;              // heads per softmax thread
     static constexpr int PW = HH < 16 ? HH : 16;   // heads handled per TMEM read
@@ -54,10 +57,12 @@ struct GroupedCfg {
     static constexpr uint32_t OFF_TMAX = OFF_ALPHA + GH * 4;
     static constexpr uint32_t OFF_LRED = OFF_TMAX + GH * 4;
     static constexpr uint32_t OFF_BAR = OFF_LRED + 4 * GH * 4;      // lred: [4 row quarters][GH]
-    static constexpr int NBAR = 4 * NBUF + 2 + 2 + 4 + 1;
+    static constexpr int NBAR = 7 * NBUF + 2 + 2 + 4 + 1;   // full/hi/lo per chunk kind, empty, and the tile barriers
     static constexpr uint32_t OFF_TMEM = OFF_BAR + NBAR * 8;
     static constexpr uint32_t OFF_ABORT = OFF_TMEM + 4;
-    static constexpr size_t SMEM_BYTES = OFF_ABORT + 4;
+    static constexpr uint32_t OFF_ACC = OFF_ABORT + 4;        // "weighted sum of this tile adds to the accumulator"
+    static constexpr size_t SMEM_BYTES = OFF_ACC + 4;
+    static constexpr int FOLD_EVERY = 4;           // tiles accumulated by the tensor core between folds
     static_assert(GH == 16 || GH == 32 || GH == 64, "group size");
     static_assert(OFF_RING % 1024 == 0, "swizzled tiles need 1024-byte alignment");
 };
@@ -77,8 +82,10 @@ struct GroupedArgs {
 // Bounded mbarrier wait that also gives up when another role has already failed.
 __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int *abort_flag)
 {
+    // test_wait polls without suspending the thread: the hand-offs of this kernel are short
+    // and on the critical path, so a prompt wake-up matters more than the issue slots
     for (uint32_t it = 0; it < kWaitLimit; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
+        if (mbar_test_wait(bar, parity)) return true;
         if ((it & 255u) == 255u && *abort_flag) return false;
     }
     *abort_flag = 1;
@@ -152,17 +159,22 @@ grouped_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_co
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + C::OFF_BAR);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + C::OFF_TMEM);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + C::OFF_ABORT);
+    volatile uint32_t *acc_flag = reinterpret_cast<volatile uint32_t *>(smem + C::OFF_ACC);
 
     const uint32_t sbase = smem_u32(smem);
     const uint32_t sQ = sbase + C::OFF_Q, sP = sbase + C::OFF_P, sRing = sbase + C::OFF_RING;
-    auto bar_full = [&](int b) { return smem_u32(&bars[b]); };
-    auto bar_hi = [&](int b) { return smem_u32(&bars[NBUF + b]); };
-    auto bar_lo = [&](int b) { return smem_u32(&bars[2 * NBUF + b]); };
-    auto bar_empty = [&](int b) { return smem_u32(&bars[3 * NBUF + b]); };
-    auto bar_sfull = [&](int s) { return smem_u32(&bars[4 * NBUF + s]); };
-    auto bar_sfree = [&](int s) { return smem_u32(&bars[4 * NBUF + 2 + s]); };
-    auto bar_pfull = [&](int c) { return smem_u32(&bars[4 * NBUF + 4 + c]); };
-    const uint32_t bar_pvdone = smem_u32(&bars[4 * NBUF + 8]);
+    // A ring buffer is used by K chunks and V chunks in turn, but the roles of one kind never
+    // look at the other kind's chunks.  A parity wait is only safe for a waiter that sees
+    // every phase of its barrier, so "data landed", "hi product done" and "lo part ready"
+    // exist once per kind; each role keeps one parity bit per buffer for its own kind.
+    auto bar_full = [&](bool k, int b) { return smem_u32(&bars[(k ? 0 : NBUF) + b]); };
+    auto bar_hi = [&](bool k, int b) { return smem_u32(&bars[(k ? 2 : 3) * NBUF + b]); };
+    auto bar_lo = [&](bool k, int b) { return smem_u32(&bars[(k ? 4 : 5) * NBUF + b]); };
+    auto bar_empty = [&](int b) { return smem_u32(&bars[6 * NBUF + b]); };
+    auto bar_sfull = [&](int s) { return smem_u32(&bars[7 * NBUF + s]); };
+    auto bar_sfree = [&](int s) { return smem_u32(&bars[7 * NBUF + 2 + s]); };
+    auto bar_pfull = [&](int c) { return smem_u32(&bars[7 * NBUF + 4 + c]); };
+    const uint32_t bar_pvdone = smem_u32(&bars[7 * NBUF + 8]);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     // CTA order: the virtual heads that share one stored K/V head are neighbours, so they run
@@ -181,14 +193,18 @@ grouped_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_co
     // ---- set-up --------------------------------------------------------------------------
     if (tid == 0) {
         for (int i = 0; i < NBUF; ++i) {
-            mbar_init(bar_full(i), 1); mbar_init(bar_hi(i), 1);
-            mbar_init(bar_lo(i), C::NCONV / 32); mbar_init(bar_empty(i), 1);
+            for (int k = 0; k < 2; ++k) {
+                mbar_init(bar_full(k != 0, i), 1); mbar_init(bar_hi(k != 0, i), 1);
+                mbar_init(bar_lo(k != 0, i), k != 0 ? C::KCONV_WARPS : C::VCONV_WARPS);
+            }
+            mbar_init(bar_empty(i), 1);
         }
         for (int i = 0; i < 2; ++i) { mbar_init(bar_sfull(i), 1); mbar_init(bar_sfree(i), 8); }
         for (int i = 0; i < 4; ++i) mbar_init(bar_pfull(i), 2);
         mbar_init(bar_pvdone, 1);
         mbar_fence_init();
         *abort_flag = 0;
+        *acc_flag = 0u;
         tc::prefetch_tmap(&tmapK);
         tc::prefetch_tmap(&tmapV);
     }
@@ -224,13 +240,14 @@ grouped_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_co
                 const int buf = s.seq % NBUF, use = s.seq / NBUF;
                 if (use > 0 && !wait_or_abort(bar_empty(buf), (uint32_t)(use - 1) & 1u, abort_flag)) break;
                 const uint32_t dst = sRing + (uint32_t)buf * C::CHUNK;
-                mbar_expect_tx(bar_full(buf), C::CHUNK);
+                const uint32_t fb = bar_full(s.is_k, buf);
+                mbar_expect_tx(fb, C::CHUNK);
                 const int row = row_base + s.t * C::TILE;
                 if (s.is_k) {
-                    tc::tma_load_3d(dst, &tmapK, 32 * s.c, row, unit, bar_full(buf));
+                    tc::tma_load_3d(dst, &tmapK, 32 * s.c, row, unit, fb);
                 } else {
                     for (int dg = 0; dg < 4; ++dg)
-                        tc::tma_load_3d(dst + dg * 4096, &tmapV, 32 * dg, row + 32 * s.c, unit, bar_full(buf));
+                        tc::tma_load_3d(dst + dg * 4096, &tmapV, 32 * dg, row + 32 * s.c, unit, fb);
                 }
             }
         }
@@ -269,39 +286,43 @@ grouped_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_co
                 return false;
             };
             bool ok = true;
+            uint32_t par_hi = 0, par_lo = 0;      // per ring buffer: parity of this kind's next use
             for (int t = 0; ok && t < T; ++t) {
                 const int gi = kind_k ? (t == 0 ? 0 : 2 * t - 1) : (t < T - 1 ? 2 * t + 2 : 2 * T - 1);
                 const int seq0 = 4 * gi;
                 const uint32_t d_hi = kind_k ? tS_of(t) : tO;
                 if (kind_k && t >= 2) ok = spin(bar_sfree(t & 1), (uint32_t)(t / 2 - 1) & 1u);
+                uint32_t acc_first = 0u;      // does the tile's first product add to the accumulator?
                 if (!kind_k) {
-                    // chunk 0 overwrites the whole per-tile accumulator, which every softmax
-                    // warp reads while folding the previous tile: wait for all of them
+                    // chunk 0 may overwrite the whole accumulator, which every softmax warp
+                    // reads while folding: wait for all of them
                     for (int w = 0; ok && w < 4; ++w) ok = spin(bar_pfull(w), (uint32_t)t & 1u);
+                    acc_first = *acc_flag;
                 }
+                const int b0 = seq0 % NBUF;
 #pragma unroll
                 for (int step = 0; step < 8; ++step) {
                     // steps: H0 H1 H2 L0 H3 L1 L2 L3
                     const bool is_hi = (step < 3) || (step == 4);
                     const int c = is_hi ? (step < 3 ? step : 3) : (step == 3 ? 0 : step - 4);
-                    const int seq = seq0 + c;
-                    const int buf = seq % NBUF;
-                    const uint32_t ph = (uint32_t)(seq / NBUF) & 1u;
+                    const int buf = (b0 + c >= NBUF) ? b0 + c - NBUF : b0 + c;
                     if (!ok) break;
-                    ok = spin(is_hi ? bar_full(buf) : bar_lo(buf), ph);
+                    if (is_hi) { ok = spin(bar_full(kind_k, buf), (par_hi >> buf) & 1u); par_hi ^= 1u << buf; }
+                    else { ok = spin(bar_lo(kind_k, buf), (par_lo >> buf) & 1u); par_lo ^= 1u << buf; }
                     if (!ok) break;
                     tc::fence_after_sync();
                     const uint32_t a_lo = a_base + (uint32_t)buf * (C::CHUNK >> 4);
                     const uint32_t b_lo = b_base + (uint32_t)c * (C::OPCH >> 4);
                     if (is_hi) {
-                        // the first product of a tile overwrites its accumulator (the weighted
-                        // sum is folded into an fp32 master copy by the softmax group every tile)
-                        tc::mma_tf32_ss(d_hi, tc::pack64(a_lo, a_hiword), tc::pack64(b_lo, b_hiword), idesc_hi, (uint32_t)c);
+                        // the first product of a tile overwrites the accumulator unless the softmax
+                        // group said to keep adding (it folds the weighted sum into an fp32 master
+                        // copy every few tiles, because the tensor core accumulates with truncation)
+                        tc::mma_tf32_ss(d_hi, tc::pack64(a_lo, a_hiword), tc::pack64(b_lo, b_hiword), idesc_hi, (uint32_t)c | acc_first);
 #pragma unroll
                         for (uint32_t ks = 1; ks < 4; ++ks)
                             tc::mma_tf32_ss(d_hi, tc::pack64(a_lo + ks * a_step, a_hiword),
                                             tc::pack64(b_lo + ks * 2u, b_hiword), idesc_hi, 1u);
-                        tc::mma_commit(bar_hi(buf));
+                        tc::mma_commit(bar_hi(kind_k, buf));
                     } else {
 #pragma unroll
                         for (uint32_t ks = 0; ks < 4; ++ks)
@@ -326,9 +347,38 @@ grouped_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_co
         for (int g = 0; g < HH; ++g) lsum[g] = 0.f;
         unsigned char *pch = smem + C::OFF_P + (uint32_t)q4 * C::OPCH;     // this row quarter's P chunk
         bool ok = true;
+        uint32_t par_v = 0;                          // per ring buffer: parity of the next V use
+        bool have_master = false;                    // has anything been folded into the master copy?
+        // Turn the four V chunks of tile tv into their lo parts, each as soon as its hi
+        // product has completed (all 256 threads: four float4 each per chunk).
+        auto convert_v = [&](int tv) -> bool {
+            const int seq0 = 4 * (tv < T - 1 ? 2 * tv + 2 : 2 * T - 1);
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+                const int buf = (seq0 + c) % NBUF;
+                const uint32_t ph = (par_v >> buf) & 1u;
+                par_v ^= 1u << buf;
+                if (!wait_or_abort(bar_hi(false, buf), ph, abort_flag)) return false;
+                float4 *pv = reinterpret_cast<float4 *>(smem + C::OFF_RING + (uint32_t)buf * C::CHUNK);
+                float4 v[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) v[i] = pv[st + i * NS];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    v[i].x -= tf32_hi(v[i].x); v[i].y -= tf32_hi(v[i].y);
+                    v[i].z -= tf32_hi(v[i].z); v[i].w -= tf32_hi(v[i].w);
+                    pv[st + i * NS] = v[i];
+                }
+                tc::fence_async_smem();
+                __syncwarp();
+                if (lane == 0) tc::mbar_arrive(bar_lo(false, buf));
+            }
+            return true;
+        };
         for (int t = 0; ok && t < T; ++t) {
             const int sb = t & 1;
-            ok = wait_or_abort(bar_sfull(sb), (uint32_t)(t >> 1) & 1u, abort_flag);
+            if (t > 0) ok = convert_v(t - 1);        // (a failure is shared at the vote just below)
+            ok = ok && wait_or_abort(bar_sfull(sb), (uint32_t)(t >> 1) & 1u, abort_flag);
             if (named_or(1, NS, !ok)) { ok = false; break; }     // leave together or not at all
             tc::fence_after_sync();
             const bool valid = (row_base + t * C::TILE + row_in_tile) < a.n;
@@ -395,30 +445,36 @@ grouped_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_co
             if (lane == 0) tc::mbar_arrive(bar_sfree(sb));
 #pragma unroll
             for (int g = 0; g < HH; ++g) lsum[g] += p[g];
-            // The previous tile's weighted sum is complete: fold it into the fp32 master copy
-            // (the tensor core accumulates with truncation, so its chains are kept one tile
-            // long), which also frees the P buffers and the per-tile accumulator.
+            // The previous tile's weighted sum is complete, so the P buffers are free.  Every
+            // FOLD_EVERY tiles, and whenever the references were raised, the accumulator is
+            // folded into the fp32 master copy (the tensor core accumulates with truncation, so
+            // its chains are kept short) and the next tile starts it afresh.
             if (t > 0) {
                 ok = wait_or_abort(bar_pvdone, (uint32_t)(t - 1) & 1u, abort_flag);
                 if (named_or(1, NS, !ok)) { ok = false; break; }
                 tc::fence_after_sync();
+                const bool fold = raise || (t % C::FOLD_EVERY) == 0;
+                if (fold) {
 #pragma unroll
-                for (int j = 0; j < NP; ++j) {
-                    uint32_t hi[PW], lo[PW], ms[PW];
-                    tc::tmem_ld_piece<PW>(tO + lane_addr + h0 + PW * j, hi);
-                    tc::tmem_ld_piece<PW>(tO + lane_addr + GH + h0 + PW * j, lo);
-                    if (t > 1) tc::tmem_ld_piece<PW>(tOm + lane_addr + h0 + PW * j, ms);
-                    tc::tmem_ld_wait();
+                    for (int j = 0; j < NP; ++j) {
+                        uint32_t hi[PW], lo[PW], ms[PW];
+                        tc::tmem_ld_piece<PW>(tO + lane_addr + h0 + PW * j, hi);
+                        tc::tmem_ld_piece<PW>(tO + lane_addr + GH + h0 + PW * j, lo);
+                        if (have_master) tc::tmem_ld_piece<PW>(tOm + lane_addr + h0 + PW * j, ms);
+                        tc::tmem_ld_wait();
 #pragma unroll
-                    for (int i = 0; i < PW; ++i) {
-                        float add = __uint_as_float(hi[i]) + __uint_as_float(lo[i]);
-                        if (t > 1) add += __uint_as_float(ms[i]);
-                        if (raise) add *= alpha_s[h0 + PW * j + i];
-                        ms[i] = __float_as_uint(add);
+                        for (int i = 0; i < PW; ++i) {
+                            float add = __uint_as_float(hi[i]) + __uint_as_float(lo[i]);
+                            if (have_master) add += __uint_as_float(ms[i]);
+                            if (raise) add *= alpha_s[h0 + PW * j + i];
+                            ms[i] = __float_as_uint(add);
+                        }
+                        tc::tmem_st_piece<PW>(tOm + lane_addr + h0 + PW * j, ms);
                     }
-                    tc::tmem_st_piece<PW>(tOm + lane_addr + h0 + PW * j, ms);
+                    tc::tmem_st_wait();
+                    have_master = true;
                 }
-                tc::tmem_st_wait();
+                if (st == 0) *acc_flag = fold ? 0u : 1u;     // read by the issuer after the P barriers
             }
             // probabilities, split into hi|lo, as the K-major B operand of this row quarter
 #pragma unroll
@@ -434,7 +490,7 @@ grouped_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_co
         }
         // ---- epilogue: this split's partial (m_ref, l, o) per head
         if (ok) {                            // (ok is uniform across the group here)
-            ok = wait_or_abort(bar_pvdone, (uint32_t)(T - 1) & 1u, abort_flag);
+            ok = convert_v(T - 1) && wait_or_abort(bar_pvdone, (uint32_t)(T - 1) & 1u, abort_flag);
             if (named_or(1, NS, !ok)) ok = false;
         }
         if (ok) {
@@ -454,12 +510,12 @@ grouped_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_co
                 uint32_t hi[PW], lo[PW], ms[PW];
                 tc::tmem_ld_piece<PW>(tO + lane_addr + h0 + PW * j, hi);
                 tc::tmem_ld_piece<PW>(tO + lane_addr + GH + h0 + PW * j, lo);
-                if (T > 1) tc::tmem_ld_piece<PW>(tOm + lane_addr + h0 + PW * j, ms);
+                if (have_master) tc::tmem_ld_piece<PW>(tOm + lane_addr + h0 + PW * j, ms);
                 tc::tmem_ld_wait();
 #pragma unroll
                 for (int i = 0; i < PW; ++i) {
                     float add = __uint_as_float(hi[i]) + __uint_as_float(lo[i]);
-                    if (T > 1) add += __uint_as_float(ms[i]);
+                    if (have_master) add += __uint_as_float(ms[i]);
                     slot[(size_t)(h0 + PW * j + i) * PS + d] = add;
                 }
             }
@@ -469,23 +525,36 @@ grouped_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_co
             }
         }
     } else {
-        // ================= converters: chunk -> its lo part, in place =================
-        const int ct = (warp == 3 ? 0 : warp - 11) * 32 + lane;            // 0..95
+        // ================= K converters: chunk -> its lo part, in place =================
+        constexpr int TT = C::KCONV_WARPS * 32;                        // 160 threads
+        constexpr int FULL = (C::CHUNK / 16) / TT;                     // float4 every thread handles
+        const int ct = (warp == 3 ? 0 : warp - 11) * 32 + lane;
         bool ok = true;
+        uint32_t par = 0;                          // per ring buffer: parity of the next K use
         for (ChunkSeq s(T); ok && !s.done; s.next()) {
-            const int buf = s.seq % NBUF, use = s.seq / NBUF;
-            ok = wait_or_abort(bar_full(buf), (uint32_t)use & 1u, abort_flag) &&
-                 wait_or_abort(bar_hi(buf), (uint32_t)use & 1u, abort_flag);
+            if (!s.is_k) continue;
+            const int buf = s.seq % NBUF;
+            const uint32_t ph = (par >> buf) & 1u;
+            par ^= 1u << buf;
+            ok = wait_or_abort(bar_hi(true, buf), ph, abort_flag);
             if (!ok) break;
             float4 *p = reinterpret_cast<float4 *>(smem + C::OFF_RING + (uint32_t)buf * C::CHUNK);
-            for (int i = ct; i < C::CHUNK / 16; i += C::NCONV) {
-                float4 v = p[i];
-                v.x -= tf32_hi(v.x); v.y -= tf32_hi(v.y); v.z -= tf32_hi(v.z); v.w -= tf32_hi(v.w);
-                p[i] = v;
+            float4 v[FULL + 1];
+#pragma unroll
+            for (int i = 0; i < FULL; ++i) v[i] = p[ct + i * TT];
+            const bool extra = ct + FULL * TT < C::CHUNK / 16;
+            if (extra) v[FULL] = p[ct + FULL * TT];
+#pragma unroll
+            for (int i = 0; i <= FULL; ++i) {
+                v[i].x -= tf32_hi(v[i].x); v[i].y -= tf32_hi(v[i].y);
+                v[i].z -= tf32_hi(v[i].z); v[i].w -= tf32_hi(v[i].w);
             }
+#pragma unroll
+            for (int i = 0; i < FULL; ++i) p[ct + i * TT] = v[i];
+            if (extra) p[ct + FULL * TT] = v[FULL];
             tc::fence_async_smem();
             __syncwarp();
-            if (lane == 0) tc::mbar_arrive(bar_lo(buf));
+            if (lane == 0) tc::mbar_arrive(bar_lo(true, buf));
         }
     }
 
