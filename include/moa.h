@@ -212,9 +212,11 @@ int moa_last_path(void);
 /*
  * Launch accounting for benchmarks (host-only state plus CUDA events; off by default).
  * moa_profile(1) clears the counters and starts counting every kernel the library
- * launches; while on, each launch of the dominant decode kernel (streaming, grouped or
- * generic) is also bracketed by a pair of CUDA events on the caller's stream (at most
- * MOA_PROFILE_MAX_EVENTS pairs are kept; later launches are counted but not timed).
+ * launches.  moa_profile(2) does the same and also brackets each launch of the dominant
+ * decode kernel (streaming, grouped or generic) with a pair of CUDA events on the caller's
+ * stream (at most MOA_PROFILE_MAX_EVENTS pairs are kept; later launches are counted but
+ * not timed).  The events cost a few microseconds per launch, so a throughput
+ * measurement should use mode 1.
  * moa_profile_read synchronises the device and reports the summed event time of the
  * timed decode-kernel launches in milliseconds, how many of them were timed, and the
  * total number of kernels launched since moa_profile(1).  Any pointer may be NULL.

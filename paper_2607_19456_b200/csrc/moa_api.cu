@@ -33,6 +33,7 @@ static int g_last_path = 0;
 
 // ---- launch accounting (moa_profile) ----------------------------------------------------
 static bool g_prof_on = false;
+static bool g_prof_events = false;    // also bracket the dominant kernel with CUDA events
 static long long g_prof_all = 0;          // kernels launched while profiling
 static long long g_prof_timed = 0;        // decode-kernel launches bracketed by events
 static cudaEvent_t *g_prof_ev = nullptr;  // 2 * MOA_PROFILE_MAX_EVENTS events, created lazily
@@ -42,7 +43,7 @@ struct TimedLaunch {                      // RAII: event before / after the domi
     long long slot = -1;
     explicit TimedLaunch(cudaStream_t s) : st(s)
     {
-        if (!g_prof_on || g_prof_timed >= MOA_PROFILE_MAX_EVENTS) return;
+        if (!g_prof_on || !g_prof_events || g_prof_timed >= MOA_PROFILE_MAX_EVENTS) return;
         if (!g_prof_ev) {
             g_prof_ev = new cudaEvent_t[2 * MOA_PROFILE_MAX_EVENTS]();
             for (int i = 0; i < 2 * MOA_PROFILE_MAX_EVENTS; ++i)
@@ -725,6 +726,7 @@ int moa_last_path(void) { return g_last_path; }
 int moa_profile(int enable)
 {
     g_prof_on = enable != 0;
+    g_prof_events = enable == 2;
     if (g_prof_on) { g_prof_all = 0; g_prof_timed = 0; }
     return MOA_OK;
 }

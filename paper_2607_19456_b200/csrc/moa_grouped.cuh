@@ -151,7 +151,8 @@ grouped_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_co
                       const GroupedArgs a)
 {
     constexpr int GH = C::GH, N1 = C::N1, NBUF = C::NBUF, PS = C::PS;
-    extern __shared__ __align__(1024) unsigned char smem[];
+    extern __shared__ __align__(1024) unsigned char smem_g[];
+    unsigned char *const smem = smem_g;
     float *mref = reinterpret_cast<float *>(smem + C::OFF_MREF);
     float *alpha_s = reinterpret_cast<float *>(smem + C::OFF_ALPHA);
     uint32_t *tmax = reinterpret_cast<uint32_t *>(smem + C::OFF_TMAX);
