@@ -261,7 +261,11 @@ grouped_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_co
         // ready, so a chunk waiting for its converters never holds up the ones behind it.
         // A lone thread retires an instruction every few cycles, so the issue path is kept to
         // a handful of instructions per MMA (descriptor words are advanced, not rebuilt).
-        if (lane == 0) {
+        {
+            // Polling a barrier costs a shared-memory round trip of a few hundred cycles, far
+            // more than issuing a product, so the whole warp polls: lane s checks the barrier
+            // that step s of the current group waits for, one ballot tells lane 0 how many of
+            // the next steps can go, and lane 0 issues them back to back.
             const bool kind_k = (warp == 1);
             const uint32_t idesc_hi = kind_k ? tc::idesc_tf32(128, N1, false, false) : tc::idesc_tf32(128, N1, true, false);
             const uint32_t idesc_lo = kind_k ? tc::idesc_tf32(128, GH, false, false) : tc::idesc_tf32(128, GH, true, false);
@@ -277,62 +281,83 @@ grouped_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_co
             // result differ from run to run.  The two-chunk lag gives the converters time.
             // In the chunk sequence the K groups sit at group indices 0,1,3,5,... and the V
             // groups at 2,4,...,2T-2,2T-1; a group's first chunk is number 4*index.
-            auto spin = [&](uint32_t bar, uint32_t parity) -> bool {      // bounded, non-suspending
-                for (uint32_t it = 0; it < kWaitLimit; ++it) {
-                    if (mbar_test_wait(bar, parity)) return true;
-                    if ((it & 255u) == 255u && *abort_flag) return false;
-                }
-                *abort_flag = 1;
-                raise_status(MOA_STATUS_WAIT_TIMEOUT);
-                return false;
-            };
+            // step s of a group: is it a hi product, and of which chunk?
+            const bool my_is_hi = (lane < 3) || (lane == 4);
+            const int my_c = my_is_hi ? (lane < 3 ? lane : 3) : (lane == 3 ? 0 : lane - 4);
             bool ok = true;
-            uint32_t par_hi = 0, par_lo = 0;      // per ring buffer: parity of this kind's next use
+            uint32_t par = 0;                      // per ring buffer: parity of this kind's next use
+            uint32_t idle = 0;
             for (int t = 0; ok && t < T; ++t) {
                 const int gi = kind_k ? (t == 0 ? 0 : 2 * t - 1) : (t < T - 1 ? 2 * t + 2 : 2 * T - 1);
-                const int seq0 = 4 * gi;
+                const int b0 = (4 * gi) % NBUF;
                 const uint32_t d_hi = kind_k ? tS_of(t) : tO;
-                if (kind_k && t >= 2) ok = spin(bar_sfree(t & 1), (uint32_t)(t / 2 - 1) & 1u);
-                uint32_t acc_first = 0u;      // does the tile's first product add to the accumulator?
-                if (!kind_k) {
-                    // chunk 0 may overwrite the whole accumulator, which every softmax warp
-                    // reads while folding: wait for all of them
-                    for (int w = 0; ok && w < 4; ++w) ok = spin(bar_pfull(w), (uint32_t)t & 1u);
-                    acc_first = *acc_flag;
+                // ---- group dependencies: the score buffer is free / all probabilities are stored
+                // (chunk 0 of a weighted sum may overwrite the whole accumulator, which every
+                // softmax warp reads while folding, so all of them have to be done)
+                for (;;) {
+                    bool r = true;
+                    if (kind_k) { if (t >= 2 && lane == 0) r = mbar_test_wait(bar_sfree(t & 1), (uint32_t)(t / 2 - 1) & 1u); }
+                    else if (lane < 4) r = mbar_test_wait(bar_pfull(lane), (uint32_t)t & 1u);
+                    if (__all_sync(0xffffffffu, r)) break;
+                    if (++idle >= kWaitLimit) { if (lane == 0) { *abort_flag = 1; raise_status(MOA_STATUS_WAIT_TIMEOUT); } ok = false; break; }
+                    if ((idle & 255u) == 255u && *abort_flag) { ok = false; break; }
                 }
-                const int b0 = seq0 % NBUF;
-#pragma unroll
-                for (int step = 0; step < 8; ++step) {
-                    // steps: H0 H1 H2 L0 H3 L1 L2 L3
-                    const bool is_hi = (step < 3) || (step == 4);
-                    const int c = is_hi ? (step < 3 ? step : 3) : (step == 3 ? 0 : step - 4);
-                    const int buf = (b0 + c >= NBUF) ? b0 + c - NBUF : b0 + c;
-                    if (!ok) break;
-                    if (is_hi) { ok = spin(bar_full(kind_k, buf), (par_hi >> buf) & 1u); par_hi ^= 1u << buf; }
-                    else { ok = spin(bar_lo(kind_k, buf), (par_lo >> buf) & 1u); par_lo ^= 1u << buf; }
-                    if (!ok) break;
-                    tc::fence_after_sync();
-                    const uint32_t a_lo = a_base + (uint32_t)buf * (C::CHUNK >> 4);
-                    const uint32_t b_lo = b_base + (uint32_t)c * (C::OPCH >> 4);
-                    if (is_hi) {
-                        // the first product of a tile overwrites the accumulator unless the softmax
-                        // group said to keep adding (it folds the weighted sum into an fp32 master
-                        // copy every few tiles, because the tensor core accumulates with truncation)
-                        tc::mma_tf32_ss(d_hi, tc::pack64(a_lo, a_hiword), tc::pack64(b_lo, b_hiword), idesc_hi, (uint32_t)c | acc_first);
-#pragma unroll
-                        for (uint32_t ks = 1; ks < 4; ++ks)
-                            tc::mma_tf32_ss(d_hi, tc::pack64(a_lo + ks * a_step, a_hiword),
-                                            tc::pack64(b_lo + ks * 2u, b_hiword), idesc_hi, 1u);
-                        tc::mma_commit(bar_hi(kind_k, buf));
-                    } else {
-#pragma unroll
-                        for (uint32_t ks = 0; ks < 4; ++ks)
-                            tc::mma_tf32_ss(d_hi + GH, tc::pack64(a_lo + ks * a_step, a_hiword),
-                                            tc::pack64(b_lo + ks * 2u, b_hiword), idesc_lo, 1u);
-                        tc::mma_commit(bar_empty(buf));
-                        if (c == 3) tc::mma_commit(kind_k ? bar_sfull(t & 1) : bar_pvdone);
+                if (!ok) break;
+                idle = 0;
+                const uint32_t acc_first = kind_k ? 0u : *acc_flag;   // does the tile add to the accumulator?
+                // this lane's barrier for its step
+                const int my_buf = (b0 + my_c >= NBUF) ? b0 + my_c - NBUF : b0 + my_c;
+                const uint32_t my_bar = my_is_hi ? bar_full(kind_k, my_buf) : bar_lo(kind_k, my_buf);
+                const uint32_t my_par = (par >> my_buf) & 1u;
+                int step = 0;
+                while (step < 8) {
+                    const bool r = (lane < 8 && lane >= step) ? mbar_test_wait(my_bar, my_par) : false;
+                    const uint32_t m = __ballot_sync(0xffffffffu, r) >> step;
+                    const int run = __ffs(~m) - 1;               // consecutive ready steps from `step`
+                    if (run == 0) {
+                        if (++idle >= kWaitLimit) { if (lane == 0) { *abort_flag = 1; raise_status(MOA_STATUS_WAIT_TIMEOUT); } ok = false; break; }
+                        if ((idle & 255u) == 255u && *abort_flag) { ok = false; break; }
+                        continue;
                     }
+                    idle = 0;
+                    if (lane == 0) {
+                        tc::fence_after_sync();
+#pragma unroll
+                        for (int sidx = 0; sidx < 8; ++sidx) {
+                            if (sidx < step || sidx >= step + run) continue;
+                            const bool is_hi = (sidx < 3) || (sidx == 4);
+                            const int c = is_hi ? (sidx < 3 ? sidx : 3) : (sidx == 3 ? 0 : sidx - 4);
+                            const int buf = (b0 + c >= NBUF) ? b0 + c - NBUF : b0 + c;
+                            const uint32_t a_lo = a_base + (uint32_t)buf * (C::CHUNK >> 4);
+                            const uint32_t b_lo = b_base + (uint32_t)c * (C::OPCH >> 4);
+                            if (is_hi) {
+                                // the first product of a tile overwrites the accumulator unless the
+                                // softmax group said to keep adding (it folds the weighted sum into an
+                                // fp32 master copy every few tiles, because the tensor core
+                                // accumulates with truncation)
+                                tc::mma_tf32_ss(d_hi, tc::pack64(a_lo, a_hiword), tc::pack64(b_lo, b_hiword), idesc_hi,
+                                                (uint32_t)c | acc_first);
+#pragma unroll
+                                for (uint32_t ks = 1; ks < 4; ++ks)
+                                    tc::mma_tf32_ss(d_hi, tc::pack64(a_lo + ks * a_step, a_hiword),
+                                                    tc::pack64(b_lo + ks * 2u, b_hiword), idesc_hi, 1u);
+                                tc::mma_commit(bar_hi(kind_k, buf));
+                            } else {
+#pragma unroll
+                                for (uint32_t ks = 0; ks < 4; ++ks)
+                                    tc::mma_tf32_ss(d_hi + GH, tc::pack64(a_lo + ks * a_step, a_hiword),
+                                                    tc::pack64(b_lo + ks * 2u, b_hiword), idesc_lo, 1u);
+                                tc::mma_commit(bar_empty(buf));
+                                if (c == 3) tc::mma_commit(kind_k ? bar_sfull(t & 1) : bar_pvdone);
+                            }
+                        }
+                    }
+                    step += run;
+                    __syncwarp();
                 }
+                // this kind has now used the four buffers once more
+#pragma unroll
+                for (int c = 0; c < 4; ++c) par ^= 1u << ((b0 + c >= NBUF) ? b0 + c - NBUF : b0 + c);
             }
         }
     } else if (warp >= 4 && warp < 12) {
