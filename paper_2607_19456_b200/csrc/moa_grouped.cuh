@@ -590,6 +590,8 @@ grouped_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_co
 }
 
 // Merge the per-split partials of the grouped kernel.  One warp per (batch, query head).
+// The (m, l) pairs of up to 32 splits are read by the lanes in parallel; the weighted-sum
+// rows are then accumulated split by split, in split order, with independent loads.
 template <int GH>
 __global__ void __launch_bounds__(128) grouped_combine_kernel(const GroupedArgs a)
 {
@@ -605,16 +607,29 @@ __global__ void __launch_bounds__(128) grouped_combine_kernel(const GroupedArgs 
     const float *base = a.ws + ((size_t)unit * a.splits * GH + g) * PS;
     const size_t stride = (size_t)GH * PS;
     float M = -INFINITY;
-    for (int s = 0; s < used; ++s) M = fmaxf(M, base[s * stride + 128]);
+    for (int s0 = 0; s0 < used; s0 += 32) {
+        float m = (s0 + lane < used) ? base[(size_t)(s0 + lane) * stride + 128] : -INFINITY;
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+        M = fmaxf(M, m);
+    }
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float L = 0.f;
-    for (int s = 0; s < used; ++s) {
-        const float *p = base + s * stride;
-        const float f = exp2_diff(p[128], M);
-        L = fmaf(p[129], f, L);
-        const float4 t = *reinterpret_cast<const float4 *>(p + lane * 4);
-        acc.x = fmaf(t.x, f, acc.x); acc.y = fmaf(t.y, f, acc.y);
-        acc.z = fmaf(t.z, f, acc.z); acc.w = fmaf(t.w, f, acc.w);
+    for (int s0 = 0; s0 < used; s0 += 32) {
+        const bool mine = s0 + lane < used;
+        const float f_mine = mine ? exp2_diff(base[(size_t)(s0 + lane) * stride + 128], M) : 0.f;
+        float lf = mine ? base[(size_t)(s0 + lane) * stride + 129] * f_mine : 0.f;
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) lf += __shfl_xor_sync(0xffffffffu, lf, off);
+        L += lf;
+        const int cnt = (used - s0 < 32) ? used - s0 : 32;
+#pragma unroll 4
+        for (int j = 0; j < cnt; ++j) {
+            const float f = __shfl_sync(0xffffffffu, f_mine, j);
+            const float4 t = *reinterpret_cast<const float4 *>(base + (size_t)(s0 + j) * stride + lane * 4);
+            acc.x = fmaf(t.x, f, acc.x); acc.y = fmaf(t.y, f, acc.y);
+            acc.z = fmaf(t.z, f, acc.z); acc.w = fmaf(t.w, f, acc.w);
+        }
     }
     const float inv = 1.0f / L;
     *reinterpret_cast<float4 *>(a.out + ((size_t)b * a.h_q + gq) * 128 + lane * 4) =
