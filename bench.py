@@ -41,7 +41,10 @@ L2_BYTES_ASSUMED = 126 * 1024 * 1024
 # DRAM traffic of one launch of the dominant kernel, from an ncu capture
 # (dram__bytes_read.sum + dram__bytes_write.sum), per workload; the summaries these come
 # from are kept as text under profiles/.  None = not captured.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    "gqa": 1074650112 + 3750144,        # profiles/stream_decode_kernel_gqa.md (full-size launch)
+    "mqa_long": 537828864 + 5385984,    # profiles/grouped_decode_kernel_mqa_long.md (full-size launch)
+}
 
 
 def env_int(name, default):
