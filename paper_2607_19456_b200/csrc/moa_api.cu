@@ -117,13 +117,14 @@ static int stream_group(int g_s, int *share)
 static int rows_per_block(int D, int G)
 {
     if (D == 128) return (G == 8) ? 4 : 8;
-    return (G == 1 || G == 2) ? 16 : (G == 4 ? 8 : 4);
+    if (D == 64) return (G == 1 || G == 2) ? 16 : (G == 4 ? 8 : 4);
+    return 32 / G;                       // D == 32
 }
 
 static StreamPlan plan_stream(int g_s, int d_k, int d_v)
 {
     StreamPlan p;
-    if (d_k != d_v || (d_k != 64 && d_k != 128)) return p;
+    if (d_k != d_v || (d_k != 32 && d_k != 64 && d_k != 128)) return p;
     p.D = d_k;
     p.G = stream_group(g_s, &p.share);
     p.R = rows_per_block(p.D, p.G);
@@ -179,20 +180,30 @@ static cudaError_t launch_stream_cfg(const DecodeArgs &a, int num_ctas, cudaStre
 static cudaError_t launch_stream(const StreamPlan &p, const DecodeArgs &a, int num_ctas,
                                  cudaStream_t st)
 {
+    // The heavier configurations (many FMAs per fetched byte) run 16 warps per CTA: with
+    // eight, two warps per scheduler cannot hide the shuffle and FMA latencies.
     //                                   D    G  RV  S  W
     if (p.D == 128) {
         switch (p.G) {
         case 1: return launch_stream_cfg<StreamCfg<128, 1, 8, 3, 8>>(a, num_ctas, st);
         case 2: return launch_stream_cfg<StreamCfg<128, 2, 8, 3, 8>>(a, num_ctas, st);
         case 4: return launch_stream_cfg<StreamCfg<128, 4, 8, 3, 8>>(a, num_ctas, st);
-        default: return launch_stream_cfg<StreamCfg<128, 8, 4, 5, 8>>(a, num_ctas, st);
+        default: return launch_stream_cfg<StreamCfg<128, 8, 4, 2, 16>>(a, num_ctas, st);
         }
     }
-    switch (p.G) {
-    case 1: return launch_stream_cfg<StreamCfg<64, 1, 8, 3, 8>>(a, num_ctas, st);
-    case 2: return launch_stream_cfg<StreamCfg<64, 2, 8, 3, 8>>(a, num_ctas, st);
-    case 4: return launch_stream_cfg<StreamCfg<64, 4, 4, 6, 8>>(a, num_ctas, st);
-    default: return launch_stream_cfg<StreamCfg<64, 8, 2, 8, 8>>(a, num_ctas, st);
+    if (p.D == 64) {
+        switch (p.G) {
+        case 1: return launch_stream_cfg<StreamCfg<64, 1, 8, 3, 8>>(a, num_ctas, st);
+        case 2: return launch_stream_cfg<StreamCfg<64, 2, 8, 3, 8>>(a, num_ctas, st);
+        case 4: return launch_stream_cfg<StreamCfg<64, 4, 4, 2, 16>>(a, num_ctas, st);
+        default: return launch_stream_cfg<StreamCfg<64, 8, 2, 4, 16>>(a, num_ctas, st);
+        }
+    }
+    switch (p.G) {                       // D == 32: eight lanes per row, four rows per 512-byte read
+    case 1: return launch_stream_cfg<StreamCfg<32, 1, 8, 3, 8>>(a, num_ctas, st);
+    case 2: return launch_stream_cfg<StreamCfg<32, 2, 4, 3, 16>>(a, num_ctas, st);
+    case 4: return launch_stream_cfg<StreamCfg<32, 4, 2, 5, 16>>(a, num_ctas, st);
+    default: return launch_stream_cfg<StreamCfg<32, 8, 1, 8, 16>>(a, num_ctas, st);
     }
 }
 

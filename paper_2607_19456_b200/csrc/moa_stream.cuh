@@ -41,7 +41,7 @@ struct StreamCfg {
     static constexpr int PS = D + 4;          // floats per partial: o[D], m, l, 2 pad
     static constexpr int STAGE_FLOATS = 2 * R * D;
     static constexpr int THREADS = W * 32;
-    static_assert(D == 64 || D == 128, "row must be 256 or 512 bytes");
+    static_assert(D == 32 || D == 64 || D == 128, "row must be 128, 256 or 512 bytes");
     static_assert(NV >= 4 && NV <= 32 && NV <= LPR && (NV & (NV - 1)) == 0, "bad NV");
     static_assert(NV % 4 == 0, "p is fetched as float4");
     static_assert(G * LPR <= THREADS, "merge uses one thread per (head, float4)");

@@ -42,13 +42,13 @@ def test_paper_decode_shapes_d64(n):
 @pytest.mark.parametrize("hkv", [8, 4, 2, 1])
 def test_paper_gqa_shapes_d32(hkv):
     q, K, V, s = make(20 + hkv, 1, 8, hkv, 64, 32, 32)
-    assert max_err(gpu_decode(q, K, V, s), oracle.decode(q, K, V, s)) <= TOL
+    assert max_err(gpu_decode(q, K, V, s, expect_path=moa.PATH_STREAM), oracle.decode(q, K, V, s)) <= TOL
 
 
 # ---------------------------------------------------------------------------------------
 # streaming kernel: every compiled (D, G) variant, ragged tails, several tiles, splits
 # ---------------------------------------------------------------------------------------
-@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("D", [32, 64, 128])
 @pytest.mark.parametrize("gs", [1, 2, 3, 4, 5, 8, 12, 16, 64])
 def test_stream_kernel_group_sizes(D, gs):
     hkv = 2
@@ -67,6 +67,8 @@ def test_stream_kernel_every_tail_length(n):
     q, K, V, s = make(300 + n, 3, 8, 2, n, 128, 128)
     assert max_err(gpu_decode(q, K, V, s, expect_path=moa.PATH_STREAM), oracle.decode(q, K, V, s)) <= TOL
     q, K, V, s = make(400 + n, 2, 2, 2, n, 64, 64)
+    assert max_err(gpu_decode(q, K, V, s, expect_path=moa.PATH_STREAM), oracle.decode(q, K, V, s)) <= TOL
+    q, K, V, s = make(500 + n, 2, 4, 1, n, 32, 32)
     assert max_err(gpu_decode(q, K, V, s, expect_path=moa.PATH_STREAM), oracle.decode(q, K, V, s)) <= TOL
 
 
@@ -244,7 +246,7 @@ def test_append_out_of_range_position_is_skipped_and_reported():
 # multi-step decode: append then attend, token by token
 # ---------------------------------------------------------------------------------------
 @pytest.mark.parametrize("fused", [True, False])
-@pytest.mark.parametrize("D,hq,hkv", [(128, 8, 2), (64, 2, 1), (16, 4, 4)])
+@pytest.mark.parametrize("D,hq,hkv", [(128, 8, 2), (64, 2, 1), (32, 8, 1), (16, 4, 4)])
 def test_multistep_small(fused, D, hq, hkv):
     w = mi.Workload("ms", 950 + D, 4, hq, hkv, 80, D, D, steps=40, len_lo=1, len_hi=40)
     B, n_max = w.batch, w.n
@@ -280,7 +282,7 @@ def test_multistep_small(fused, D, hq, hkv):
 
 
 @pytest.mark.parametrize("ctas,misalign_new", [(0, 0), (4000, 0), (0, 1), (5, 0)])
-@pytest.mark.parametrize("D,hq,hkv", [(128, 32, 8), (64, 16, 1), (128, 6, 2)])
+@pytest.mark.parametrize("D,hq,hkv", [(128, 32, 8), (64, 16, 1), (128, 6, 2), (32, 2, 2)])
 def test_append_decode_single_call(ctas, misalign_new, D, hq, hkv):
     # one call appends at pos[b] and attends over pos[b]+1 rows; lengths are not modified.
     # ctas=4000 and a k_new that is only 4-byte aligned take the three-launch fallback.
