@@ -19,7 +19,7 @@ OK, ERR_INVALID, ERR_UNSUPPORTED, ERR_ALIGN, ERR_CAPACITY, ERR_WORKSPACE, ERR_CU
 STATUS_APPEND_RANGE, STATUS_SEQLEN_RANGE, STATUS_WAIT_TIMEOUT = 1, 2, 4
 OPT_FORCE_PATH, OPT_NUM_CTAS, OPT_GROUPED_HEADS = 1, 2, 3
 NOALLOC_SCRATCH_BYTES = 2 << 20
-PATH_AUTO, PATH_GENERIC, PATH_STREAM, PATH_GROUPED = 0, 1, 2, 3
+PATH_AUTO, PATH_GENERIC, PATH_STREAM, PATH_GROUPED, PATH_MMA = 0, 1, 2, 3, 4
 
 _lib = None
 

@@ -9,6 +9,7 @@
 #include "moa_device.cuh"
 #include "moa_generic.cuh"
 #include "moa_stream.cuh"
+#include "moa_mma.cuh"
 #include "moa_grouped.cuh"
 
 namespace moa {
@@ -98,6 +99,7 @@ struct StreamPlan {
     int G = 0;       // heads per (virtual) kv head handled by one CTA pass
     int share = 1;   // virtual kv heads per physical kv head (g_s = share * G when g_s > 8)
     int R = 0;       // rows per block of the chosen configuration
+    bool mma = false;  // groups of 8 heads: the contractions run on the warp-level MMA
 };
 
 static int stream_group(int g_s, int *share)
@@ -121,13 +123,18 @@ static int rows_per_block(int D, int G)
     return 32 / G;                       // D == 32
 }
 
+// Which of the two streaming kernels a call uses is part of the plan, because the row-block
+// size (and with it the whole decomposition) differs.  MOA_PATH_STREAM forces the FMA kernel.
+static bool mma_allowed() { return g_force_path != MOA_PATH_STREAM; }
+
 static StreamPlan plan_stream(int g_s, int d_k, int d_v)
 {
     StreamPlan p;
     if (d_k != d_v || (d_k != 32 && d_k != 64 && d_k != 128)) return p;
     p.D = d_k;
     p.G = stream_group(g_s, &p.share);
-    p.R = rows_per_block(p.D, p.G);
+    p.mma = mma_allowed() && p.G == 8 && p.D >= 64;     // (the caller drops it for huge caches)
+    p.R = p.mma ? 16 : rows_per_block(p.D, p.G);
     p.ok = true;
     return p;
 }
@@ -177,9 +184,45 @@ static cudaError_t launch_stream_cfg(const DecodeArgs &a, int num_ctas, cudaStre
     return cudaGetLastError();
 }
 
+static bool make_rows_map(CUtensorMap *m, const float *base, long long rows_total, int D);
+
+template <class C>
+static cudaError_t launch_mma_cfg(const DecodeArgs &a, int num_ctas, cudaStream_t st)
+{
+    // The caches as [d/32 column groups][rows][32 floats]: one box is a 16-row tile.
+    const long long rows_total = (long long)a.batch * (a.h_kv / a.kv_share) * a.n_max;
+    CUtensorMap mk, mv;
+    if (!make_rows_map(&mk, a.K, rows_total, C::D) || !make_rows_map(&mv, a.V, rows_total, C::D))
+        return cudaErrorInvalidValue;
+    static bool attr_set[kMaxDevices] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (!attr_set[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(mma_decode_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)C::SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        attr_set[dev] = true;
+    }
+    {
+        TimedLaunch t(st);
+        mma_decode_kernel<C><<<num_ctas, C::THREADS, C::SMEM_BYTES, st>>>(mk, mv, a);
+    }
+    count_launch();
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess || a.tickets != nullptr) return e;
+    const long long warps = (long long)a.batch * a.h_q;
+    stream_combine_kernel<C::D, C::R><<<(int)((warps + 3) / 4), 128, 0, st>>>(a, num_ctas, C::G);
+    count_launch();
+    return cudaGetLastError();
+}
+
 static cudaError_t launch_stream(const StreamPlan &p, const DecodeArgs &a, int num_ctas,
                                  cudaStream_t st)
 {
+    if (p.mma) {                         //                                     D   S  W
+        if (p.D == 128) return launch_mma_cfg<MmaCfg<128, 2, 5>>(a, num_ctas, st);
+        return launch_mma_cfg<MmaCfg<64, 2, 8>>(a, num_ctas, st);
+    }
     // The heavier configurations (many FMAs per fetched byte) run 16 warps per CTA: with
     // eight, two warps per scheduler cannot hide the shuffle and FMA latencies.
     //                                   D    G  RV  S  W
@@ -276,6 +319,21 @@ static bool make_cache_map(CUtensorMap *m, const float *base, long long units, i
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Tensor map over a cache seen as rows of D floats: dimensions (32 floats, rows, D/32 column
+// groups), so that one box of 16 rows lands as D/32 swizzled [16 rows][128 bytes] sub-tiles.
+static bool make_rows_map(CUtensorMap *m, const float *base, long long rows_total, int D)
+{
+    TmapEncodeFn enc = tmap_encoder();
+    if (!enc) return false;
+    cuuint64_t dims[3] = {32, (cuuint64_t)rows_total, (cuuint64_t)(D / 32)};
+    cuuint64_t strides[2] = {(cuuint64_t)D * 4, 128};
+    cuuint32_t box[3] = {32, 16, (cuuint32_t)(D / 32)};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int GH>
 static cudaError_t launch_grouped_cfg(const CUtensorMap &mk, const CUtensorMap &mv, const GroupedArgs &ga,
                                       int grid, cudaStream_t st)
@@ -348,8 +406,12 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
 
     const int g_s = h_q / h_kv;
     StreamPlan plan = plan_stream(g_s, d_k, d_v);
+    if (plan.mma && (long long)batch * h_kv * n_max > 0x7fffff00LL) {   // row coordinates are 32-bit
+        plan.mma = false;
+        plan.R = rows_per_block(plan.D, plan.G);
+    }
     const bool fast_ok = plan.ok && aligned(q, 16) && aligned(K, 16) && aligned(V, 16) && aligned(out, 16);
-    int path = fast_ok ? MOA_PATH_STREAM : MOA_PATH_GENERIC;
+    int path = fast_ok ? (plan.mma ? MOA_PATH_MMA : MOA_PATH_STREAM) : MOA_PATH_GENERIC;
     // Large head groups over a dense cache go to the tensor cores.
     GroupedPlan gplan;
     if (fast_ok && allow_grouped && fused == nullptr && seq_lens == nullptr)
@@ -359,6 +421,9 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
     else if (g_force_path == MOA_PATH_STREAM) {
         if (!fast_ok) return MOA_ERR_UNSUPPORTED;
         path = MOA_PATH_STREAM;
+    } else if (g_force_path == MOA_PATH_MMA) {
+        if (!fast_ok || !plan.mma) return MOA_ERR_UNSUPPORTED;
+        path = MOA_PATH_MMA;
     } else if (g_force_path == MOA_PATH_GROUPED) {
         if (path != MOA_PATH_GROUPED) return MOA_ERR_UNSUPPORTED;
     } else if (g_force_path != 0) return MOA_ERR_UNSUPPORTED;
@@ -371,7 +436,7 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
     a.qscale = scale * kLog2e;
     a.Kw = nullptr; a.Vw = nullptr; a.k_new = nullptr; a.v_new = nullptr; a.lens_rw = nullptr;
     a.tickets = nullptr;
-    if (fused != nullptr && path != MOA_PATH_STREAM) return MOA_ERR_UNSUPPORTED;
+    if (fused != nullptr && path != MOA_PATH_STREAM && path != MOA_PATH_MMA) return MOA_ERR_UNSUPPORTED;
 
     cudaError_t e;
     if (path == MOA_PATH_GROUPED) {
@@ -398,7 +463,7 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
         if (gplan.GH == 16) e = launch_grouped_cfg<16>(mk, mv, ga, grid, st);
         else if (gplan.GH == 32) e = launch_grouped_cfg<32>(mk, mv, ga, grid, st);
         else e = launch_grouped_cfg<64>(mk, mv, ga, grid, st);
-    } else if (path == MOA_PATH_STREAM) {
+    } else if (path == MOA_PATH_STREAM || path == MOA_PATH_MMA) {
         const int num_ctas = stream_grid(*dev, plan, batch, h_kv, n_max);
         const size_t need = stream_ws_bytes(plan, num_ctas);
         if (library_ws) {
@@ -572,7 +637,7 @@ static int step_impl(const float *q, float *K, float *V, const float *k_new, con
     const StreamPlan plan = plan_stream(h_q / h_kv, d_k, d_v);
     const bool fast_ok = plan.ok && aligned(q, 16) && aligned(K, 16) && aligned(V, 16) && aligned(out, 16);
     const bool stream_path = fast_ok && g_force_path != MOA_PATH_GENERIC;
-    if (g_force_path == MOA_PATH_STREAM && !fast_ok) return MOA_ERR_UNSUPPORTED;
+    if ((g_force_path == MOA_PATH_STREAM || g_force_path == MOA_PATH_MMA) && !fast_ok) return MOA_ERR_UNSUPPORTED;
     if (stream_path) {          // validate the scratch before anything is written
         if (!workspace || workspace_bytes < stream_ws_bytes(plan, stream_num_ctas(*dev))) return MOA_ERR_WORKSPACE;
         if (!aligned(workspace, 256)) return MOA_ERR_ALIGN;
@@ -715,7 +780,7 @@ const char *moa_strerror(int code)
 int moa_set_option(int option, int value)
 {
     if (option == MOA_OPT_FORCE_PATH) {
-        if (value < 0 || value > MOA_PATH_GROUPED) return MOA_ERR_INVALID;
+        if (value < 0 || value > MOA_PATH_MMA) return MOA_ERR_INVALID;
         g_force_path = value;
         return MOA_OK;
     }

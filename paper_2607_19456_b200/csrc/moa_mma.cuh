@@ -1,0 +1,495 @@
+// moa_mma.cuh -- split-sequence streaming decode kernel for groups of 8 (or 16) query
+// heads per K/V head, with the two contractions on the warp-level tensor-core MMA.
+//
+// Steps I-III of Algorithm 1 (eqs. (1)-(3)) in online-softmax form with the psi-selection
+// of section 6.1, as in the FMA streaming kernel, and with the same decomposition: the
+// cached rows of every (batch, kv head) unit are cut into 16-row tiles, all tiles form one
+// flat list dealt to persistent CTAs in equal contiguous ranges, every warp owns a private
+// ring of shared-memory stages filled by bulk asynchronous copies, split units are merged
+// by the CTA that delivers the last partial.  What differs is the arithmetic of a tile.
+// With 8 query heads per fetched row the FMA kernel is bound by instruction issue, not by
+// HBM; here a warp computes
+//     S^T [16 rows x 8 heads]   = K_tile [16 x d]  * Q^T [d x 8]        (m16n8k8, TF32)
+//     O^T [d features x 8 heads] += V_tile^T [d x 16] * P^T [16 x 8]
+// Every product is formed three times (hi*hi + lo*hi + hi*lo, where hi is the value cut to
+// TF32 and lo the remainder), which restores fp32-grade accuracy.  The split happens in
+// registers, on the fragments a thread has just loaded, so a K/V element crosses shared
+// memory once (tensor-core instructions that take their operands from shared memory
+// would need the lo parts written back, several times the traffic).  Accumulator chains
+// are kept short (a tile's products start from zero and are added to fp32 running
+// values with ordinary FMAs), because the tensor core's accumulation is not rounded to
+// nearest.
+//
+// Fragment bookkeeping.  The contraction index of an MMA and the order of rows and
+// features may be permuted freely as long as both operands agree, which is used to load
+// every fragment with 128-bit shared-memory reads: lane (g = lane/4, t = lane%4) reads,
+// of a K row, the float4 chunks t, t+4, t+8, ... (each chunk feeds two k-steps) and, of V
+// rows 2t, 2t+1, 2t+8, 2t+9, the chunks g, g+8, g+16, g+24 (each chunk feeds two 16-feature
+// output tiles).  A tile is fetched by one tiled bulk-tensor copy per operand (an SM retires
+// only about one bulk copy per 70 cycles whatever its size, so copies are kept large): the
+// cache is described as [d/32 column groups][rows][32 floats] with the 128-byte swizzle,
+// so a tile lands as d/32 sub-tiles of [16 rows][128 bytes] whose 16-byte chunks are
+// XOR-ed with the row number, and with the row <-> fragment-slot assignment used below
+// both read patterns are free of bank conflicts.
+#pragma once
+
+#include <cuda.h>
+
+#include "moa_device.cuh"
+#include "moa_tc.cuh"
+
+namespace moa {
+
+template <int D_, int S_, int W_>
+struct MmaCfg {
+    static constexpr int D = D_;              // d_k == d_v
+    static constexpr int G = 8;               // query heads per (virtual) kv head
+    static constexpr int S = S_;              // ring stages per warp
+    static constexpr int W = W_;              // warps per CTA
+    static constexpr int R = 16;              // rows per tile
+    static constexpr int LPR = D / 4;         // float4 per row
+    static constexpr int NJ = D / 16;         // K chunks a lane reads per row (2 k-steps each)
+    static constexpr int NU = D / 32;         // V chunks a lane reads per row (2 feature tiles each)
+    static constexpr int MT = D / 16;         // 16-feature output tiles
+    static constexpr int CG = D / 32;         // 128-byte column groups of a row
+    static constexpr int SUBT = R * 32;       // floats of one [16 rows][32 floats] sub-tile
+    static constexpr int OFF_V = R * D;       // stage: K tile, V tile, new K row, new V row
+    static constexpr int OFF_NEW = 2 * R * D;
+    static constexpr int STAGE_FLOATS = ((2 * R * D + 2 * D) * 4 + 1023) / 1024 * 256;   // whole KB
+    static constexpr int PT_STRIDE = 20;      // floats between heads in the P^T staging buffer
+    static constexpr int PS = D + 4;          // floats per partial: o[D], m, l, 2 pad
+    static constexpr int THREADS = W * 32;
+    static_assert(D == 64 || D == 128, "row must be 256 or 512 bytes");
+
+    static_assert((STAGE_FLOATS * 4) % 1024 == 0, "swizzled sub-tiles need 1024-byte alignment");
+    static constexpr size_t OFF_RING = 0;             // from the 1024-byte aligned base
+    static constexpr size_t OFF_MERGE_O = OFF_RING + sizeof(float) * W * S * STAGE_FLOATS;
+    static constexpr size_t OFF_MERGE_ML = OFF_MERGE_O + sizeof(float) * W * G * D;
+    static constexpr size_t OFF_PT = OFF_MERGE_ML + sizeof(float) * W * G * 2;
+    static constexpr size_t OFF_BAR = (OFF_PT + sizeof(float) * W * G * PT_STRIDE + 15) / 16 * 16;
+    static constexpr size_t SMEM_BYTES = OFF_BAR + sizeof(uint64_t) * W * S + 1024;   // + alignment slack
+};
+
+__device__ __forceinline__ void mma_tf32_16x8x8(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                                uint32_t b0, uint32_t b1)
+{
+    asm("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "{%0, %1, %2, %3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// x = hi + lo with hi exactly representable in TF32 (10 mantissa bits kept).
+struct Split4 {
+    uint32_t h[4], l[4];
+};
+__device__ __forceinline__ Split4 split4(const float4 &v)
+{
+    Split4 s;
+    const float x[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint32_t hb = __float_as_uint(x[i]) & 0xFFFFE000u;
+        s.h[i] = hb;
+        s.l[i] = __float_as_uint(x[i] - __uint_as_float(hb));
+    }
+    return s;
+}
+
+// D += A * B with both operands split; the two small terms go to accumulators of their own
+// (three independent chains, so that consecutive MMAs never wait for one another).
+__device__ __forceinline__ void mma3(float (&acc_hh)[4], float (&acc_lh)[4], float (&acc_hl)[4],
+                                     const uint32_t (&ah)[4], const uint32_t (&al)[4], uint32_t bh0, uint32_t bh1,
+                                     uint32_t bl0, uint32_t bl1)
+{
+    mma_tf32_16x8x8(acc_hh, ah[0], ah[1], ah[2], ah[3], bh0, bh1);
+    mma_tf32_16x8x8(acc_lh, al[0], al[1], al[2], al[3], bh0, bh1);
+    mma_tf32_16x8x8(acc_hl, ah[0], ah[1], ah[2], ah[3], bl0, bl1);
+}
+
+template <class C>
+__global__ void __launch_bounds__(C::THREADS, 1)
+mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant__ CUtensorMap tmapV, const DecodeArgs a)
+{
+    constexpr int D = C::D, G = C::G, S = C::S, W = C::W, R = C::R, LPR = C::LPR, NJ = C::NJ, NU = C::NU,
+                  MT = C::MT, SUBT = C::SUBT, PS = C::PS, PTS = C::PT_STRIDE;
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    unsigned char *const smem_m = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    float *ring = reinterpret_cast<float *>(smem_m + C::OFF_RING);
+    float *merge_o = reinterpret_cast<float *>(smem_m + C::OFF_MERGE_O);
+    float *merge_ml = reinterpret_cast<float *>(smem_m + C::OFF_MERGE_ML);
+    float *pt_all = reinterpret_cast<float *>(smem_m + C::OFF_PT);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_m + C::OFF_BAR);
+    __shared__ int s_last;
+    __shared__ int s_pref[kPrefixBatch + 1];
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int g = lane >> 2, t = lane & 3;
+    // MMA row index m (0..7) <-> tile row: the two rows read in one shared-memory phase (g even
+    // and odd) lie four rows apart, which the swizzle turns into disjoint halves of the banks.
+    const int rowA = (g >> 1) + 4 * (g & 1), rowB = rowA + 8;
+    const int h_stored = a.h_kv / a.kv_share;
+
+    if (tid < W * S) mbar_init(smem_u32(&bars[tid]), 1);
+    if (tid == 0) { tc::prefetch_tmap(&tmapK); tc::prefetch_tmap(&tmapV); }
+    mbar_fence_init();
+    __syncthreads();
+
+    const int *pref = nullptr;
+    if (a.seq_lens != nullptr && a.batch <= kPrefixBatch) {
+        if (warp == 0) build_block_prefix<R>(a, s_pref, lane);
+        __syncthreads();
+        pref = s_pref;
+    }
+    const long long total = pref ? (long long)pref[a.batch] * a.h_kv : total_blocks<R>(a, lane);
+    const long long bpc = (total + gridDim.x - 1) / gridDim.x;
+    const long long c0 = (long long)blockIdx.x * bpc;
+    const long long c1 = (c0 + bpc < total) ? c0 + bpc : total;
+
+    if (c0 < c1) {                            // uniform for the whole CTA
+    float *my_ring = ring + (size_t)warp * S * C::STAGE_FLOATS;
+    const uint32_t my_bar0 = smem_u32(&bars[warp * S]);
+    float *my_pt = pt_all + (size_t)warp * G * PTS;
+
+    // ---- load side: this warp's tiles are c0+warp, c0+warp+W, ... ------------------------
+    long long jl = c0 + warp;
+    int kl = 0;
+    Cursor lc = cursor_at<R>(a, (jl < c1) ? jl : c0, pref);
+    size_t slab = 0;                           // stored (batch, kv head) of the unit under lc
+    bool writes_new = false;                   // this virtual head stores the appended row
+    auto load_unit_changed = [&]() {
+        const int hs = lc.h / a.kv_share;
+        slab = (size_t)lc.b * h_stored + hs;
+        writes_new = (a.k_new != nullptr) && (lc.h == hs * a.kv_share);
+    };
+    load_unit_changed();
+    auto issue_next_load = [&]() {
+        if (jl >= lc.first + lc.ub) {
+            do cursor_next_unit<R>(a, lc); while (jl >= lc.first + lc.ub);
+            load_unit_changed();
+        }
+        const int row0 = (int)(jl - lc.first) * R;
+        const int nr = (lc.len - row0 < R) ? lc.len - row0 : R;
+        // Fused append: the unit's last row is the token being appended; it comes from
+        // k_new / v_new (it lands beside the tile and replaces the tile's last row before use)
+        // and this warp also stores it into the cache.
+        const bool has_new = (a.k_new != nullptr) && (row0 + nr == lc.len);
+        const int nr_cache = has_new ? nr - 1 : nr;
+        const size_t row = slab * (size_t)a.n_max + row0;
+        if (lane == 0) {
+            const int stage = kl % S;
+            const uint32_t bar = my_bar0 + 8u * stage;
+            const uint32_t dst = smem_u32(my_ring + (size_t)stage * C::STAGE_FLOATS);
+            // A box is always transferred whole (rows past the end of the cache read as zero;
+            // rows past the end of the unit belong to the next unit and are masked later).
+            mbar_expect_tx(bar, (2u * R + (has_new ? 2u : 0u)) * D * 4u);
+            tc::tma_load_3d(dst, &tmapK, 0, (int)row, 0, bar);
+            tc::tma_load_3d(dst + C::OFF_V * 4u, &tmapV, 0, (int)row, 0, bar);
+            if (has_new) {
+                bulk_g2s(dst + C::OFF_NEW * 4u, a.k_new + slab * D, D * 4u, bar);
+                bulk_g2s(dst + (C::OFF_NEW + D) * 4u, a.v_new + slab * D, D * 4u, bar);
+            }
+        }
+        if (has_new && writes_new && lane < LPR) {
+            const size_t dst_row = (row + (size_t)nr_cache) * D + lane * 4;
+            *reinterpret_cast<float4 *>(a.Kw + dst_row) =
+                *reinterpret_cast<const float4 *>(a.k_new + slab * D + lane * 4);
+            *reinterpret_cast<float4 *>(a.Vw + dst_row) =
+                *reinterpret_cast<const float4 *>(a.v_new + slab * D + lane * 4);
+        }
+        jl += W;
+        ++kl;
+    };
+#pragma unroll 1
+    for (int i = 0; i < S && jl < c1; ++i) issue_next_load();
+
+    // ---- compute side ------------------------------------------------------------------
+    Cursor cc = cursor_at<R>(a, c0, pref);
+    // Q^T fragments of head g: chunk t+4j of the scaled query row, split.  Running state of
+    // heads 2t and 2t+1: maximum, this thread's share of the sum, and the O^T fragments.
+    uint32_t qh[NJ][4], ql[NJ][4];
+    float om[MT][4];
+    float m_run[2], l_run[2];
+    auto begin_unit = [&]() {
+        const float *qb = a.q + ((size_t)cc.b * a.h_q + (size_t)cc.h * a.g_s) * D;
+#pragma unroll
+        for (int j = 0; j < NJ; ++j) {
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (g < a.g_s) v = *reinterpret_cast<const float4 *>(qb + (size_t)g * D + (t + 4 * j) * 4);
+            const Split4 s = split4(make_float4(v.x * a.qscale, v.y * a.qscale, v.z * a.qscale, v.w * a.qscale));
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { qh[j][i] = s.h[i]; ql[j][i] = s.l[i]; }
+        }
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) om[mt][i] = 0.f;
+        m_run[0] = m_run[1] = -INFINITY;
+        l_run[0] = l_run[1] = 0.f;
+    };
+
+    // Merge the W running states of this CTA for the unit under `cc` and emit either the
+    // final output rows or this CTA's partial triple; with completion counters in use, the
+    // CTA that delivers the last partial of a split unit also merges that unit's partials.
+    auto finish_unit = [&]() {
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            float l = l_run[i];
+            l += __shfl_xor_sync(0xffffffffu, l, 4);
+            l += __shfl_xor_sync(0xffffffffu, l, 8);
+            l += __shfl_xor_sync(0xffffffffu, l, 16);
+            if (g == 0) {
+                merge_ml[(warp * G + 2 * t + i) * 2 + 0] = m_run[i];
+                merge_ml[(warp * G + 2 * t + i) * 2 + 1] = l;
+            }
+        }
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+            // output tile mt = 2u+e holds features 32u + 4g + 2e (+1) of heads 2t (+1)
+            const int f = 32 * (mt >> 1) + 4 * g + 2 * (mt & 1);
+            float *o0 = merge_o + ((size_t)(warp * G + 2 * t)) * D + f;
+            o0[0] = om[mt][0]; o0[D] = om[mt][1]; o0[1] = om[mt][2]; o0[D + 1] = om[mt][3];
+        }
+        __syncthreads();
+        const long long seg_begin = (c0 > cc.first) ? c0 : cc.first;
+        const long long unit_end = cc.first + cc.ub;
+        const long long seg_end = (c1 < unit_end) ? c1 : unit_end;
+        const bool complete = (seg_begin == cc.first) && (seg_end == unit_end);
+        for (int idx = tid; idx < G * LPR; idx += C::THREADS) {
+            const int hg = idx / LPR, d4 = idx % LPR;
+            float M = -INFINITY;
+#pragma unroll
+            for (int v = 0; v < W; ++v) M = fmaxf(M, merge_ml[(v * G + hg) * 2]);
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            float L = 0.f;
+#pragma unroll
+            for (int v = 0; v < W; ++v) {
+                const float f = exp2_diff(merge_ml[(v * G + hg) * 2], M);
+                const float4 x = *reinterpret_cast<const float4 *>(merge_o + ((size_t)(v * G + hg)) * D + d4 * 4);
+                acc.x = fmaf(x.x, f, acc.x); acc.y = fmaf(x.y, f, acc.y);
+                acc.z = fmaf(x.z, f, acc.z); acc.w = fmaf(x.w, f, acc.w);
+                L = fmaf(merge_ml[(v * G + hg) * 2 + 1], f, L);
+            }
+            if (complete) {
+                if (hg < a.g_s) {
+                    const float inv = 1.0f / L;
+                    float *dst = a.out + ((size_t)cc.b * a.h_q + (size_t)cc.h * a.g_s + hg) * D + d4 * 4;
+                    *reinterpret_cast<float4 *>(dst) = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+                }
+            } else {
+                const int slot = (seg_begin == c0) ? 0 : 1;
+                float *dst = a.ws + (((size_t)blockIdx.x * 2 + slot) * G + hg) * PS;
+                *reinterpret_cast<float4 *>(dst + d4 * 4) = acc;
+                if (d4 == 0) { dst[D] = M; dst[D + 1] = L; }
+            }
+        }
+        __syncthreads();
+        if (!complete && a.tickets != nullptr) {
+            const long long c_first = cc.first / bpc, c_last = (unit_end - 1) / bpc;
+            if (tid == 0) {
+                __threadfence();               // this CTA's partial is visible before it is counted
+                const unsigned arrived = atomicAdd(&a.tickets[c_first], 1u);
+                const int last = (arrived == (unsigned)(c_last - c_first));
+                if (last) a.tickets[c_first] = 0u;
+                s_last = last;
+            }
+            __syncthreads();
+            if (s_last) {                          // uniform for the CTA
+                __threadfence();
+                const int ns = (int)(c_last - c_first) + 1;
+                float *stage = merge_o;            // [ns][G][2]; merge_o is idle here
+                for (int i = tid; i < ns * G; i += C::THREADS) {
+                    const long long c = c_first + i / G;
+                    const int hg = i % G;
+                    const int slot = (cc.first <= c * bpc) ? 0 : 1;
+                    const float *p = a.ws + (((size_t)c * 2 + slot) * G + hg) * PS;
+                    stage[2 * i] = __ldcg(p + D);
+                    stage[2 * i + 1] = __ldcg(p + D + 1);
+                }
+                __syncthreads();
+                for (int idx = tid; idx < G * LPR; idx += C::THREADS) {
+                    const int hg = idx / LPR, d4 = idx % LPR;
+                    float M = -INFINITY;
+                    for (int i = 0; i < ns; ++i) M = fmaxf(M, stage[(i * G + hg) * 2]);
+                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                    float L = 0.f;
+#pragma unroll 8
+                    for (int i = 0; i < ns; ++i) {      // partials in CTA order; the loads are independent
+                        const long long c = c_first + i;
+                        const int slot = (cc.first <= c * bpc) ? 0 : 1;
+                        const float *p = a.ws + (((size_t)c * 2 + slot) * G + hg) * PS;
+                        const float f = exp2_diff(stage[(i * G + hg) * 2], M);
+                        L = fmaf(stage[(i * G + hg) * 2 + 1], f, L);
+                        const float4 x = __ldcg(reinterpret_cast<const float4 *>(p + d4 * 4));
+                        acc.x = fmaf(x.x, f, acc.x); acc.y = fmaf(x.y, f, acc.y);
+                        acc.z = fmaf(x.z, f, acc.z); acc.w = fmaf(x.w, f, acc.w);
+                    }
+                    if (hg < a.g_s) {
+                        const float inv = 1.0f / L;
+                        float *dst = a.out + ((size_t)cc.b * a.h_q + (size_t)cc.h * a.g_s + hg) * D + d4 * 4;
+                        *reinterpret_cast<float4 *>(dst) = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+                    }
+                }
+                __syncthreads();                   // merge_o is written again by the next unit
+            }
+        }
+    };
+
+    // float offset, inside a tile, of 16-byte chunk `ch` of row r
+    auto chunk_at = [](int r, int ch) { return (ch >> 3) * SUBT + r * 32 + (((ch & 7) ^ (r & 7)) << 2); };
+    auto process_tile = [&](float *stage_base, int nr, bool has_new, auto full_tag) {
+        constexpr bool FULL = decltype(full_tag)::value;
+        float *sK = stage_base, *sV = stage_base + C::OFF_V;
+        if (has_new) {                             // the appended token is the tile's last row
+            if (lane < LPR) {
+                const float4 kn = *reinterpret_cast<const float4 *>(stage_base + C::OFF_NEW + lane * 4);
+                const float4 vn = *reinterpret_cast<const float4 *>(stage_base + C::OFF_NEW + D + lane * 4);
+                *reinterpret_cast<float4 *>(sK + chunk_at(nr - 1, lane)) = kn;
+                *reinterpret_cast<float4 *>(sV + chunk_at(nr - 1, lane)) = vn;
+            }
+            __syncwarp();
+        }
+        // ---- S^T = K_tile * Q^T: 2*NJ k-steps, two accumulator chains each for hi and lo
+        float sh[2][4], sl[2][4], sm[2][4];
+#pragma unroll
+        for (int c = 0; c < 2; ++c)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { sh[c][i] = 0.f; sl[c][i] = 0.f; sm[c][i] = 0.f; }
+#pragma unroll
+        for (int j = 0; j < NJ; ++j) {
+            const Split4 ka = split4(*reinterpret_cast<const float4 *>(sK + chunk_at(rowA, t + 4 * j)));
+            const Split4 kb = split4(*reinterpret_cast<const float4 *>(sK + chunk_at(rowB, t + 4 * j)));
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {          // elements (2e, 2e+1) of the chunk are k-slots (t, t+4)
+                const uint32_t ah[4] = {ka.h[2 * e], kb.h[2 * e], ka.h[2 * e + 1], kb.h[2 * e + 1]};
+                const uint32_t al[4] = {ka.l[2 * e], kb.l[2 * e], ka.l[2 * e + 1], kb.l[2 * e + 1]};
+                mma3(sh[e], sl[e], sm[e], ah, al, qh[j][2 * e], qh[j][2 * e + 1], ql[j][2 * e], ql[j][2 * e + 1]);
+            }
+        }
+        // this thread's scores: rows rowA (0,1) and rowB (2,3) of heads 2t (0,2) and 2t+1 (1,3)
+        float s[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) s[i] = (sh[0][i] + sh[1][i]) + ((sl[0][i] + sl[1][i]) + (sm[0][i] + sm[1][i]));
+        if (!FULL) {
+            if (rowA >= nr) { s[0] = -INFINITY; s[1] = -INFINITY; }
+            if (rowB >= nr) { s[2] = -INFINITY; s[3] = -INFINITY; }
+        }
+        // ---- online softmax per head (row maximum across the 8 lanes with the same t)
+        float alpha[2], p[4];
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            float bm = fmaxf(s[i], s[i + 2]);
+            bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 4));
+            bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 8));
+            bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 16));
+            const float m_new = fmaxf(m_run[i], bm);
+            alpha[i] = exp2_diff(m_run[i], m_new);
+            p[i] = exp2_diff(s[i], m_new);
+            p[i + 2] = exp2_diff(s[i + 2], m_new);
+            l_run[i] = fmaf(l_run[i], alpha[i], p[i] + p[i + 2]);
+            m_run[i] = m_new;
+        }
+        // ---- P^T through shared memory: lane (g, t) fetches rows 2t, 2t+1, 2t+8, 2t+9 of head g
+        // (the rows whose V it loads) with one 128-bit read
+        {
+            const int pa = 4 * ((rowA >> 1) & 3) + (rowA & 1), pb = pa + 2;
+            my_pt[(2 * t) * PTS + pa] = p[0];
+            my_pt[(2 * t + 1) * PTS + pa] = p[1];
+            my_pt[(2 * t) * PTS + pb] = p[2];
+            my_pt[(2 * t + 1) * PTS + pb] = p[3];
+        }
+        __syncwarp();
+        const Split4 pp = split4(*reinterpret_cast<const float4 *>(my_pt + g * PTS + 4 * t));
+        __syncwarp();                              // the buffer may be rewritten by the next tile
+        // ---- O^T += V_tile^T * P^T, tile by tile of 16 features; each tile's products start from
+        // zero and are then added to the running values, rescaled by alpha
+#pragma unroll
+        for (int u = 0; u < NU; ++u) {
+            Split4 v[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int r = 2 * t + (i & 1) + 8 * (i >> 1);
+                float4 x = *reinterpret_cast<const float4 *>(sV + chunk_at(r, g + 8 * u));
+                if (!FULL && r >= nr) x = make_float4(0.f, 0.f, 0.f, 0.f);
+                v[i] = split4(x);
+            }
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                float oh[4] = {0.f, 0.f, 0.f, 0.f}, ol[4] = {0.f, 0.f, 0.f, 0.f}, ox[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int kp = 0; kp < 2; ++kp) {   // rows (2t+8kp, 2t+1+8kp) are k-slots (t, t+4)
+                    const uint32_t ah[4] = {v[2 * kp].h[2 * e], v[2 * kp].h[2 * e + 1], v[2 * kp + 1].h[2 * e],
+                                            v[2 * kp + 1].h[2 * e + 1]};
+                    const uint32_t al[4] = {v[2 * kp].l[2 * e], v[2 * kp].l[2 * e + 1], v[2 * kp + 1].l[2 * e],
+                                            v[2 * kp + 1].l[2 * e + 1]};
+                    mma3(oh, ol, ox, ah, al, pp.h[2 * kp], pp.h[2 * kp + 1], pp.l[2 * kp], pp.l[2 * kp + 1]);
+                }
+                const int mt = 2 * u + e;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) om[mt][i] = fmaf(om[mt][i], alpha[i & 1], oh[i] + (ol[i] + ox[i]));
+            }
+        }
+    };
+
+    begin_unit();
+    bool failed = false;
+    int k = 0;
+#pragma unroll 1
+    for (long long j = c0 + warp; j < c1; j += W, ++k) {
+        while (j >= cc.first + cc.ub) {
+            finish_unit();
+            cursor_next_unit<R>(a, cc);
+            begin_unit();
+        }
+        const int stage = k % S;
+        if (!failed && !mbar_test_wait(my_bar0 + 8u * stage, (uint32_t)(k / S) & 1u) &&
+            !mbar_wait_bounded(my_bar0 + 8u * stage, (uint32_t)(k / S) & 1u)) {
+            failed = true;
+            if (lane == 0) raise_status(MOA_STATUS_WAIT_TIMEOUT);
+        }
+        if (!failed) {
+            const int row0 = (int)(j - cc.first) * R;
+            const int nr = (cc.len - row0 < R) ? cc.len - row0 : R;
+            float *stage_base = my_ring + (size_t)stage * C::STAGE_FLOATS;
+            const bool has_new = (a.k_new != nullptr) && (row0 + nr == cc.len);
+            if (nr == R) process_tile(stage_base, nr, has_new, std::true_type{});
+            else process_tile(stage_base, nr, has_new, std::false_type{});
+            if (has_new) tc::fence_async_smem();   // plain stores to the stage precede the next bulk copy
+        }
+        __syncwarp();                          // all lanes are done with this stage
+        if (!failed && jl < c1) issue_next_load();
+    }
+    while (cc.first + cc.ub < c1) {            // units after this warp's last tile
+        finish_unit();
+        cursor_next_unit<R>(a, cc);
+        begin_unit();
+    }
+    finish_unit();
+    }  // c0 < c1
+
+    // ---- whole-grid completion: range report and length advance by the last CTA ---------
+    if (a.tickets != nullptr) {
+        __syncthreads();
+        if (tid == 0) {
+            __threadfence();
+            const unsigned done = atomicAdd(&a.tickets[kTicketCtas], 1u);
+            const int last = (done == gridDim.x - 1);
+            if (last) a.tickets[kTicketCtas] = 0u;
+            s_last = last;
+        }
+        __syncthreads();
+        if (s_last && a.seq_lens != nullptr) {   // every CTA has finished reading the lengths
+            for (int b = tid; b < a.batch; b += blockDim.x) {
+                const int raw = a.seq_lens[b];
+                const int len = raw + a.len_bias;
+                if (len < 1 || len > a.n_max) {
+                    raise_status(MOA_STATUS_SEQLEN_RANGE | (a.k_new != nullptr ? MOA_STATUS_APPEND_RANGE : 0));
+                } else if (a.lens_rw != nullptr) {
+                    a.lens_rw[b] = raw + 1;
+                }
+            }
+        }
+    }
+}
+
+}  // namespace moa

@@ -48,18 +48,35 @@ def test_paper_gqa_shapes_d32(hkv):
 # ---------------------------------------------------------------------------------------
 # streaming kernel: every compiled (D, G) variant, ragged tails, several tiles, splits
 # ---------------------------------------------------------------------------------------
+def automatic_path(D, gs):
+    """The kernel family the library picks for a dense, aligned call."""
+    if D == 128 and gs in (16, 32, 64):
+        return moa.PATH_GROUPED
+    if gs <= 8:
+        G = 1
+        while G < gs:
+            G *= 2
+    else:
+        G = 8
+        while gs % G:
+            G //= 2
+    return moa.PATH_MMA if (G == 8 and D >= 64) else moa.PATH_STREAM
+
+
 @pytest.mark.parametrize("D", [32, 64, 128])
-@pytest.mark.parametrize("gs", [1, 2, 3, 4, 5, 8, 12, 16, 64])
+@pytest.mark.parametrize("gs", [1, 2, 3, 4, 5, 8, 12, 16, 24, 64])
 def test_stream_kernel_group_sizes(D, gs):
     hkv = 2
     for n in (1, 7, 130, 1037):
         q, K, V, s = make(1000 * D + 10 * gs + n, 2, gs * hkv, hkv, n, D, D)
-        want = moa.PATH_GROUPED if (D == 128 and gs in (16, 32, 64)) else moa.PATH_STREAM
+        want = automatic_path(D, gs)
         out = gpu_decode(q, K, V, s, expect_path=want)
         ref = oracle.decode(q, K, V, s)
         assert max_err(out, ref) <= TOL, (D, gs, n)
-        if want == moa.PATH_GROUPED:         # the same shape through the FFMA kernel
-            assert max_err(gpu_decode(q, K, V, s, path=moa.PATH_STREAM), ref) <= TOL, (D, gs, n)
+        if want != moa.PATH_STREAM:          # the same shape through the other streaming kernels
+            assert max_err(gpu_decode(q, K, V, s, path=moa.PATH_STREAM, expect_path=moa.PATH_STREAM), ref) <= TOL
+        if want == moa.PATH_GROUPED:
+            assert max_err(gpu_decode(q, K, V, s, path=moa.PATH_MMA, expect_path=moa.PATH_MMA), ref) <= TOL
 
 
 @pytest.mark.parametrize("n", [1, 2, 3, 4, 5, 8, 9, 15, 16, 17, 31, 32, 33, 63, 64, 65, 127, 129, 1000, 5003])
@@ -70,6 +87,10 @@ def test_stream_kernel_every_tail_length(n):
     assert max_err(gpu_decode(q, K, V, s, expect_path=moa.PATH_STREAM), oracle.decode(q, K, V, s)) <= TOL
     q, K, V, s = make(500 + n, 2, 4, 1, n, 32, 32)
     assert max_err(gpu_decode(q, K, V, s, expect_path=moa.PATH_STREAM), oracle.decode(q, K, V, s)) <= TOL
+    q, K, V, s = make(600 + n, 2, 16, 2, n, 128, 128)
+    assert max_err(gpu_decode(q, K, V, s, expect_path=moa.PATH_MMA), oracle.decode(q, K, V, s)) <= TOL
+    q, K, V, s = make(700 + n, 1, 7, 1, n, 64, 64)
+    assert max_err(gpu_decode(q, K, V, s, expect_path=moa.PATH_MMA), oracle.decode(q, K, V, s)) <= TOL
 
 
 @pytest.mark.parametrize("ctas", [1, 2, 3, 7, 37, 148, 500, 4000])
@@ -78,6 +99,9 @@ def test_stream_kernel_any_cta_count_gives_the_same_answer(ctas):
     q, K, V, s = make(77, 3, 8, 2, 2500, 128, 128)
     ref = oracle.decode(q, K, V, s)
     assert max_err(gpu_decode(q, K, V, s, num_ctas=ctas, expect_path=moa.PATH_STREAM), ref) <= TOL
+    q, K, V, s = make(78, 3, 16, 2, 2500, 128, 128)
+    ref = oracle.decode(q, K, V, s)
+    assert max_err(gpu_decode(q, K, V, s, num_ctas=ctas, expect_path=moa.PATH_MMA), ref) <= TOL
 
 
 # ---------------------------------------------------------------------------------------
@@ -124,6 +148,10 @@ def test_results_are_deterministic():
     a = gpu_decode(q, K, V, s)
     b = gpu_decode(q, K, V, s)
     assert np.array_equal(a.view(np.uint32), b.view(np.uint32))
+    q, K, V, s = make(79, 2, 32, 4, 3000, 128, 128)
+    a = gpu_decode(q, K, V, s, expect_path=moa.PATH_MMA)
+    b = gpu_decode(q, K, V, s, expect_path=moa.PATH_MMA)
+    assert np.array_equal(a.view(np.uint32), b.view(np.uint32))
 
 
 def test_large_scores_and_uniform_values():
@@ -167,7 +195,7 @@ def test_unaligned_pointers_take_the_generic_kernel():
 # ---------------------------------------------------------------------------------------
 # ragged lengths over a pre-allocated cache
 # ---------------------------------------------------------------------------------------
-@pytest.mark.parametrize("D,hq,hkv", [(128, 8, 2), (64, 4, 4), (128, 16, 1), (32, 4, 2)])
+@pytest.mark.parametrize("D,hq,hkv", [(128, 8, 2), (64, 4, 4), (128, 16, 1), (32, 4, 2), (64, 8, 1)])
 def test_varlen_matches_oracle(D, hq, hkv):
     B, n_max = 5, 700
     q, K, V, s = make(700 + D, B, hq, hkv, n_max, D, D)
@@ -246,7 +274,7 @@ def test_append_out_of_range_position_is_skipped_and_reported():
 # multi-step decode: append then attend, token by token
 # ---------------------------------------------------------------------------------------
 @pytest.mark.parametrize("fused", [True, False])
-@pytest.mark.parametrize("D,hq,hkv", [(128, 8, 2), (64, 2, 1), (32, 8, 1), (16, 4, 4)])
+@pytest.mark.parametrize("D,hq,hkv", [(128, 8, 2), (64, 2, 1), (32, 8, 1), (16, 4, 4), (128, 8, 1), (64, 32, 2)])
 def test_multistep_small(fused, D, hq, hkv):
     w = mi.Workload("ms", 950 + D, 4, hq, hkv, 80, D, D, steps=40, len_lo=1, len_hi=40)
     B, n_max = w.batch, w.n
@@ -282,7 +310,7 @@ def test_multistep_small(fused, D, hq, hkv):
 
 
 @pytest.mark.parametrize("ctas,misalign_new", [(0, 0), (4000, 0), (0, 1), (5, 0)])
-@pytest.mark.parametrize("D,hq,hkv", [(128, 32, 8), (64, 16, 1), (128, 6, 2), (32, 2, 2)])
+@pytest.mark.parametrize("D,hq,hkv", [(128, 32, 8), (64, 16, 1), (128, 6, 2), (32, 2, 2), (128, 16, 2)])
 def test_append_decode_single_call(ctas, misalign_new, D, hq, hkv):
     # one call appends at pos[b] and attends over pos[b]+1 rows; lengths are not modified.
     # ctas=4000 and a k_new that is only 4-byte aligned take the three-launch fallback.
