@@ -219,9 +219,9 @@ static cudaError_t launch_mma_cfg(const DecodeArgs &a, int num_ctas, cudaStream_
 static cudaError_t launch_stream(const StreamPlan &p, const DecodeArgs &a, int num_ctas,
                                  cudaStream_t st)
 {
-    if (p.mma) {                         //                                     D   S  W
-        if (p.D == 128) return launch_mma_cfg<MmaCfg<128, 2, 5>>(a, num_ctas, st);
-        return launch_mma_cfg<MmaCfg<64, 2, 8>>(a, num_ctas, st);
+    if (p.mma) {                         //                                     D   S  P  paired
+        if (p.D == 128) return launch_mma_cfg<MmaCfg<128, 3, 4, true>>(a, num_ctas, st);
+        return launch_mma_cfg<MmaCfg<64, 2, 8, false>>(a, num_ctas, st);
     }
     // The heavier configurations (many FMAs per fetched byte) run 16 warps per CTA: with
     // eight, two warps per scheduler cannot hide the shuffle and FMA latencies.
@@ -265,6 +265,9 @@ static GroupedPlan plan_grouped(const DeviceState &s, int batch, int h_q, int h_
     GroupedPlan p;
     const int g_s = h_q / h_kv;
     if (d_k != 128 || d_v != 128 || (g_s != 16 && g_s != 32 && g_s != 64)) return p;
+    // Groups of 16 are faster as two groups of 8 on the warp-MMA streaming kernel (the K/V tile
+    // is read twice, the second time from L2); this kernel takes them only when forced.
+    if (g_s == 16 && g_force_path != MOA_PATH_GROUPED) return p;
     const long long units = (long long)batch * h_kv;
     if (units > 0x7fffffffLL / 256 || (long long)n > 0x7fffffffLL - 256) return p;
     // One CTA takes the whole group (measured faster than cutting a group of 64 into two

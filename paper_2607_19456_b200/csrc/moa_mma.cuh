@@ -6,7 +6,10 @@
 // cached rows of every (batch, kv head) unit are cut into 16-row tiles, all tiles form one
 // flat list dealt to persistent CTAs in equal contiguous ranges, every warp owns a private
 // ring of shared-memory stages filled by bulk asynchronous copies, split units are merged
-// by the CTA that delivers the last partial.  What differs is the arithmetic of a tile.
+// by the CTA that delivers the last partial.  What differs is the arithmetic of a tile, and
+// that warps work in pairs: one warp owns the K tiles (scores, online softmax), its partner
+// the V tiles (weighted sum); probabilities and rescale factors pass from one to the other
+// through a double-buffered shared-memory slot guarded by two mbarriers each way.
 // With 8 query heads per fetched row the FMA kernel is bound by instruction issue, not by
 // HBM; here a warp computes
 //     S^T [16 rows x 8 heads]   = K_tile [16 x d]  * Q^T [d x 8]        (m16n8k8, TF32)
@@ -40,34 +43,35 @@
 
 namespace moa {
 
-template <int D_, int S_, int W_>
+template <int D_, int S_, int P_, bool PAIRED_>
 struct MmaCfg {
     static constexpr int D = D_;              // d_k == d_v
     static constexpr int G = 8;               // query heads per (virtual) kv head
     static constexpr int S = S_;              // ring stages per warp
-    static constexpr int W = W_;              // warps per CTA
+    static constexpr bool PAIRED = PAIRED_;   // a tile is worked on by a warp pair / by one warp
+    static constexpr int P = P_;              // independent tile streams (pairs or single warps) per CTA
+    static constexpr int W = PAIRED ? 2 * P : P;   // warps per CTA
     static constexpr int R = 16;              // rows per tile
     static constexpr int LPR = D / 4;         // float4 per row
     static constexpr int NJ = D / 16;         // K chunks a lane reads per row (2 k-steps each)
     static constexpr int NU = D / 32;         // V chunks a lane reads per row (2 feature tiles each)
     static constexpr int MT = D / 16;         // 16-feature output tiles
-    static constexpr int CG = D / 32;         // 128-byte column groups of a row
     static constexpr int SUBT = R * 32;       // floats of one [16 rows][32 floats] sub-tile
-    static constexpr int OFF_V = R * D;       // stage: K tile, V tile, new K row, new V row
-    static constexpr int OFF_NEW = 2 * R * D;
-    static constexpr int STAGE_FLOATS = ((2 * R * D + 2 * D) * 4 + 1023) / 1024 * 256;   // whole KB
-    static constexpr int PT_STRIDE = 20;      // floats between heads in the P^T staging buffer
+    static constexpr int STAGE_FLOATS = PAIRED ? R * D : 2 * R * D;   // one operand's tile / K tile + V tile
+    static constexpr int PT_STRIDE = 20;      // floats between heads in a P^T hand-over buffer
+    static constexpr int PBUF_FLOATS = G * PT_STRIDE + G;   // P^T [8 heads][16 rows] + alpha [8 heads]
     static constexpr int PS = D + 4;          // floats per partial: o[D], m, l, 2 pad
     static constexpr int THREADS = W * 32;
     static_assert(D == 64 || D == 128, "row must be 256 or 512 bytes");
-
     static_assert((STAGE_FLOATS * 4) % 1024 == 0, "swizzled sub-tiles need 1024-byte alignment");
+
     static constexpr size_t OFF_RING = 0;             // from the 1024-byte aligned base
     static constexpr size_t OFF_MERGE_O = OFF_RING + sizeof(float) * W * S * STAGE_FLOATS;
-    static constexpr size_t OFF_MERGE_ML = OFF_MERGE_O + sizeof(float) * W * G * D;
-    static constexpr size_t OFF_PT = OFF_MERGE_ML + sizeof(float) * W * G * 2;
-    static constexpr size_t OFF_BAR = (OFF_PT + sizeof(float) * W * G * PT_STRIDE + 15) / 16 * 16;
-    static constexpr size_t SMEM_BYTES = OFF_BAR + sizeof(uint64_t) * W * S + 1024;   // + alignment slack
+    static constexpr size_t OFF_MERGE_ML = OFF_MERGE_O + sizeof(float) * P * G * D;
+    static constexpr size_t OFF_PBUF = OFF_MERGE_ML + sizeof(float) * P * G * 2;
+    static constexpr size_t OFF_BAR = (OFF_PBUF + sizeof(float) * P * 2 * PBUF_FLOATS + 15) / 16 * 16;
+    static constexpr int NBAR = W * S + 4 * P;        // tile landed; per pair: P^T ready x2, P^T consumed x2 (paired mode)
+    static constexpr size_t SMEM_BYTES = OFF_BAR + sizeof(uint64_t) * NBAR + 1024;   // + alignment slack
 };
 
 __device__ __forceinline__ void mma_tf32_16x8x8(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
@@ -107,30 +111,49 @@ __device__ __forceinline__ void mma3(float (&acc_hh)[4], float (&acc_lh)[4], flo
     mma_tf32_16x8x8(acc_hl, ah[0], ah[1], ah[2], ah[3], bl0, bl1);
 }
 
+// Per-thread running state of the two halves of a tile's work.
+template <int NJ>
+struct ScoreState {
+    uint32_t qh[NJ][4], ql[NJ][4];   // Q^T fragments of head g (chunk t+4j of the scaled query row), split
+    float m_run[2], l_run[2];        // heads 2t, 2t+1: running maximum, this thread's share of the sum
+};
+template <int MT>
+struct PvState {
+    float om[MT][4];                 // O^T fragments: features (by 16-feature tile) x heads 2t, 2t+1
+};
+
 template <class C>
 __global__ void __launch_bounds__(C::THREADS, 1)
 mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant__ CUtensorMap tmapV, const DecodeArgs a)
 {
-    constexpr int D = C::D, G = C::G, S = C::S, W = C::W, R = C::R, LPR = C::LPR, NJ = C::NJ, NU = C::NU,
+    constexpr int D = C::D, G = C::G, S = C::S, P = C::P, R = C::R, LPR = C::LPR, NJ = C::NJ, NU = C::NU,
                   MT = C::MT, SUBT = C::SUBT, PS = C::PS, PTS = C::PT_STRIDE;
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     unsigned char *const smem_m = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     float *ring = reinterpret_cast<float *>(smem_m + C::OFF_RING);
     float *merge_o = reinterpret_cast<float *>(smem_m + C::OFF_MERGE_O);
     float *merge_ml = reinterpret_cast<float *>(smem_m + C::OFF_MERGE_ML);
-    float *pt_all = reinterpret_cast<float *>(smem_m + C::OFF_PT);
+    float *pbuf_all = reinterpret_cast<float *>(smem_m + C::OFF_PBUF);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem_m + C::OFF_BAR);
     __shared__ int s_last;
     __shared__ int s_pref[kPrefixBatch + 1];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = lane >> 2, t = lane & 3;
+    // Paired mode: the two warps of a pair work on the same tiles, the score warp (even) turns a
+    // K tile into probabilities, the weighted-sum warp (odd) multiplies them into the V tile one
+    // or two tiles later; each fetches its own operand into its own ring.  It halves the
+    // registers a warp needs (d = 128).  Single mode: one warp does both, one after the other,
+    // on a stage that holds the K and the V tile; fewer fixed costs per tile (d = 64).
+    constexpr bool PAIRED = C::PAIRED;
+    const int pair = PAIRED ? (warp >> 1) : warp;
+    const bool is_pv = PAIRED && (warp & 1) != 0;
     // MMA row index m (0..7) <-> tile row: the two rows read in one shared-memory phase (g even
     // and odd) lie four rows apart, which the swizzle turns into disjoint halves of the banks.
     const int rowA = (g >> 1) + 4 * (g & 1), rowB = rowA + 8;
     const int h_stored = a.h_kv / a.kv_share;
 
-    if (tid < W * S) mbar_init(smem_u32(&bars[tid]), 1);
+    if (tid < C::NBAR) mbar_init(smem_u32(&bars[tid]), 1);
     if (tid == 0) { tc::prefetch_tmap(&tmapK); tc::prefetch_tmap(&tmapV); }
     mbar_fence_init();
     __syncthreads();
@@ -149,10 +172,14 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
     if (c0 < c1) {                            // uniform for the whole CTA
     float *my_ring = ring + (size_t)warp * S * C::STAGE_FLOATS;
     const uint32_t my_bar0 = smem_u32(&bars[warp * S]);
-    float *my_pt = pt_all + (size_t)warp * G * PTS;
+    float *my_pbuf = pbuf_all + (size_t)pair * 2 * C::PBUF_FLOATS;
+    const uint32_t bar_pfull0 = smem_u32(&bars[C::W * S + 4 * pair]), bar_pfree0 = bar_pfull0 + 16u;
+    const CUtensorMap *my_map = is_pv ? &tmapV : &tmapK;
+    const float *my_new = is_pv ? a.v_new : a.k_new;
+    float *my_cache = is_pv ? a.Vw : a.Kw;
 
-    // ---- load side: this warp's tiles are c0+warp, c0+warp+W, ... ------------------------
-    long long jl = c0 + warp;
+    // ---- load side: this pair's tiles are c0+pair, c0+pair+P, ... ------------------------
+    long long jl = c0 + pair;
     int kl = 0;
     Cursor lc = cursor_at<R>(a, (jl < c1) ? jl : c0, pref);
     size_t slab = 0;                           // stored (batch, kv head) of the unit under lc
@@ -169,35 +196,27 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
             load_unit_changed();
         }
         const int row0 = (int)(jl - lc.first) * R;
-        const int nr = (lc.len - row0 < R) ? lc.len - row0 : R;
-        // Fused append: the unit's last row is the token being appended; it comes from
-        // k_new / v_new (it lands beside the tile and replaces the tile's last row before use)
-        // and this warp also stores it into the cache.
-        const bool has_new = (a.k_new != nullptr) && (row0 + nr == lc.len);
-        const int nr_cache = has_new ? nr - 1 : nr;
         const size_t row = slab * (size_t)a.n_max + row0;
         if (lane == 0) {
             const int stage = kl % S;
             const uint32_t bar = my_bar0 + 8u * stage;
-            const uint32_t dst = smem_u32(my_ring + (size_t)stage * C::STAGE_FLOATS);
             // A box is always transferred whole (rows past the end of the cache read as zero;
             // rows past the end of the unit belong to the next unit and are masked later).
-            mbar_expect_tx(bar, (2u * R + (has_new ? 2u : 0u)) * D * 4u);
-            tc::tma_load_3d(dst, &tmapK, 0, (int)row, 0, bar);
-            tc::tma_load_3d(dst + C::OFF_V * 4u, &tmapV, 0, (int)row, 0, bar);
-            if (has_new) {
-                bulk_g2s(dst + C::OFF_NEW * 4u, a.k_new + slab * D, D * 4u, bar);
-                bulk_g2s(dst + (C::OFF_NEW + D) * 4u, a.v_new + slab * D, D * 4u, bar);
-            }
+            const uint32_t dst = smem_u32(my_ring + (size_t)stage * C::STAGE_FLOATS);
+            mbar_expect_tx(bar, (uint32_t)C::STAGE_FLOATS * 4u);
+            tc::tma_load_3d(dst, my_map, 0, (int)row, 0, bar);
+            if (!PAIRED) tc::tma_load_3d(dst + R * D * 4u, &tmapV, 0, (int)row, 0, bar);
         }
-        if (has_new && writes_new && lane < LPR) {
-            const size_t dst_row = (row + (size_t)nr_cache) * D + lane * 4;
-            *reinterpret_cast<float4 *>(a.Kw + dst_row) =
-                *reinterpret_cast<const float4 *>(a.k_new + slab * D + lane * 4);
-            *reinterpret_cast<float4 *>(a.Vw + dst_row) =
-                *reinterpret_cast<const float4 *>(a.v_new + slab * D + lane * 4);
+        // Fused append: the unit's last row is the token being appended.  The warp that fetches
+        // the tile holding it also stores it into the cache (K by the score warp, V by the other);
+        // the tile's copy of that row is replaced from k_new / v_new before use.
+        if (writes_new && row0 + R >= lc.len && lane < LPR) {
+            const size_t dst = (slab * (size_t)a.n_max + (size_t)(lc.len - 1)) * D + lane * 4;
+            *reinterpret_cast<float4 *>(my_cache + dst) = *reinterpret_cast<const float4 *>(my_new + slab * D + lane * 4);
+            if (!PAIRED)
+                *reinterpret_cast<float4 *>(a.Vw + dst) = *reinterpret_cast<const float4 *>(a.v_new + slab * D + lane * 4);
         }
-        jl += W;
+        jl += P;
         ++kl;
     };
 #pragma unroll 1
@@ -205,51 +224,15 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
 
     // ---- compute side ------------------------------------------------------------------
     Cursor cc = cursor_at<R>(a, c0, pref);
-    // Q^T fragments of head g: chunk t+4j of the scaled query row, split.  Running state of
-    // heads 2t and 2t+1: maximum, this thread's share of the sum, and the O^T fragments.
-    uint32_t qh[NJ][4], ql[NJ][4];
-    float om[MT][4];
-    float m_run[2], l_run[2];
-    auto begin_unit = [&]() {
-        const float *qb = a.q + ((size_t)cc.b * a.h_q + (size_t)cc.h * a.g_s) * D;
-#pragma unroll
-        for (int j = 0; j < NJ; ++j) {
-            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (g < a.g_s) v = *reinterpret_cast<const float4 *>(qb + (size_t)g * D + (t + 4 * j) * 4);
-            const Split4 s = split4(make_float4(v.x * a.qscale, v.y * a.qscale, v.z * a.qscale, v.w * a.qscale));
-#pragma unroll
-            for (int i = 0; i < 4; ++i) { qh[j][i] = s.h[i]; ql[j][i] = s.l[i]; }
-        }
-#pragma unroll
-        for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) om[mt][i] = 0.f;
-        m_run[0] = m_run[1] = -INFINITY;
-        l_run[0] = l_run[1] = 0.f;
-    };
+    // float offset, inside a tile, of 16-byte chunk `ch` of row r
+    auto chunk_at = [](int r, int ch) { return (ch >> 3) * SUBT + r * 32 + (((ch & 7) ^ (r & 7)) << 2); };
 
-    // Merge the W running states of this CTA for the unit under `cc` and emit either the
-    // final output rows or this CTA's partial triple; with completion counters in use, the
-    // CTA that delivers the last partial of a split unit also merges that unit's partials.
-    auto finish_unit = [&]() {
-#pragma unroll
-        for (int i = 0; i < 2; ++i) {
-            float l = l_run[i];
-            l += __shfl_xor_sync(0xffffffffu, l, 4);
-            l += __shfl_xor_sync(0xffffffffu, l, 8);
-            l += __shfl_xor_sync(0xffffffffu, l, 16);
-            if (g == 0) {
-                merge_ml[(warp * G + 2 * t + i) * 2 + 0] = m_run[i];
-                merge_ml[(warp * G + 2 * t + i) * 2 + 1] = l;
-            }
-        }
-#pragma unroll
-        for (int mt = 0; mt < MT; ++mt) {
-            // output tile mt = 2u+e holds features 32u + 4g + 2e (+1) of heads 2t (+1)
-            const int f = 32 * (mt >> 1) + 4 * g + 2 * (mt & 1);
-            float *o0 = merge_o + ((size_t)(warp * G + 2 * t)) * D + f;
-            o0[0] = om[mt][0]; o0[D] = om[mt][1]; o0[1] = om[mt][2]; o0[D + 1] = om[mt][3];
-        }
+    // Merge the P running states of this CTA for the unit under `cc` (each pair has published
+    // (m, l) and O through `publish`) and emit either the final output rows or this CTA's
+    // partial triple; with completion counters in use, the CTA that delivers the last partial
+    // of a split unit also merges that unit's partials.
+    auto finish_unit = [&](auto publish) {
+        publish();
         __syncthreads();
         const long long seg_begin = (c0 > cc.first) ? c0 : cc.first;
         const long long unit_end = cc.first + cc.ub;
@@ -259,11 +242,11 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
             const int hg = idx / LPR, d4 = idx % LPR;
             float M = -INFINITY;
 #pragma unroll
-            for (int v = 0; v < W; ++v) M = fmaxf(M, merge_ml[(v * G + hg) * 2]);
+            for (int v = 0; v < P; ++v) M = fmaxf(M, merge_ml[(v * G + hg) * 2]);
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
             float L = 0.f;
 #pragma unroll
-            for (int v = 0; v < W; ++v) {
+            for (int v = 0; v < P; ++v) {
                 const float f = exp2_diff(merge_ml[(v * G + hg) * 2], M);
                 const float4 x = *reinterpret_cast<const float4 *>(merge_o + ((size_t)(v * G + hg)) * D + d4 * 4);
                 acc.x = fmaf(x.x, f, acc.x); acc.y = fmaf(x.y, f, acc.y);
@@ -335,21 +318,89 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
         }
     };
 
-    // float offset, inside a tile, of 16-byte chunk `ch` of row r
-    auto chunk_at = [](int r, int ch) { return (ch >> 3) * SUBT + r * 32 + (((ch & 7) ^ (r & 7)) << 2); };
-    auto process_tile = [&](float *stage_base, int nr, bool has_new, auto full_tag) {
-        constexpr bool FULL = decltype(full_tag)::value;
-        float *sK = stage_base, *sV = stage_base + C::OFF_V;
-        if (has_new) {                             // the appended token is the tile's last row
-            if (lane < LPR) {
-                const float4 kn = *reinterpret_cast<const float4 *>(stage_base + C::OFF_NEW + lane * 4);
-                const float4 vn = *reinterpret_cast<const float4 *>(stage_base + C::OFF_NEW + D + lane * 4);
-                *reinterpret_cast<float4 *>(sK + chunk_at(nr - 1, lane)) = kn;
-                *reinterpret_cast<float4 *>(sV + chunk_at(nr - 1, lane)) = vn;
+    // One loop for both roles: walk this pair's tiles, closing units on the way.  `begin`,
+    // `publish` and `tile` are the role's parts.
+    auto run = [&](auto begin, auto publish, auto tile) {
+        begin();
+        bool failed = false;
+        int k = 0;
+#pragma unroll 1
+        for (long long j = c0 + pair; j < c1; j += P, ++k) {
+            while (j >= cc.first + cc.ub) {
+                finish_unit(publish);
+                cursor_next_unit<R>(a, cc);
+                begin();
             }
-            __syncwarp();
+            const int stage = k % S;
+            if (!failed && !mbar_test_wait(my_bar0 + 8u * stage, (uint32_t)(k / S) & 1u) &&
+                !mbar_wait_bounded(my_bar0 + 8u * stage, (uint32_t)(k / S) & 1u)) {
+                failed = true;
+                if (lane == 0) raise_status(MOA_STATUS_WAIT_TIMEOUT);
+            }
+            if (!failed) {
+                const int row0 = (int)(j - cc.first) * R;
+                const int nr = (cc.len - row0 < R) ? cc.len - row0 : R;
+                float *tile_base = my_ring + (size_t)stage * C::STAGE_FLOATS;
+                if ((a.k_new != nullptr) && (row0 + nr == cc.len)) {
+                    // the appended token is this tile's last row: take it from k_new / v_new
+                    if (lane < LPR) {
+                        const size_t cslab = (size_t)cc.b * h_stored + cc.h / a.kv_share;
+                        *reinterpret_cast<float4 *>(tile_base + chunk_at(nr - 1, lane)) =
+                            *reinterpret_cast<const float4 *>(my_new + cslab * D + lane * 4);
+                        if (!PAIRED)
+                            *reinterpret_cast<float4 *>(tile_base + R * D + chunk_at(nr - 1, lane)) =
+                                *reinterpret_cast<const float4 *>(a.v_new + cslab * D + lane * 4);
+                    }
+                    tc::fence_async_smem();        // plain stores to the stage precede its next bulk copy
+                    __syncwarp();
+                }
+                if (nr == R) failed = !tile(tile_base, nr, k, std::true_type{});
+                else failed = !tile(tile_base, nr, k, std::false_type{});
+                if (failed && lane == 0) raise_status(MOA_STATUS_WAIT_TIMEOUT);
+            }
+            __syncwarp();                          // all lanes are done with this stage
+            if (!failed && jl < c1) issue_next_load();
         }
-        // ---- S^T = K_tile * Q^T: 2*NJ k-steps, two accumulator chains each for hi and lo
+        while (cc.first + cc.ub < c1) {            // units after this pair's last tile
+            finish_unit(publish);
+            cursor_next_unit<R>(a, cc);
+            begin();
+        }
+        finish_unit(publish);
+    };
+
+    // ================= score part: S^T = K_tile * Q^T, online softmax, P^T hand-over ==========
+    // State: Q^T fragments of head g (chunk t+4j of the scaled query row, split), running
+    // maximum and this thread's share of the sum for heads 2t and 2t+1.
+    auto score_begin = [&](ScoreState<NJ> &st) {
+        const float *qb = a.q + ((size_t)cc.b * a.h_q + (size_t)cc.h * a.g_s) * D;
+#pragma unroll
+        for (int j = 0; j < NJ; ++j) {
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (g < a.g_s) v = *reinterpret_cast<const float4 *>(qb + (size_t)g * D + (t + 4 * j) * 4);
+            const Split4 s = split4(make_float4(v.x * a.qscale, v.y * a.qscale, v.z * a.qscale, v.w * a.qscale));
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { st.qh[j][i] = s.h[i]; st.ql[j][i] = s.l[i]; }
+        }
+        st.m_run[0] = st.m_run[1] = -INFINITY;
+        st.l_run[0] = st.l_run[1] = 0.f;
+    };
+    auto score_publish = [&](const ScoreState<NJ> &st) {
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            float l = st.l_run[i];
+            l += __shfl_xor_sync(0xffffffffu, l, 4);
+            l += __shfl_xor_sync(0xffffffffu, l, 8);
+            l += __shfl_xor_sync(0xffffffffu, l, 16);
+            if (g == 0) {
+                merge_ml[(pair * G + 2 * t + i) * 2 + 0] = st.m_run[i];
+                merge_ml[(pair * G + 2 * t + i) * 2 + 1] = l;
+            }
+        }
+    };
+    auto score_tile = [&](ScoreState<NJ> &st, const float *sK, int nr, int k, auto full_tag) -> bool {
+        constexpr bool FULL = decltype(full_tag)::value;
+        // 2*NJ k-steps, two accumulator chains for each of the three products
         float sh[2][4], sl[2][4], sm[2][4];
 #pragma unroll
         for (int c = 0; c < 2; ++c)
@@ -363,7 +414,7 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
             for (int e = 0; e < 2; ++e) {          // elements (2e, 2e+1) of the chunk are k-slots (t, t+4)
                 const uint32_t ah[4] = {ka.h[2 * e], kb.h[2 * e], ka.h[2 * e + 1], kb.h[2 * e + 1]};
                 const uint32_t al[4] = {ka.l[2 * e], kb.l[2 * e], ka.l[2 * e + 1], kb.l[2 * e + 1]};
-                mma3(sh[e], sl[e], sm[e], ah, al, qh[j][2 * e], qh[j][2 * e + 1], ql[j][2 * e], ql[j][2 * e + 1]);
+                mma3(sh[e], sl[e], sm[e], ah, al, st.qh[j][2 * e], st.qh[j][2 * e + 1], st.ql[j][2 * e], st.ql[j][2 * e + 1]);
             }
         }
         // this thread's scores: rows rowA (0,1) and rowB (2,3) of heads 2t (0,2) and 2t+1 (1,3)
@@ -374,7 +425,7 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
             if (rowA >= nr) { s[0] = -INFINITY; s[1] = -INFINITY; }
             if (rowB >= nr) { s[2] = -INFINITY; s[3] = -INFINITY; }
         }
-        // ---- online softmax per head (row maximum across the 8 lanes with the same t)
+        // online softmax per head (row maximum across the 8 lanes with the same t)
         float alpha[2], p[4];
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
@@ -382,27 +433,59 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
             bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 4));
             bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 8));
             bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 16));
-            const float m_new = fmaxf(m_run[i], bm);
-            alpha[i] = exp2_diff(m_run[i], m_new);
+            const float m_new = fmaxf(st.m_run[i], bm);
+            alpha[i] = exp2_diff(st.m_run[i], m_new);
             p[i] = exp2_diff(s[i], m_new);
             p[i + 2] = exp2_diff(s[i + 2], m_new);
-            l_run[i] = fmaf(l_run[i], alpha[i], p[i] + p[i + 2]);
-            m_run[i] = m_new;
+            st.l_run[i] = fmaf(st.l_run[i], alpha[i], p[i] + p[i + 2]);
+            st.m_run[i] = m_new;
         }
-        // ---- P^T through shared memory: lane (g, t) fetches rows 2t, 2t+1, 2t+8, 2t+9 of head g
-        // (the rows whose V it loads) with one 128-bit read
-        {
-            const int pa = 4 * ((rowA >> 1) & 3) + (rowA & 1), pb = pa + 2;
-            my_pt[(2 * t) * PTS + pa] = p[0];
-            my_pt[(2 * t + 1) * PTS + pa] = p[1];
-            my_pt[(2 * t) * PTS + pb] = p[2];
-            my_pt[(2 * t + 1) * PTS + pb] = p[3];
-        }
+        // P^T and the rescale factors go to the weighted-sum part through one of two buffers:
+        // lane (g, t) there fetches rows 2t, 2t+1, 2t+8, 2t+9 of head g (the rows whose V it
+        // loads) with one 128-bit read
+        const int b = k & 1, use = k >> 1;
+        if (PAIRED && use >= 1 && !mbar_wait_bounded(bar_pfree0 + 8u * b, (uint32_t)(use - 1) & 1u)) return false;
+        float *pt = my_pbuf + b * C::PBUF_FLOATS;
+        const int pa = 4 * ((rowA >> 1) & 3) + (rowA & 1), pb = pa + 2;
+        pt[(2 * t) * PTS + pa] = p[0];
+        pt[(2 * t + 1) * PTS + pa] = p[1];
+        pt[(2 * t) * PTS + pb] = p[2];
+        pt[(2 * t + 1) * PTS + pb] = p[3];
+        if (g == 0) { pt[G * PTS + 2 * t] = alpha[0]; pt[G * PTS + 2 * t + 1] = alpha[1]; }
         __syncwarp();
-        const Split4 pp = split4(*reinterpret_cast<const float4 *>(my_pt + g * PTS + 4 * t));
-        __syncwarp();                              // the buffer may be rewritten by the next tile
-        // ---- O^T += V_tile^T * P^T, tile by tile of 16 features; each tile's products start from
-        // zero and are then added to the running values, rescaled by alpha
+        if (PAIRED && lane == 0) tc::mbar_arrive(bar_pfull0 + 8u * b);
+        return true;
+    };
+
+    // ================= weighted-sum part: O^T += V_tile^T * P^T ================================
+    // State: O^T fragments, features (by 16-feature tile) x heads 2t, 2t+1.
+    auto pv_begin = [&](PvState<MT> &st) {
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) st.om[mt][i] = 0.f;
+    };
+    auto pv_publish = [&](const PvState<MT> &st) {
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+            // output tile mt = 2u+e holds features 32u + 4g + 2e (+1) of heads 2t (+1)
+            const int f = 32 * (mt >> 1) + 4 * g + 2 * (mt & 1);
+            float *o0 = merge_o + ((size_t)(pair * G + 2 * t)) * D + f;
+            o0[0] = st.om[mt][0]; o0[D] = st.om[mt][1]; o0[1] = st.om[mt][2]; o0[D + 1] = st.om[mt][3];
+        }
+    };
+    auto pv_tile = [&](PvState<MT> &st, const float *sV, int nr, int k, auto full_tag) -> bool {
+        constexpr bool FULL = decltype(full_tag)::value;
+        const int b = k & 1, use = k >> 1;
+        if (PAIRED && !mbar_test_wait(bar_pfull0 + 8u * b, (uint32_t)use & 1u) &&
+            !mbar_wait_bounded(bar_pfull0 + 8u * b, (uint32_t)use & 1u)) return false;
+        const float *pt = my_pbuf + b * C::PBUF_FLOATS;
+        const Split4 pp = split4(*reinterpret_cast<const float4 *>(pt + g * PTS + 4 * t));
+        const float alpha[2] = {pt[G * PTS + 2 * t], pt[G * PTS + 2 * t + 1]};
+        __syncwarp();
+        if (PAIRED && lane == 0) tc::mbar_arrive(bar_pfree0 + 8u * b);
+        // 16 features at a time; a tile's products start from zero and are then added to the
+        // running values, rescaled by alpha
 #pragma unroll
         for (int u = 0; u < NU; ++u) {
             Split4 v[4];
@@ -426,45 +509,32 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
                 }
                 const int mt = 2 * u + e;
 #pragma unroll
-                for (int i = 0; i < 4; ++i) om[mt][i] = fmaf(om[mt][i], alpha[i & 1], oh[i] + (ol[i] + ox[i]));
+                for (int i = 0; i < 4; ++i) st.om[mt][i] = fmaf(st.om[mt][i], alpha[i & 1], oh[i] + (ol[i] + ox[i]));
             }
         }
+        return true;
     };
 
-    begin_unit();
-    bool failed = false;
-    int k = 0;
-#pragma unroll 1
-    for (long long j = c0 + warp; j < c1; j += W, ++k) {
-        while (j >= cc.first + cc.ub) {
-            finish_unit();
-            cursor_next_unit<R>(a, cc);
-            begin_unit();
-        }
-        const int stage = k % S;
-        if (!failed && !mbar_test_wait(my_bar0 + 8u * stage, (uint32_t)(k / S) & 1u) &&
-            !mbar_wait_bounded(my_bar0 + 8u * stage, (uint32_t)(k / S) & 1u)) {
-            failed = true;
-            if (lane == 0) raise_status(MOA_STATUS_WAIT_TIMEOUT);
-        }
-        if (!failed) {
-            const int row0 = (int)(j - cc.first) * R;
-            const int nr = (cc.len - row0 < R) ? cc.len - row0 : R;
-            float *stage_base = my_ring + (size_t)stage * C::STAGE_FLOATS;
-            const bool has_new = (a.k_new != nullptr) && (row0 + nr == cc.len);
-            if (nr == R) process_tile(stage_base, nr, has_new, std::true_type{});
-            else process_tile(stage_base, nr, has_new, std::false_type{});
-            if (has_new) tc::fence_async_smem();   // plain stores to the stage precede the next bulk copy
-        }
-        __syncwarp();                          // all lanes are done with this stage
-        if (!failed && jl < c1) issue_next_load();
+    if (!PAIRED) {
+        ScoreState<NJ> ss;
+        PvState<MT> ps;
+        run([&]() { score_begin(ss); pv_begin(ps); }, [&]() { score_publish(ss); pv_publish(ps); },
+            [&](const float *tile_base, int nr, int k, auto full_tag) -> bool {
+                return score_tile(ss, tile_base, nr, k, full_tag) && pv_tile(ps, tile_base + R * D, nr, k, full_tag);
+            });
+    } else if (!is_pv) {
+        ScoreState<NJ> ss;
+        run([&]() { score_begin(ss); }, [&]() { score_publish(ss); },
+            [&](const float *tile_base, int nr, int k, auto full_tag) -> bool {
+                return score_tile(ss, tile_base, nr, k, full_tag);
+            });
+    } else {
+        PvState<MT> ps;
+        run([&]() { pv_begin(ps); }, [&]() { pv_publish(ps); },
+            [&](const float *tile_base, int nr, int k, auto full_tag) -> bool {
+                return pv_tile(ps, tile_base, nr, k, full_tag);
+            });
     }
-    while (cc.first + cc.ub < c1) {            // units after this warp's last tile
-        finish_unit();
-        cursor_next_unit<R>(a, cc);
-        begin_unit();
-    }
-    finish_unit();
     }  // c0 < c1
 
     // ---- whole-grid completion: range report and length advance by the last CTA ---------

@@ -50,7 +50,7 @@ def test_paper_gqa_shapes_d32(hkv):
 # ---------------------------------------------------------------------------------------
 def automatic_path(D, gs):
     """The kernel family the library picks for a dense, aligned call."""
-    if D == 128 and gs in (16, 32, 64):
+    if D == 128 and gs in (32, 64):
         return moa.PATH_GROUPED
     if gs <= 8:
         G = 1
@@ -112,7 +112,7 @@ def test_stream_kernel_any_cta_count_gives_the_same_answer(ctas):
                                      (3, 1, 4133), (1, 1, 20000), (40, 4, 300)])
 def test_grouped_kernel_shapes(gs, B, hkv, n):
     q, K, V, s = make(2000 + gs + n, B, gs * hkv, hkv, n, 128, 128)
-    out = gpu_decode(q, K, V, s, expect_path=moa.PATH_GROUPED)
+    out = gpu_decode(q, K, V, s, path=moa.PATH_GROUPED, expect_path=moa.PATH_GROUPED)
     assert max_err(out, oracle.decode(q, K, V, s)) <= TOL
 
 
@@ -130,7 +130,8 @@ def test_grouped_kernel_larger_scores_rising_maximum_and_small_n():
     K, V = np.ascontiguousarray(K[:, :, order]), np.ascontiguousarray(V[:, :, order])
     q2 = q.copy()
     q2[:] = q[:, :1]                       # every head sees the same ascending order
-    assert max_err(gpu_decode(q2 * 8, K, V, s, expect_path=moa.PATH_GROUPED), oracle.decode(q2 * 8, K, V, s)) <= TOL
+    assert max_err(gpu_decode(q2 * 8, K, V, s, path=moa.PATH_GROUPED, expect_path=moa.PATH_GROUPED),
+                   oracle.decode(q2 * 8, K, V, s)) <= TOL
     # few rows: no averaging hides a product error (this is what the three-term split is for)
     q, K, V, s = make(2102, 2, 64, 1, 3, 128, 128)
     assert max_err(gpu_decode(q, K, V, s, expect_path=moa.PATH_GROUPED), oracle.decode(q, K, V, s)) <= TOL
