@@ -135,6 +135,16 @@ def pinned_like(shape):
     return torch.empty(shape, dtype=torch.float32, pin_memory=True)
 
 
+# Shapes outside the five benchmark configurations, timed only, to show the kernels that
+# those five do not reach: groups of 8 and 16 heads (warp-MMA streaming kernel) and d = 32.
+EXTRA_WORKLOADS = {
+    "extra_group8_d128": mi.Workload("extra_group8_d128", 1101, 16, 64, 8, 8192, 128, 128),
+    "extra_group8_d64": mi.Workload("extra_group8_d64", 1102, 16, 64, 8, 16384, 64, 64),
+    "extra_group16_d128": mi.Workload("extra_group16_d128", 1103, 16, 128, 8, 8192, 128, 128),
+    "extra_mha_d32": mi.Workload("extra_mha_d32", 1104, 64, 32, 32, 4096, 32, 32),
+}
+
+
 class DenseRun:
     """append one row at the last position, then decode over n rows (dense cache)."""
 
@@ -513,10 +523,9 @@ def main():
     if rank == 0 and world == 1 and not args.no_others:
         del run
         torch.cuda.empty_cache()
-        for name in mi.WORKLOADS:
+        for name, ow in list(mi.WORKLOADS.items()) + list(EXTRA_WORKLOADS.items()):
             if name == wname:
                 continue
-            ow = mi.WORKLOADS[name]
             try:
                 if name == "multi_step":
                     r = MultiStepRun(ow)

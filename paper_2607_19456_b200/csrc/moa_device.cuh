@@ -269,4 +269,75 @@ __device__ __forceinline__ void cursor_next_unit(const DecodeArgs &a, Cursor &c)
     }
 }
 
+// ---- merge of a split unit's partials by the CTA that delivered the last one -------------
+// The partial triples (m, l, o[D]) of the unit live in slots of `a.ws`, one per CTA c in
+// [c_first, c_last] (slot 0 or 1 of that CTA: 0 if the unit starts before the CTA's range).
+// They are merged in CTA order, so the result does not depend on which CTA does it.  The
+// (m, l) pairs are first fetched by all threads at once into `stage` (one L2 round trip
+// instead of one per partial); `stage_floats` bounds how many partials are handled per
+// round, further rounds continue the same online merge.  Ends with a block barrier.
+template <int D>
+__device__ __forceinline__ void merge_unit_partials(const DecodeArgs &a, float *stage, int stage_floats, int G,
+                                                    long long c_first, long long c_last, long long bpc,
+                                                    long long unit_first, int b, int h, int tid, int nthreads)
+{
+    constexpr int LPR = D / 4, PS = D + 4;
+    const int ns = (int)(c_last - c_first) + 1;
+    const int per_round = stage_floats / (2 * G);
+    auto slot_of = [&](long long c, int hg) {
+        const int slot = (unit_first <= c * bpc) ? 0 : 1;
+        return a.ws + (((size_t)c * 2 + slot) * G + hg) * PS;
+    };
+    // thread -> (head, float4 column); with fewer threads than G * LPR a thread takes several
+    constexpr int kMaxItems = 4;
+    float M[kMaxItems], L[kMaxItems];
+    float4 acc[kMaxItems];
+#pragma unroll
+    for (int it = 0; it < kMaxItems; ++it) { M[it] = -INFINITY; L[it] = 0.f; acc[it] = make_float4(0.f, 0.f, 0.f, 0.f); }
+    for (int base = 0; base < ns; base += per_round) {
+        const int cnt = (ns - base < per_round) ? ns - base : per_round;
+        for (int i = tid; i < cnt * G; i += nthreads) {
+            const float *p = slot_of(c_first + base + i / G, i % G);
+            stage[2 * i] = __ldcg(p + D);
+            stage[2 * i + 1] = __ldcg(p + D + 1);
+        }
+        __syncthreads();
+#pragma unroll
+        for (int it = 0; it < kMaxItems; ++it) {
+            const int idx = tid + it * nthreads;
+            if (idx < G * LPR) {
+                const int hg = idx / LPR, d4 = idx % LPR;
+                float Mn = M[it];
+                for (int i = 0; i < cnt; ++i) Mn = fmaxf(Mn, stage[(i * G + hg) * 2]);
+                const float keep = exp2_diff(M[it], Mn);
+                acc[it].x *= keep; acc[it].y *= keep; acc[it].z *= keep; acc[it].w *= keep;
+                L[it] *= keep;
+                M[it] = Mn;
+#pragma unroll 8
+                for (int i = 0; i < cnt; ++i) {      // partials in CTA order; the loads are independent
+                    const float f = exp2_diff(stage[(i * G + hg) * 2], Mn);
+                    L[it] = fmaf(stage[(i * G + hg) * 2 + 1], f, L[it]);
+                    const float4 x = __ldcg(reinterpret_cast<const float4 *>(slot_of(c_first + base + i, hg) + d4 * 4));
+                    acc[it].x = fmaf(x.x, f, acc[it].x); acc[it].y = fmaf(x.y, f, acc[it].y);
+                    acc[it].z = fmaf(x.z, f, acc[it].z); acc[it].w = fmaf(x.w, f, acc[it].w);
+                }
+            }
+        }
+        __syncthreads();                       // the stage is rewritten by the next round / next unit
+    }
+#pragma unroll
+    for (int it = 0; it < kMaxItems; ++it) {
+        const int idx = tid + it * nthreads;
+        if (idx < G * LPR) {
+            const int hg = idx / LPR, d4 = idx % LPR;
+            if (hg < a.g_s) {
+                const float inv = 1.0f / L[it];
+                float *dst = a.out + ((size_t)b * a.h_q + (size_t)h * a.g_s + hg) * D + d4 * 4;
+                *reinterpret_cast<float4 *>(dst) =
+                    make_float4(acc[it].x * inv, acc[it].y * inv, acc[it].z * inv, acc[it].w * inv);
+            }
+        }
+    }
+}
+
 }  // namespace moa

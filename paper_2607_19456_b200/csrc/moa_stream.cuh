@@ -248,43 +248,8 @@ __global__ void __launch_bounds__(C::THREADS, 1) stream_decode_kernel(const Deco
             __syncthreads();
             if (s_last) {                          // uniform for the CTA
                 __threadfence();
-                // (m, l) of every partial of the unit, fetched by all threads at once: one L2
-                // round trip instead of one per partial
-                const int ns = (int)(c_last - c_first) + 1;
-                float *stage = merge_o;            // [ns][G][2]; merge_o is idle here
-                for (int i = tid; i < ns * G; i += C::THREADS) {
-                    const long long c = c_first + i / G;
-                    const int g = i % G;
-                    const int slot = (cc.first <= c * bpc) ? 0 : 1;
-                    const float *p = a.ws + (((size_t)c * 2 + slot) * G + g) * PS;
-                    stage[2 * i] = __ldcg(p + D);
-                    stage[2 * i + 1] = __ldcg(p + D + 1);
-                }
-                __syncthreads();
-                if (tid < G * LPR) {
-                    const int g = tid / LPR, d4 = tid % LPR;
-                    float M = -INFINITY;
-                    for (int i = 0; i < ns; ++i) M = fmaxf(M, stage[(i * G + g) * 2]);
-                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                    float L = 0.f;
-#pragma unroll 8
-                    for (int i = 0; i < ns; ++i) {      // partials in CTA order; the loads are independent
-                        const long long c = c_first + i;
-                        const int slot = (cc.first <= c * bpc) ? 0 : 1;
-                        const float *p = a.ws + (((size_t)c * 2 + slot) * G + g) * PS;
-                        const float f = exp2_diff(stage[(i * G + g) * 2], M);
-                        L = fmaf(stage[(i * G + g) * 2 + 1], f, L);
-                        const float4 t = __ldcg(reinterpret_cast<const float4 *>(p + d4 * 4));
-                        acc.x = fmaf(t.x, f, acc.x); acc.y = fmaf(t.y, f, acc.y);
-                        acc.z = fmaf(t.z, f, acc.z); acc.w = fmaf(t.w, f, acc.w);
-                    }
-                    if (g < a.g_s) {
-                        const float inv = 1.0f / L;
-                        float *dst = a.out + ((size_t)cc.b * a.h_q + (size_t)cc.h * a.g_s + g) * D + d4 * 4;
-                        *reinterpret_cast<float4 *>(dst) = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
-                    }
-                }
-                __syncthreads();                   // merge_o is written again by the next unit
+                merge_unit_partials<D>(a, merge_o, VW * G * D, G, c_first, c_last, bpc, cc.first, cc.b, cc.h, tid,
+                                       C::THREADS);
             }
         }
     };
