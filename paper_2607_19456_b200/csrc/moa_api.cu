@@ -134,6 +134,7 @@ static StreamPlan plan_stream(int g_s, int d_k, int d_v)
     p.D = d_k;
     p.G = stream_group(g_s, &p.share);
     p.mma = mma_allowed() && p.G == 8 && p.D >= 64;     // (the caller drops it for huge caches)
+    if (p.mma && g_s % 16 == 0) { p.G = 16; p.share = g_s / 16; }   // two 8-head tiles per fetched row
     p.R = p.mma ? 16 : rows_per_block(p.D, p.G);
     p.ok = true;
     return p;
@@ -220,8 +221,10 @@ static cudaError_t launch_stream(const StreamPlan &p, const DecodeArgs &a, int n
                                  cudaStream_t st)
 {
     if (p.mma) {                         //                                     D   S  P  paired
-        if (p.D == 128) return launch_mma_cfg<MmaCfg<128, 3, 4, true>>(a, num_ctas, st);
-        return launch_mma_cfg<MmaCfg<64, 2, 8, false>>(a, num_ctas, st);
+        if (p.D == 128 && p.G == 16) return launch_mma_cfg<MmaCfg<128, 3, 4, true, 2>>(a, num_ctas, st);
+        if (p.D == 128) return launch_mma_cfg<MmaCfg<128, 3, 4, true, 1>>(a, num_ctas, st);
+        if (p.G == 16) return launch_mma_cfg<MmaCfg<64, 2, 8, false, 2>>(a, num_ctas, st);
+        return launch_mma_cfg<MmaCfg<64, 2, 8, false, 1>>(a, num_ctas, st);
     }
     // The heavier configurations (many FMAs per fetched byte) run 16 warps per CTA: with
     // eight, two warps per scheduler cannot hide the shuffle and FMA latencies.
@@ -411,6 +414,7 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
     StreamPlan plan = plan_stream(g_s, d_k, d_v);
     if (plan.mma && (long long)batch * h_kv * n_max > 0x7fffff00LL) {   // row coordinates are 32-bit
         plan.mma = false;
+        plan.G = stream_group(g_s, &plan.share);
         plan.R = rows_per_block(plan.D, plan.G);
     }
     const bool fast_ok = plan.ok && aligned(q, 16) && aligned(K, 16) && aligned(V, 16) && aligned(out, 16);

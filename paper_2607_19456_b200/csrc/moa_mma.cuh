@@ -1,4 +1,4 @@
-// moa_mma.cuh -- split-sequence streaming decode kernel for groups of 8 (or 16) query
+// moa_mma.cuh -- split-sequence streaming decode kernel for groups of 8 or 16 query
 // heads per K/V head, with the two contractions on the warp-level tensor-core MMA.
 //
 // Steps I-III of Algorithm 1 (eqs. (1)-(3)) in online-softmax form with the psi-selection
@@ -43,10 +43,11 @@
 
 namespace moa {
 
-template <int D_, int S_, int P_, bool PAIRED_>
+template <int D_, int S_, int P_, bool PAIRED_, int NT_>
 struct MmaCfg {
     static constexpr int D = D_;              // d_k == d_v
-    static constexpr int G = 8;               // query heads per (virtual) kv head
+    static constexpr int NT = NT_;            // 8-head column tiles of the score matrix
+    static constexpr int G = 8 * NT;          // query heads per (virtual) kv head
     static constexpr int S = S_;              // ring stages per warp
     static constexpr bool PAIRED = PAIRED_;   // a tile is worked on by a warp pair / by one warp
     static constexpr int P = P_;              // independent tile streams (pairs or single warps) per CTA
@@ -63,12 +64,14 @@ struct MmaCfg {
     static constexpr int PS = D + 4;          // floats per partial: o[D], m, l, 2 pad
     static constexpr int THREADS = W * 32;
     static_assert(D == 64 || D == 128, "row must be 256 or 512 bytes");
+    static_assert(NT == 1 || NT == 2, "8 or 16 heads");
+    static_assert(G * LPR <= 4 * THREADS, "merge_unit_partials handles four items per thread");
     static_assert((STAGE_FLOATS * 4) % 1024 == 0, "swizzled sub-tiles need 1024-byte alignment");
 
     static constexpr size_t OFF_RING = 0;             // from the 1024-byte aligned base
     static constexpr size_t OFF_MERGE_O = OFF_RING + sizeof(float) * W * S * STAGE_FLOATS;
-    static constexpr size_t OFF_MERGE_ML = OFF_MERGE_O + sizeof(float) * P * G * D;
-    static constexpr size_t OFF_PBUF = OFF_MERGE_ML + sizeof(float) * P * G * 2;
+    static constexpr size_t OFF_MERGE_ML = OFF_MERGE_O + sizeof(float) * P * 8 * D;   // 8 heads at a time
+    static constexpr size_t OFF_PBUF = OFF_MERGE_ML + sizeof(float) * P * 8 * 2;
     static constexpr size_t OFF_BAR = (OFF_PBUF + sizeof(float) * P * 2 * PBUF_FLOATS + 15) / 16 * 16;
     static constexpr int NBAR = W * S + 4 * P;        // tile landed; per pair: P^T ready x2, P^T consumed x2 (paired mode)
     static constexpr size_t SMEM_BYTES = OFF_BAR + sizeof(uint64_t) * NBAR + 1024;   // + alignment slack
@@ -112,21 +115,21 @@ __device__ __forceinline__ void mma3(float (&acc_hh)[4], float (&acc_lh)[4], flo
 }
 
 // Per-thread running state of the two halves of a tile's work.
-template <int NJ>
+template <int NJ, int NT>
 struct ScoreState {
-    uint32_t qh[NJ][4], ql[NJ][4];   // Q^T fragments of head g (chunk t+4j of the scaled query row), split
-    float m_run[2], l_run[2];        // heads 2t, 2t+1: running maximum, this thread's share of the sum
+    uint32_t qh[NT][NJ][4], ql[NT][NJ][4];   // Q^T fragments of head 8nt+g (chunk t+4j of the scaled query row), split
+    float m_run[2 * NT], l_run[2 * NT];      // heads 8nt+2t, 8nt+2t+1: running maximum, this thread's share of the sum
 };
-template <int MT>
+template <int MT, int NT>
 struct PvState {
-    float om[MT][4];                 // O^T fragments: features (by 16-feature tile) x heads 2t, 2t+1
+    float om[MT][NT][4];                     // O^T fragments: features (by 16-feature tile) x heads 8nt+2t, 8nt+2t+1
 };
 
 template <class C>
 __global__ void __launch_bounds__(C::THREADS, 1)
 mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant__ CUtensorMap tmapV, const DecodeArgs a)
 {
-    constexpr int D = C::D, G = C::G, S = C::S, P = C::P, R = C::R, LPR = C::LPR, NJ = C::NJ, NU = C::NU,
+    constexpr int D = C::D, G = C::G, NT = C::NT, S = C::S, P = C::P, R = C::R, LPR = C::LPR, NJ = C::NJ, NU = C::NU,
                   MT = C::MT, SUBT = C::SUBT, PS = C::PS, PTS = C::PT_STRIDE;
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     unsigned char *const smem_m = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -232,41 +235,44 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
     // partial triple; with completion counters in use, the CTA that delivers the last partial
     // of a split unit also merges that unit's partials.
     auto finish_unit = [&](auto publish) {
-        publish();
-        __syncthreads();
         const long long seg_begin = (c0 > cc.first) ? c0 : cc.first;
         const long long unit_end = cc.first + cc.ub;
         const long long seg_end = (c1 < unit_end) ? c1 : unit_end;
         const bool complete = (seg_begin == cc.first) && (seg_end == unit_end);
-        for (int idx = tid; idx < G * LPR; idx += C::THREADS) {
-            const int hg = idx / LPR, d4 = idx % LPR;
-            float M = -INFINITY;
+#pragma unroll 1
+        for (int hb = 0; hb < NT; ++hb) {          // eight heads at a time through the merge buffers
+            publish(hb);
+            __syncthreads();
+            for (int idx = tid; idx < 8 * LPR; idx += C::THREADS) {
+                const int h8 = idx / LPR, d4 = idx % LPR, hg = 8 * hb + h8;
+                float M = -INFINITY;
 #pragma unroll
-            for (int v = 0; v < P; ++v) M = fmaxf(M, merge_ml[(v * G + hg) * 2]);
-            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-            float L = 0.f;
+                for (int v = 0; v < P; ++v) M = fmaxf(M, merge_ml[(v * 8 + h8) * 2]);
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                float L = 0.f;
 #pragma unroll
-            for (int v = 0; v < P; ++v) {
-                const float f = exp2_diff(merge_ml[(v * G + hg) * 2], M);
-                const float4 x = *reinterpret_cast<const float4 *>(merge_o + ((size_t)(v * G + hg)) * D + d4 * 4);
-                acc.x = fmaf(x.x, f, acc.x); acc.y = fmaf(x.y, f, acc.y);
-                acc.z = fmaf(x.z, f, acc.z); acc.w = fmaf(x.w, f, acc.w);
-                L = fmaf(merge_ml[(v * G + hg) * 2 + 1], f, L);
-            }
-            if (complete) {
-                if (hg < a.g_s) {
-                    const float inv = 1.0f / L;
-                    float *dst = a.out + ((size_t)cc.b * a.h_q + (size_t)cc.h * a.g_s + hg) * D + d4 * 4;
-                    *reinterpret_cast<float4 *>(dst) = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+                for (int v = 0; v < P; ++v) {
+                    const float f = exp2_diff(merge_ml[(v * 8 + h8) * 2], M);
+                    const float4 x = *reinterpret_cast<const float4 *>(merge_o + ((size_t)(v * 8 + h8)) * D + d4 * 4);
+                    acc.x = fmaf(x.x, f, acc.x); acc.y = fmaf(x.y, f, acc.y);
+                    acc.z = fmaf(x.z, f, acc.z); acc.w = fmaf(x.w, f, acc.w);
+                    L = fmaf(merge_ml[(v * 8 + h8) * 2 + 1], f, L);
                 }
-            } else {
-                const int slot = (seg_begin == c0) ? 0 : 1;
-                float *dst = a.ws + (((size_t)blockIdx.x * 2 + slot) * G + hg) * PS;
-                *reinterpret_cast<float4 *>(dst + d4 * 4) = acc;
-                if (d4 == 0) { dst[D] = M; dst[D + 1] = L; }
+                if (complete) {
+                    if (hg < a.g_s) {
+                        const float inv = 1.0f / L;
+                        float *dst = a.out + ((size_t)cc.b * a.h_q + (size_t)cc.h * a.g_s + hg) * D + d4 * 4;
+                        *reinterpret_cast<float4 *>(dst) = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+                    }
+                } else {
+                    const int slot = (seg_begin == c0) ? 0 : 1;
+                    float *dst = a.ws + (((size_t)blockIdx.x * 2 + slot) * G + hg) * PS;
+                    *reinterpret_cast<float4 *>(dst + d4 * 4) = acc;
+                    if (d4 == 0) { dst[D] = M; dst[D + 1] = L; }
+                }
             }
+            __syncthreads();
         }
-        __syncthreads();
         if (!complete && a.tickets != nullptr) {
             const long long c_first = cc.first / bpc, c_last = (unit_end - 1) / bpc;
             if (tid == 0) {
@@ -279,7 +285,7 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
             __syncthreads();
             if (s_last) {                          // uniform for the CTA
                 __threadfence();
-                merge_unit_partials<D>(a, merge_o, P * G * D, G, c_first, c_last, bpc, cc.first, cc.b, cc.h, tid,
+                merge_unit_partials<D>(a, merge_o, P * 8 * D, G, c_first, c_last, bpc, cc.first, cc.b, cc.h, tid,
                                        C::THREADS);
             }
         }
@@ -339,40 +345,48 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
     // ================= score part: S^T = K_tile * Q^T, online softmax, P^T hand-over ==========
     // State: Q^T fragments of head g (chunk t+4j of the scaled query row, split), running
     // maximum and this thread's share of the sum for heads 2t and 2t+1.
-    auto score_begin = [&](ScoreState<NJ> &st) {
+    auto score_begin = [&](ScoreState<NJ, NT> &st) {
         const float *qb = a.q + ((size_t)cc.b * a.h_q + (size_t)cc.h * a.g_s) * D;
 #pragma unroll
-        for (int j = 0; j < NJ; ++j) {
-            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (g < a.g_s) v = *reinterpret_cast<const float4 *>(qb + (size_t)g * D + (t + 4 * j) * 4);
-            const Split4 s = split4(make_float4(v.x * a.qscale, v.y * a.qscale, v.z * a.qscale, v.w * a.qscale));
+        for (int nt = 0; nt < NT; ++nt) {
+            const int hg = 8 * nt + g;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) { st.qh[j][i] = s.h[i]; st.ql[j][i] = s.l[i]; }
+            for (int j = 0; j < NJ; ++j) {
+                float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (hg < a.g_s) v = *reinterpret_cast<const float4 *>(qb + (size_t)hg * D + (t + 4 * j) * 4);
+                const Split4 s = split4(make_float4(v.x * a.qscale, v.y * a.qscale, v.z * a.qscale, v.w * a.qscale));
+#pragma unroll
+                for (int i = 0; i < 4; ++i) { st.qh[nt][j][i] = s.h[i]; st.ql[nt][j][i] = s.l[i]; }
+            }
         }
-        st.m_run[0] = st.m_run[1] = -INFINITY;
-        st.l_run[0] = st.l_run[1] = 0.f;
+#pragma unroll
+        for (int i = 0; i < 2 * NT; ++i) { st.m_run[i] = -INFINITY; st.l_run[i] = 0.f; }
     };
-    auto score_publish = [&](const ScoreState<NJ> &st) {
+    auto score_publish = [&](const ScoreState<NJ, NT> &st, int hb) {
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
-            float l = st.l_run[i];
+            float l = (NT == 2 && hb == 1) ? st.l_run[2 + i] : st.l_run[i];
+            const float m = (NT == 2 && hb == 1) ? st.m_run[2 + i] : st.m_run[i];
             l += __shfl_xor_sync(0xffffffffu, l, 4);
             l += __shfl_xor_sync(0xffffffffu, l, 8);
             l += __shfl_xor_sync(0xffffffffu, l, 16);
             if (g == 0) {
-                merge_ml[(pair * G + 2 * t + i) * 2 + 0] = st.m_run[i];
-                merge_ml[(pair * G + 2 * t + i) * 2 + 1] = l;
+                merge_ml[(pair * 8 + 2 * t + i) * 2 + 0] = m;
+                merge_ml[(pair * 8 + 2 * t + i) * 2 + 1] = l;
             }
         }
     };
-    auto score_tile = [&](ScoreState<NJ> &st, const float *sK, int nr, int k, auto full_tag) -> bool {
+    auto score_tile = [&](ScoreState<NJ, NT> &st, const float *sK, int nr, int k, auto full_tag) -> bool {
         constexpr bool FULL = decltype(full_tag)::value;
-        // 2*NJ k-steps, two accumulator chains for each of the three products
-        float sh[2][4], sl[2][4], sm[2][4];
+        // 2*NJ k-steps, two accumulator chains for each of the three products of each head tile;
+        // a K fragment is loaded and split once and used for all head tiles
+        float sh[NT][2][4], sl[NT][2][4], sm[NT][2][4];
 #pragma unroll
-        for (int c = 0; c < 2; ++c)
+        for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-            for (int i = 0; i < 4; ++i) { sh[c][i] = 0.f; sl[c][i] = 0.f; sm[c][i] = 0.f; }
+            for (int c = 0; c < 2; ++c)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) { sh[nt][c][i] = 0.f; sl[nt][c][i] = 0.f; sm[nt][c][i] = 0.f; }
 #pragma unroll
         for (int j = 0; j < NJ; ++j) {
             const Split4 ka = split4(*reinterpret_cast<const float4 *>(sK + chunk_at(rowA, t + 4 * j)));
@@ -381,44 +395,55 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
             for (int e = 0; e < 2; ++e) {          // elements (2e, 2e+1) of the chunk are k-slots (t, t+4)
                 const uint32_t ah[4] = {ka.h[2 * e], kb.h[2 * e], ka.h[2 * e + 1], kb.h[2 * e + 1]};
                 const uint32_t al[4] = {ka.l[2 * e], kb.l[2 * e], ka.l[2 * e + 1], kb.l[2 * e + 1]};
-                mma3(sh[e], sl[e], sm[e], ah, al, st.qh[j][2 * e], st.qh[j][2 * e + 1], st.ql[j][2 * e], st.ql[j][2 * e + 1]);
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt)
+                    mma3(sh[nt][e], sl[nt][e], sm[nt][e], ah, al, st.qh[nt][j][2 * e], st.qh[nt][j][2 * e + 1],
+                         st.ql[nt][j][2 * e], st.ql[nt][j][2 * e + 1]);
             }
         }
-        // this thread's scores: rows rowA (0,1) and rowB (2,3) of heads 2t (0,2) and 2t+1 (1,3)
-        float s[4];
+        float alpha[NT][2], p[NT][4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) s[i] = (sh[0][i] + sh[1][i]) + ((sl[0][i] + sl[1][i]) + (sm[0][i] + sm[1][i]));
-        if (!FULL) {
-            if (rowA >= nr) { s[0] = -INFINITY; s[1] = -INFINITY; }
-            if (rowB >= nr) { s[2] = -INFINITY; s[3] = -INFINITY; }
-        }
-        // online softmax per head (row maximum across the 8 lanes with the same t)
-        float alpha[2], p[4];
+        for (int nt = 0; nt < NT; ++nt) {
+            // this thread's scores: rows rowA (0,1) and rowB (2,3) of heads 8nt+2t (0,2) and 8nt+2t+1 (1,3)
+            float s[4];
 #pragma unroll
-        for (int i = 0; i < 2; ++i) {
-            float bm = fmaxf(s[i], s[i + 2]);
-            bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 4));
-            bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 8));
-            bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 16));
-            const float m_new = fmaxf(st.m_run[i], bm);
-            alpha[i] = exp2_diff(st.m_run[i], m_new);
-            p[i] = exp2_diff(s[i], m_new);
-            p[i + 2] = exp2_diff(s[i + 2], m_new);
-            st.l_run[i] = fmaf(st.l_run[i], alpha[i], p[i] + p[i + 2]);
-            st.m_run[i] = m_new;
+            for (int i = 0; i < 4; ++i)
+                s[i] = (sh[nt][0][i] + sh[nt][1][i]) + ((sl[nt][0][i] + sl[nt][1][i]) + (sm[nt][0][i] + sm[nt][1][i]));
+            if (!FULL) {
+                if (rowA >= nr) { s[0] = -INFINITY; s[1] = -INFINITY; }
+                if (rowB >= nr) { s[2] = -INFINITY; s[3] = -INFINITY; }
+            }
+            // online softmax per head (row maximum across the 8 lanes with the same t)
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                float bm = fmaxf(s[i], s[i + 2]);
+                bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 4));
+                bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 8));
+                bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 16));
+                const float m_new = fmaxf(st.m_run[2 * nt + i], bm);
+                alpha[nt][i] = exp2_diff(st.m_run[2 * nt + i], m_new);
+                p[nt][i] = exp2_diff(s[i], m_new);
+                p[nt][i + 2] = exp2_diff(s[i + 2], m_new);
+                st.l_run[2 * nt + i] = fmaf(st.l_run[2 * nt + i], alpha[nt][i], p[nt][i] + p[nt][i + 2]);
+                st.m_run[2 * nt + i] = m_new;
+            }
         }
         // P^T and the rescale factors go to the weighted-sum part through one of two buffers:
-        // lane (g, t) there fetches rows 2t, 2t+1, 2t+8, 2t+9 of head g (the rows whose V it
+        // lane (g, t) there fetches rows 2t, 2t+1, 2t+8, 2t+9 of a head (the rows whose V it
         // loads) with one 128-bit read
         const int b = k & 1, use = k >> 1;
         if (PAIRED && use >= 1 && !mbar_wait_bounded(bar_pfree0 + 8u * b, (uint32_t)(use - 1) & 1u)) return false;
         float *pt = my_pbuf + b * C::PBUF_FLOATS;
         const int pa = 4 * ((rowA >> 1) & 3) + (rowA & 1), pb = pa + 2;
-        pt[(2 * t) * PTS + pa] = p[0];
-        pt[(2 * t + 1) * PTS + pa] = p[1];
-        pt[(2 * t) * PTS + pb] = p[2];
-        pt[(2 * t + 1) * PTS + pb] = p[3];
-        if (g == 0) { pt[G * PTS + 2 * t] = alpha[0]; pt[G * PTS + 2 * t + 1] = alpha[1]; }
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            float *ph = pt + (8 * nt + 2 * t) * PTS;
+            ph[pa] = p[nt][0];
+            ph[PTS + pa] = p[nt][1];
+            ph[pb] = p[nt][2];
+            ph[PTS + pb] = p[nt][3];
+            if (g == 0) { pt[G * PTS + 8 * nt + 2 * t] = alpha[nt][0]; pt[G * PTS + 8 * nt + 2 * t + 1] = alpha[nt][1]; }
+        }
         __syncwarp();
         if (PAIRED && lane == 0) tc::mbar_arrive(bar_pfull0 + 8u * b);
         return true;
@@ -426,33 +451,42 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
 
     // ================= weighted-sum part: O^T += V_tile^T * P^T ================================
     // State: O^T fragments, features (by 16-feature tile) x heads 2t, 2t+1.
-    auto pv_begin = [&](PvState<MT> &st) {
+    auto pv_begin = [&](PvState<MT, NT> &st) {
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-            for (int i = 0; i < 4; ++i) st.om[mt][i] = 0.f;
+            for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) st.om[mt][nt][i] = 0.f;
     };
-    auto pv_publish = [&](const PvState<MT> &st) {
+    auto pv_publish = [&](const PvState<MT, NT> &st, int hb) {
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) {
             // output tile mt = 2u+e holds features 32u + 4g + 2e (+1) of heads 2t (+1)
             const int f = 32 * (mt >> 1) + 4 * g + 2 * (mt & 1);
-            float *o0 = merge_o + ((size_t)(pair * G + 2 * t)) * D + f;
-            o0[0] = st.om[mt][0]; o0[D] = st.om[mt][1]; o0[1] = st.om[mt][2]; o0[D + 1] = st.om[mt][3];
+            float *o0 = merge_o + ((size_t)(pair * 8 + 2 * t)) * D + f;
+            const float (&o)[4] = (NT == 2 && hb == 1) ? st.om[mt][NT - 1] : st.om[mt][0];
+            o0[0] = o[0]; o0[D] = o[1]; o0[1] = o[2]; o0[D + 1] = o[3];
         }
     };
-    auto pv_tile = [&](PvState<MT> &st, const float *sV, int nr, int k, auto full_tag) -> bool {
+    auto pv_tile = [&](PvState<MT, NT> &st, const float *sV, int nr, int k, auto full_tag) -> bool {
         constexpr bool FULL = decltype(full_tag)::value;
         const int b = k & 1, use = k >> 1;
         if (PAIRED && !mbar_test_wait(bar_pfull0 + 8u * b, (uint32_t)use & 1u) &&
             !mbar_wait_bounded(bar_pfull0 + 8u * b, (uint32_t)use & 1u)) return false;
         const float *pt = my_pbuf + b * C::PBUF_FLOATS;
-        const Split4 pp = split4(*reinterpret_cast<const float4 *>(pt + g * PTS + 4 * t));
-        const float alpha[2] = {pt[G * PTS + 2 * t], pt[G * PTS + 2 * t + 1]};
+        Split4 pp[NT];
+        float alpha[NT][2];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            pp[nt] = split4(*reinterpret_cast<const float4 *>(pt + (8 * nt + g) * PTS + 4 * t));
+            alpha[nt][0] = pt[G * PTS + 8 * nt + 2 * t];
+            alpha[nt][1] = pt[G * PTS + 8 * nt + 2 * t + 1];
+        }
         __syncwarp();
         if (PAIRED && lane == 0) tc::mbar_arrive(bar_pfree0 + 8u * b);
         // 16 features at a time; a tile's products start from zero and are then added to the
-        // running values, rescaled by alpha
+        // running values, rescaled by alpha; a V fragment is loaded and split once for all head tiles
 #pragma unroll
         for (int u = 0; u < NU; ++u) {
             Split4 v[4];
@@ -465,39 +499,47 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
             }
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
-                float oh[4] = {0.f, 0.f, 0.f, 0.f}, ol[4] = {0.f, 0.f, 0.f, 0.f}, ox[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-                for (int kp = 0; kp < 2; ++kp) {   // rows (2t+8kp, 2t+1+8kp) are k-slots (t, t+4)
-                    const uint32_t ah[4] = {v[2 * kp].h[2 * e], v[2 * kp].h[2 * e + 1], v[2 * kp + 1].h[2 * e],
-                                            v[2 * kp + 1].h[2 * e + 1]};
-                    const uint32_t al[4] = {v[2 * kp].l[2 * e], v[2 * kp].l[2 * e + 1], v[2 * kp + 1].l[2 * e],
-                                            v[2 * kp + 1].l[2 * e + 1]};
-                    mma3(oh, ol, ox, ah, al, pp.h[2 * kp], pp.h[2 * kp + 1], pp.l[2 * kp], pp.l[2 * kp + 1]);
-                }
                 const int mt = 2 * u + e;
+                uint32_t ah[2][4], al[2][4];       // rows (2t+8kp, 2t+1+8kp) are k-slots (t, t+4)
 #pragma unroll
-                for (int i = 0; i < 4; ++i) st.om[mt][i] = fmaf(st.om[mt][i], alpha[i & 1], oh[i] + (ol[i] + ox[i]));
+                for (int kp = 0; kp < 2; ++kp) {
+                    ah[kp][0] = v[2 * kp].h[2 * e]; ah[kp][1] = v[2 * kp].h[2 * e + 1];
+                    ah[kp][2] = v[2 * kp + 1].h[2 * e]; ah[kp][3] = v[2 * kp + 1].h[2 * e + 1];
+                    al[kp][0] = v[2 * kp].l[2 * e]; al[kp][1] = v[2 * kp].l[2 * e + 1];
+                    al[kp][2] = v[2 * kp + 1].l[2 * e]; al[kp][3] = v[2 * kp + 1].l[2 * e + 1];
+                }
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    float oh[4] = {0.f, 0.f, 0.f, 0.f}, ol[4] = {0.f, 0.f, 0.f, 0.f}, ox[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                    for (int kp = 0; kp < 2; ++kp)
+                        mma3(oh, ol, ox, ah[kp], al[kp], pp[nt].h[2 * kp], pp[nt].h[2 * kp + 1], pp[nt].l[2 * kp],
+                             pp[nt].l[2 * kp + 1]);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
+                        st.om[mt][nt][i] = fmaf(st.om[mt][nt][i], alpha[nt][i & 1], oh[i] + (ol[i] + ox[i]));
+                }
             }
         }
         return true;
     };
 
     if (!PAIRED) {
-        ScoreState<NJ> ss;
-        PvState<MT> ps;
-        run([&]() { score_begin(ss); pv_begin(ps); }, [&]() { score_publish(ss); pv_publish(ps); },
+        ScoreState<NJ, NT> ss;
+        PvState<MT, NT> ps;
+        run([&]() { score_begin(ss); pv_begin(ps); }, [&](int hb) { score_publish(ss, hb); pv_publish(ps, hb); },
             [&](const float *tile_base, int nr, int k, auto full_tag) -> bool {
                 return score_tile(ss, tile_base, nr, k, full_tag) && pv_tile(ps, tile_base + R * D, nr, k, full_tag);
             });
     } else if (!is_pv) {
-        ScoreState<NJ> ss;
-        run([&]() { score_begin(ss); }, [&]() { score_publish(ss); },
+        ScoreState<NJ, NT> ss;
+        run([&]() { score_begin(ss); }, [&](int hb) { score_publish(ss, hb); },
             [&](const float *tile_base, int nr, int k, auto full_tag) -> bool {
                 return score_tile(ss, tile_base, nr, k, full_tag);
             });
     } else {
-        PvState<MT> ps;
-        run([&]() { pv_begin(ps); }, [&]() { pv_publish(ps); },
+        PvState<MT, NT> ps;
+        run([&]() { pv_begin(ps); }, [&](int hb) { pv_publish(ps, hb); },
             [&](const float *tile_base, int nr, int k, auto full_tag) -> bool {
                 return pv_tile(ps, tile_base, nr, k, full_tag);
             });

@@ -104,6 +104,17 @@ def test_stream_kernel_any_cta_count_gives_the_same_answer(ctas):
     assert max_err(gpu_decode(q, K, V, s, num_ctas=ctas, expect_path=moa.PATH_MMA), ref) <= TOL
 
 
+def test_one_unit_split_across_more_ctas_than_one_merge_round_holds():
+    # a single (batch, kv head) unit cut into ~1000 partials: the CTA that delivers the last
+    # one merges them in several rounds of its staging buffer
+    q, K, V, s = make(81, 1, 4, 1, 16500, 128, 128)
+    ref = oracle.decode(q, K, V, s)
+    assert max_err(gpu_decode(q, K, V, s, num_ctas=1000, expect_path=moa.PATH_STREAM), ref) <= TOL
+    q, K, V, s = make(82, 1, 8, 1, 16500, 128, 128)
+    ref = oracle.decode(q, K, V, s)
+    assert max_err(gpu_decode(q, K, V, s, num_ctas=1000, expect_path=moa.PATH_MMA), ref) <= TOL
+
+
 # ---------------------------------------------------------------------------------------
 # grouped tensor-core kernel (g_s in {16, 32, 64}, d = 128, dense cache)
 # ---------------------------------------------------------------------------------------
