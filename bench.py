@@ -44,6 +44,7 @@ L2_BYTES_ASSUMED = 126 * 1024 * 1024
 NCU_TRAFFIC_BYTES = {
     "gqa": 1074650112 + 3750144,        # profiles/stream_decode_kernel_gqa.md (full-size launch)
     "mqa_long": 537828864 + 5385984,    # profiles/grouped_decode_kernel_mqa_long.md (full-size launch)
+    "extra_group8_d128": 1075588864 + 4157440,   # profiles/mma_decode_kernel_group8_d128.md (full-size launch)
 }
 
 
@@ -363,7 +364,7 @@ def run_reference(args, wname):
     if rank != 0:
         return
     import oracle
-    w = mi.WORKLOADS[wname]
+    w = mi.WORKLOADS[wname] if wname in mi.WORKLOADS else EXTRA_WORKLOADS[wname]
     if wname == "multi_step":
         w = mi.small_like(w, n=int(np.mean([w.len_lo, w.len_hi])) + w.steps // 2)
     total = args.steps + args.warmup
@@ -401,7 +402,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=list(mi.WORKLOADS))
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=list(mi.WORKLOADS) + list(EXTRA_WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-others", action="store_true", help="skip the timing-only lines of the other workloads")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
@@ -430,7 +431,7 @@ def main():
         _DIST["on"] = True
     moa.lib()                                           # fail loudly if the library is missing
 
-    w = mi.WORKLOADS[wname]
+    w = mi.WORKLOADS[wname] if wname in mi.WORKLOADS else EXTRA_WORKLOADS[wname]
     if args.batch > 0:
         w = mi.small_like(w, batch=args.batch)
     if args.n > 0 and wname != "multi_step":
@@ -464,8 +465,11 @@ def main():
         # launches, and no per-launch event overhead).  Otherwise: the bracketed figure.
         k_ms = ms if single_launch else kern_ms
         ach = decode_bytes / (k_ms * 1e-3) / 1e9
-        kname = "grouped_decode_kernel (tcgen05)" if w.group >= 16 and w.d_k == 128 and wname != "multi_step" else \
-            "stream_decode_kernel (scores, online softmax, weighted sum, append, partial merge)"
+        kname = {moa.PATH_GENERIC: "generic_decode_kernel",
+                 moa.PATH_STREAM: "stream_decode_kernel (FMA; scores, online softmax, weighted sum, append, partial merge)",
+                 moa.PATH_GROUPED: "grouped_decode_kernel (tcgen05)",
+                 moa.PATH_MMA: "mma_decode_kernel (warp-level TF32 MMA; scores, online softmax, weighted sum, append, "
+                               "partial merge)"}.get(moa.moa_last_path(), "?")
         roof = {"bound": "hbm", "kernel": kname, "achieved": ach, "peak": peak,
                 "peak_source": "of " + peak_kind, "unit": "GB/s", "frac": ach / peak,
                 "kernel_us_per_launch": k_ms * 1e3,
