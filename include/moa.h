@@ -79,6 +79,30 @@ int moa_decode_attn_varlen(const float *q, const float *K, const float *V, float
                            int n_max, int d_k, int d_v, float scale,
                            void *workspace, size_t workspace_bytes, void *stream);
 
+/*
+ * Sequence split across devices (the paper treats leading batch/head dimensions as
+ * independent outer indices, section 2; a split of the *sequence* axis is not in the paper
+ * and rests on the shift invariance of eq. (2), like the split inside one device).
+ *
+ * moa_decode_attn_partial: same arguments and layouts as moa_decode_attn, over the n rows
+ * this device holds, but instead of the normalised output it writes, per (batch, query
+ * head), the unnormalised triple
+ *     partial [batch, h_q, d_v + 4] :  o[d_v] = sum_l 2^(s2[l] - m) V[l,:],  m,  l = sum_l 2^(s2[l] - m),  2 pad
+ * with s2 = log2(e) * scale * <q, K[l,:]> and m a reference value >= every s2[l] seen
+ * (device memory, owned by the caller, 16-byte aligned when q/K/V are).
+ *
+ * moa_combine_partials: merges nparts such triples, laid out [nparts][batch][h_q][d_v+4]
+ * (e.g. the result of an all-gather), in part order, into out [batch, h_q, d_v]:
+ *     M = max_i m_i,  out = sum_i 2^(m_i - M) o_i / sum_i 2^(m_i - M) l_i.
+ * The result equals moa_decode_attn over the concatenated rows up to fp32 rounding.
+ * One kernel launch; device pointers; nothing is allocated.
+ */
+int moa_decode_attn_partial(const float *q, const float *K, const float *V, float *partial,
+                            int batch, int h_q, int h_kv, int n, int d_k, int d_v,
+                            float scale, void *stream);
+int moa_combine_partials(const float *partials, int nparts, float *out, int batch, int h_q,
+                         int d_v, void *stream);
+
 /* Workspace size in bytes that moa_decode_attn_varlen needs for these dimensions on the
  * current device (0 on invalid dimensions).  Host-only arithmetic plus one device
  * attribute query. */

@@ -42,6 +42,8 @@ def lib():
         L.moa_decode_attn.argtypes = [p, p, p, p, i, i, i, i, i, i, f, p]
         L.moa_decode_attn_noalloc.argtypes = [p, p, p, p, i, i, i, i, i, i, f, p]
         L.moa_decode_attn_varlen.argtypes = [p, p, p, p, i, i, i, p, i, i, i, f, p, sz, p]
+        L.moa_decode_attn_partial.argtypes = [p, p, p, p, i, i, i, i, i, i, f, p]
+        L.moa_combine_partials.argtypes = [p, i, p, i, i, i, p]
         L.moa_workspace_bytes.argtypes = [i, i, i, i, i, i]
         L.moa_workspace_bytes.restype = sz
         L.moa_kv_append.argtypes = [p, p, p, p, p, i, i, i, i, i, p]
@@ -111,6 +113,18 @@ def moa_decode_attn_varlen(q, K, V, out, batch, h_q, h_kv, seq_lens, n_max, d_k,
                                         _ptr(seq_lens), n_max, d_k, d_v, scale, _ptr(workspace),
                                         workspace_bytes, _stream(stream)),
            "moa_decode_attn_varlen")
+
+
+def moa_decode_attn_partial(q, K, V, partial, batch, h_q, h_kv, n, d_k, d_v, scale, stream=None):
+    """Unnormalised triples over this device's rows: partial [batch, h_q, d_v + 4]."""
+    _check(lib().moa_decode_attn_partial(_ptr(q), _ptr(K), _ptr(V), _ptr(partial), batch, h_q, h_kv, n,
+                                         d_k, d_v, scale, _stream(stream)), "moa_decode_attn_partial")
+
+
+def moa_combine_partials(partials, nparts, out, batch, h_q, d_v, stream=None):
+    """Merge [nparts, batch, h_q, d_v + 4] triples into out [batch, h_q, d_v]."""
+    _check(lib().moa_combine_partials(_ptr(partials), nparts, _ptr(out), batch, h_q, d_v, _stream(stream)),
+           "moa_combine_partials")
 
 
 def moa_workspace_bytes(batch, h_q, h_kv, n_max, d_k, d_v) -> int:

@@ -396,9 +396,10 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
                        int h_q, int h_kv, const int32_t *seq_lens, int len_bias, int n_max,
                        int d_k, int d_v, float scale, void *ws, size_t ws_bytes,
                        bool library_ws, cudaStream_t st, const FusedStep *fused = nullptr,
-                       bool allow_grouped = true)
+                       bool allow_grouped = true, float *partial_out = nullptr)
 {
-    if (!q || !K || !V || !out) return MOA_ERR_INVALID;
+    if (!q || !K || !V || (!out && !partial_out)) return MOA_ERR_INVALID;
+    if (partial_out != nullptr) out = partial_out;      // (alignment checks below apply to it)
     int rc = validate_dims(batch, h_q, h_kv, n_max, d_k, d_v);
     if (rc != MOA_OK) return rc;
     if (!isfinite(scale)) return MOA_ERR_INVALID;
@@ -443,6 +444,7 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
     a.qscale = scale * kLog2e;
     a.Kw = nullptr; a.Vw = nullptr; a.k_new = nullptr; a.v_new = nullptr; a.lens_rw = nullptr;
     a.tickets = nullptr;
+    a.partial_out = partial_out;
     if (fused != nullptr && path != MOA_PATH_STREAM && path != MOA_PATH_MMA) return MOA_ERR_UNSUPPORTED;
 
     cudaError_t e;
@@ -466,6 +468,7 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
         ga.h_kv_stored = h_kv; ga.share = gplan.share;
         ga.splits = gplan.splits; ga.tiles_per_split = gplan.tiles_per_split;
         ga.qscale = scale * kLog2e;
+        ga.partial_out = partial_out;
         const int grid = (int)(units * gplan.share * gplan.splits);
         if (gplan.GH == 16) e = launch_grouped_cfg<16>(mk, mv, ga, grid, st);
         else if (gplan.GH == 32) e = launch_grouped_cfg<32>(mk, mv, ga, grid, st);
@@ -564,6 +567,29 @@ int moa_decode_attn_noalloc(const float *q, const float *K, const float *V, floa
                      static_cast<cudaStream_t>(stream), nullptr, false);
     g_prof_on = prof_saved;
     return rc;
+}
+
+int moa_decode_attn_partial(const float *q, const float *K, const float *V, float *partial, int batch,
+                            int h_q, int h_kv, int n, int d_k, int d_v, float scale, void *stream)
+{
+    return decode_impl(q, K, V, nullptr, batch, h_q, h_kv, nullptr, 0, n, d_k, d_v, scale, nullptr, 0,
+                       true, static_cast<cudaStream_t>(stream), nullptr, true, partial);
+}
+
+int moa_combine_partials(const float *partials, int nparts, float *out, int batch, int h_q, int d_v,
+                         void *stream)
+{
+    if (!partials || !out || nparts < 1 || batch < 1 || h_q < 1 || d_v < 1) return MOA_ERR_INVALID;
+    if (d_v > MOA_MAX_DV) return MOA_ERR_UNSUPPORTED;
+    if (!aligned(partials, 4) || !aligned(out, 4)) return MOA_ERR_ALIGN;
+    const long long rows = (long long)batch * h_q;
+    if (rows > 0x7fffffffLL) return MOA_ERR_CAPACITY;
+    DeviceState *dev = nullptr;
+    int rc = current_device(&dev);
+    if (rc != MOA_OK) return rc;
+    combine_partials_kernel<<<(int)rows, 128, 0, static_cast<cudaStream_t>(stream)>>>(partials, nparts, out, rows, d_v);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? MOA_OK : MOA_ERR_CUDA;
 }
 
 int moa_decode_attn_varlen(const float *q, const float *K, const float *V, float *out, int batch,

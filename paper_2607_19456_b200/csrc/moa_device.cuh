@@ -127,7 +127,26 @@ struct DecodeArgs {
     int32_t *lens_rw;         // lengths advanced by one when the whole grid is done, or nullptr
     unsigned *tickets;        // completion counters (kTicketStride words, all zero between
                               // launches), or nullptr: partials are merged by a second kernel
+    float *partial_out;       // nullptr, or [batch, h_q, d_v + 4]: emit the unnormalised triple
+                              // (o[d_v], m, l, 2 pad) instead of the normalised output row
 };
+
+// Final emission of one float4 column group of a (batch, query head) row: the normalised
+// output, or -- for a caller that merges several row ranges itself (sequence split across
+// GPUs) -- the unnormalised weighted sum with its reference maximum (log2 domain) and sum.
+__device__ __forceinline__ void emit_columns(const DecodeArgs &a, size_t bh, int D, int d4, const float4 &acc,
+                                             float M, float L)
+{
+    if (a.partial_out != nullptr) {
+        float *dst = a.partial_out + bh * (size_t)(D + 4);
+        *reinterpret_cast<float4 *>(dst + d4 * 4) = acc;
+        if (d4 == 0) { dst[D] = M; dst[D + 1] = L; }
+    } else {
+        const float inv = 1.0f / L;
+        *reinterpret_cast<float4 *>(a.out + bh * (size_t)D + d4 * 4) =
+            make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+    }
+}
 
 // Completion counters of one launch: word c counts the CTAs that have delivered their
 // partial for the split unit whose first segment lies in CTA c; the last word counts CTAs
@@ -330,12 +349,7 @@ __device__ __forceinline__ void merge_unit_partials(const DecodeArgs &a, float *
         const int idx = tid + it * nthreads;
         if (idx < G * LPR) {
             const int hg = idx / LPR, d4 = idx % LPR;
-            if (hg < a.g_s) {
-                const float inv = 1.0f / L[it];
-                float *dst = a.out + ((size_t)b * a.h_q + (size_t)h * a.g_s + hg) * D + d4 * 4;
-                *reinterpret_cast<float4 *>(dst) =
-                    make_float4(acc[it].x * inv, acc[it].y * inv, acc[it].z * inv, acc[it].w * inv);
-            }
+            if (hg < a.g_s) emit_columns(a, (size_t)b * a.h_q + (size_t)h * a.g_s + hg, D, d4, acc[it], M[it], L[it]);
         }
     }
 }

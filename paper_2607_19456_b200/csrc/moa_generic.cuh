@@ -71,13 +71,38 @@ __global__ void __launch_bounds__(kGenericWarps * 32) generic_decode_kernel(cons
     float L = 0.f;
 #pragma unroll
     for (int w = 0; w < kGenericWarps; ++w) L = fmaf(sml[w * 2 + 1], exp2_diff(sml[w * 2], M), L);
-    float *og = a.out + ((size_t)b * a.h_q + g) * a.d_v;
+    const bool partial = a.partial_out != nullptr;
+    float *og = partial ? a.partial_out + ((size_t)b * a.h_q + g) * (size_t)(a.d_v + 4)
+                        : a.out + ((size_t)b * a.h_q + g) * a.d_v;
     for (int d = threadIdx.x; d < a.d_v; d += blockDim.x) {
         float acc = 0.f;
 #pragma unroll
         for (int w = 0; w < kGenericWarps; ++w)
             acc = fmaf(so[w * a.d_v + d], exp2_diff(sml[w * 2], M), acc);
-        og[d] = acc / L;
+        og[d] = partial ? acc : acc / L;
+    }
+    if (partial && threadIdx.x == 0) { og[a.d_v] = M; og[a.d_v + 1] = L; }
+}
+
+// Merge `nparts` unnormalised triples per (batch, query head) row -- the results of decode
+// calls over disjoint row ranges of the same sequences -- into the normalised output.
+// parts: [nparts][rows][d_v + 4] (o[d_v], m, l, 2 pad); merged in part order.  One block per row.
+__global__ void __launch_bounds__(128) combine_partials_kernel(const float *parts, int nparts, float *out,
+                                                               long long rows, int d_v)
+{
+    const long long r = blockIdx.x;
+    const size_t ps = (size_t)d_v + 4, part_stride = (size_t)rows * ps;
+    const float *base = parts + (size_t)r * ps;
+    float M = -INFINITY;
+    for (int i = 0; i < nparts; ++i) M = fmaxf(M, base[(size_t)i * part_stride + d_v]);
+    float L = 0.f;
+    for (int i = 0; i < nparts; ++i)
+        L = fmaf(base[(size_t)i * part_stride + d_v + 1], exp2_diff(base[(size_t)i * part_stride + d_v], M), L);
+    for (int d = threadIdx.x; d < d_v; d += blockDim.x) {
+        float acc = 0.f;
+        for (int i = 0; i < nparts; ++i)
+            acc = fmaf(base[(size_t)i * part_stride + d], exp2_diff(base[(size_t)i * part_stride + d_v], M), acc);
+        out[(size_t)r * d_v + d] = acc / L;
     }
 }
 

@@ -77,6 +77,7 @@ struct GroupedArgs {
     int splits;          // sequence splits per unit
     int tiles_per_split;
     float qscale;        // scale * log2(e)
+    float *partial_out;  // nullptr, or [batch, h_q, 132]: unnormalised triples instead of `out`
 };
 
 // Bounded mbarrier wait that also gives up when another role has already failed.
@@ -630,6 +631,12 @@ __global__ void __launch_bounds__(128) grouped_combine_kernel(const GroupedArgs 
             acc.x = fmaf(t.x, f, acc.x); acc.y = fmaf(t.y, f, acc.y);
             acc.z = fmaf(t.z, f, acc.z); acc.w = fmaf(t.w, f, acc.w);
         }
+    }
+    if (a.partial_out != nullptr) {
+        float *dst = a.partial_out + ((size_t)b * a.h_q + gq) * 132;
+        *reinterpret_cast<float4 *>(dst + lane * 4) = acc;
+        if (lane == 0) { dst[128] = M; dst[129] = L; }
+        return;
     }
     const float inv = 1.0f / L;
     *reinterpret_cast<float4 *>(a.out + ((size_t)b * a.h_q + gq) * 128 + lane * 4) =

@@ -259,11 +259,7 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
                     L = fmaf(merge_ml[(v * 8 + h8) * 2 + 1], f, L);
                 }
                 if (complete) {
-                    if (hg < a.g_s) {
-                        const float inv = 1.0f / L;
-                        float *dst = a.out + ((size_t)cc.b * a.h_q + (size_t)cc.h * a.g_s + hg) * D + d4 * 4;
-                        *reinterpret_cast<float4 *>(dst) = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
-                    }
+                    if (hg < a.g_s) emit_columns(a, (size_t)cc.b * a.h_q + (size_t)cc.h * a.g_s + hg, D, d4, acc, M, L);
                 } else {
                     const int slot = (seg_begin == c0) ? 0 : 1;
                     float *dst = a.ws + (((size_t)blockIdx.x * 2 + slot) * G + hg) * PS;

@@ -223,11 +223,7 @@ __global__ void __launch_bounds__(C::THREADS, 1) stream_decode_kernel(const Deco
                 L = fmaf(merge_ml[(v * G + g) * 2 + 1], f, L);
             }
             if (complete) {
-                if (g < a.g_s) {
-                    const float inv = 1.0f / L;
-                    float *dst = a.out + ((size_t)cc.b * a.h_q + (size_t)cc.h * a.g_s + g) * D + d4 * 4;
-                    *reinterpret_cast<float4 *>(dst) = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
-                }
+                if (g < a.g_s) emit_columns(a, (size_t)cc.b * a.h_q + (size_t)cc.h * a.g_s + g, D, d4, acc, M, L);
             } else {
                 const int slot = (seg_begin == c0) ? 0 : 1;
                 float *dst = a.ws + (((size_t)blockIdx.x * 2 + slot) * G + g) * PS;
@@ -421,11 +417,7 @@ __global__ void __launch_bounds__(128) stream_combine_kernel(const DecodeArgs a,
             acc.z = fmaf(t.z, f, acc.z); acc.w = fmaf(t.w, f, acc.w);
         }
     }
-    if (lane < LPR) {
-        const float inv = 1.0f / L;
-        float *dst = a.out + ((size_t)b * a.h_q + gq) * D + lane * 4;
-        *reinterpret_cast<float4 *>(dst) = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
-    }
+    if (lane < LPR) emit_columns(a, (size_t)b * a.h_q + gq, D, lane, acc, M, L);
 }
 
 }  // namespace moa

@@ -53,3 +53,63 @@ def barrier():
     import torch.distributed as dist
     if dist.is_available() and dist.is_initialized():
         dist.barrier()
+
+
+# ---- sequence split: one long sequence over several GPUs --------------------------------
+# Each rank holds a contiguous range of cached rows of every (batch, kv head) and computes
+# the unnormalised triple (o, m, l) over it (moa_decode_attn_partial); one all-gather of
+# batch * h_q * (d_v + 4) floats per rank is the only exchange, after which every rank
+# merges the triples in rank order (moa_combine_partials).  The exchange goes through the
+# process group (NCCL over NVLink on GPUs, gloo in CPU tests): remote triples land in local
+# memory first, no kernel reads a peer's memory.
+
+def shard_rows(n: int, world: int, rank: int, align: int = 16):
+    """Contiguous row range [start, start+count) owned by `rank` when n cached rows are cut
+    into `world` ranges whose sizes are multiples of `align` (except the last non-empty
+    one).  Ranks past the end of the sequence get count 0."""
+    if n < 0 or world < 1 or not (0 <= rank < world) or align < 1:
+        raise ValueError("bad shard arguments")
+    per = -(-n // world)
+    per = -(-per // align) * align
+    start = min(n, rank * per)
+    return start, min(n, start + per) - start
+
+
+def empty_partial(batch: int, h_q: int, d_v: int, like=None):
+    """The triple of an empty row range: o = 0, m = -inf, l = 0 (ignored by the merge)."""
+    import torch
+    t = torch.zeros((batch, h_q, d_v + 4), dtype=torch.float32,
+                    device=like.device if like is not None else "cpu")
+    t[:, :, d_v] = float("-inf")
+    return t
+
+
+def gather_partials(partial_local, group=None):
+    """All-gather the per-rank triples [batch, h_q, d_v+4] into [world, batch, h_q, d_v+4],
+    ordered by rank.  Without an initialised process group: a world of one."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return partial_local.unsqueeze(0).contiguous()
+    world = dist.get_world_size(group)
+    parts = [torch.empty_like(partial_local) for _ in range(world)]
+    dist.all_gather(parts, partial_local.contiguous(), group=group)
+    return torch.stack(parts, dim=0)
+
+
+def seq_split_decode(q, K_rows, V_rows, out, scale: float, group=None):
+    """Decode attention when every rank holds a row range of the same sequences.
+    q [batch, h_q, d_k] (replicated), K_rows / V_rows [batch, h_kv, n_local, d] on this
+    rank's GPU (n_local may be 0), out [batch, h_q, d_v] (every rank gets the result)."""
+    import paper_2607_19456_b200 as moa
+    batch, h_q, d_k = q.shape
+    h_kv, n_local, d_v = K_rows.shape[1], K_rows.shape[2], V_rows.shape[3]
+    if n_local > 0:
+        import torch
+        part = torch.empty((batch, h_q, d_v + 4), dtype=torch.float32, device=q.device)
+        moa.moa_decode_attn_partial(q, K_rows, V_rows, part, batch, h_q, h_kv, n_local, d_k, d_v, scale)
+    else:
+        part = empty_partial(batch, h_q, d_v, like=q)
+    parts = gather_partials(part, group)
+    moa.moa_combine_partials(parts, parts.shape[0], out, batch, h_q, d_v)
+    return out

@@ -81,3 +81,84 @@ def test_shard_batch_covers_the_batch_exactly_once():
             assert max(sizes) - min(sizes) <= 1
     with pytest.raises(ValueError):
         shard_batch(4, 2, 2)
+
+
+# ---- sequence split: every rank holds a row range, one all-gather of (o, m, l) triples ----
+def _numpy_partial(q, K, V, scale):
+    """Unnormalised triple over the given rows, in fp64, log2 domain (test code)."""
+    B, hq, _ = q.shape
+    hkv, n, dv = K.shape[1], K.shape[2], V.shape[3]
+    out = np.zeros((B, hq, dv + 4), np.float32)
+    out[:, :, dv] = -np.inf
+    if n == 0:
+        return out
+    gs = hq // hkv
+    for b in range(B):
+        for g in range(hq):
+            s2 = (K[b, g // gs].astype(np.float64) @ q[b, g].astype(np.float64)) * scale * np.log2(np.e)
+            m = s2.max()
+            w = np.exp2(s2 - m)
+            out[b, g, :dv] = w @ V[b, g // gs].astype(np.float64)
+            out[b, g, dv], out[b, g, dv + 1] = m, w.sum()
+    return out
+
+
+def _numpy_combine(parts, dv):
+    m = parts[..., dv].astype(np.float64)
+    M = m.max(axis=0)
+    f = np.where(np.isneginf(m), 0.0, np.exp2(m - M))
+    L = (parts[..., dv + 1] * f).sum(axis=0)
+    return ((parts[..., :dv] * f[..., None]).sum(axis=0) / L[..., None]).astype(np.float32)
+
+
+def _seq_worker(rank, world, port, n, q):
+    sys.path.insert(0, ROOT)
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        import moa_inputs as mi
+        from paper_2607_19456_b200 import shard
+        w = mi.Workload("sq", 91, 2, 8, 2, n, 16, 16)
+        qq, K, V = w.q(), w.K(), w.V()
+        start, count = shard.shard_rows(n, world, rank)
+        part = torch.from_numpy(_numpy_partial(qq, K[:, :, start:start + count], V[:, :, start:start + count], w.scale))
+        if count == 0:
+            assert torch.equal(part, shard.empty_partial(2, 8, 16))
+        parts = shard.gather_partials(part)
+        assert parts.shape == (world, 2, 8, 20)
+        assert torch.equal(parts[rank], part)          # rank order
+        if rank == 0:
+            q.put(_numpy_combine(parts.numpy(), 16))
+    finally:
+        dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("n", [100, 16, 5])
+def test_two_ranks_sequence_split(n):
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_seq_worker, args=(r, 2, port, n, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = q.get(timeout=120)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    sys.path.insert(0, ROOT)
+    import moa_inputs as mi
+    import oracle
+    w = mi.Workload("sq", 91, 2, 8, 2, n, 16, 16)
+    assert float(np.max(np.abs(got - oracle.decode(w.q(), w.K(), w.V(), w.scale)))) <= 1e-6
+
+
+def test_shard_rows_covers_the_sequence_exactly_once():
+    from paper_2607_19456_b200.shard import shard_rows
+    for n in (0, 1, 15, 16, 17, 100, 4096, 4097):
+        for world in (1, 2, 3, 8):
+            seen = []
+            for r in range(world):
+                s, c = shard_rows(n, world, r)
+                assert c >= 0 and (c % 16 == 0 or s + c == n)
+                seen += list(range(s, s + c))
+            assert seen == list(range(n))
