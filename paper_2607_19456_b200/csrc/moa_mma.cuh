@@ -374,13 +374,15 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
     };
     auto score_tile = [&](ScoreState<NJ, NT> &st, const float *sK, int nr, int k, auto full_tag) -> bool {
         constexpr bool FULL = decltype(full_tag)::value;
-        // 2*NJ k-steps, two accumulator chains for each of the three products of each head tile;
-        // a K fragment is loaded and split once and used for all head tiles
-        float sh[NT][2][4], sl[NT][2][4], sm[NT][2][4];
+        // 2*NJ k-steps; six independent accumulator chains in flight (three products x two chains
+        // for one head tile, three products x two head tiles otherwise); a K fragment is loaded
+        // and split once and used for all head tiles
+        constexpr int NCH = (NT == 1) ? 2 : 1;
+        float sh[NT][NCH][4], sl[NT][NCH][4], sm[NT][NCH][4];
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-            for (int c = 0; c < 2; ++c)
+            for (int c = 0; c < NCH; ++c)
 #pragma unroll
                 for (int i = 0; i < 4; ++i) { sh[nt][c][i] = 0.f; sl[nt][c][i] = 0.f; sm[nt][c][i] = 0.f; }
 #pragma unroll
@@ -393,8 +395,8 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
                 const uint32_t al[4] = {ka.l[2 * e], kb.l[2 * e], ka.l[2 * e + 1], kb.l[2 * e + 1]};
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt)
-                    mma3(sh[nt][e], sl[nt][e], sm[nt][e], ah, al, st.qh[nt][j][2 * e], st.qh[nt][j][2 * e + 1],
-                         st.ql[nt][j][2 * e], st.ql[nt][j][2 * e + 1]);
+                    mma3(sh[nt][e % NCH], sl[nt][e % NCH], sm[nt][e % NCH], ah, al, st.qh[nt][j][2 * e],
+                         st.qh[nt][j][2 * e + 1], st.ql[nt][j][2 * e], st.ql[nt][j][2 * e + 1]);
             }
         }
         float alpha[NT][2], p[NT][4];
@@ -403,8 +405,12 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
             // this thread's scores: rows rowA (0,1) and rowB (2,3) of heads 8nt+2t (0,2) and 8nt+2t+1 (1,3)
             float s[4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-                s[i] = (sh[nt][0][i] + sh[nt][1][i]) + ((sl[nt][0][i] + sl[nt][1][i]) + (sm[nt][0][i] + sm[nt][1][i]));
+            for (int i = 0; i < 4; ++i) {
+                if constexpr (NCH == 2)
+                    s[i] = (sh[nt][0][i] + sh[nt][1][i]) + ((sl[nt][0][i] + sl[nt][1][i]) + (sm[nt][0][i] + sm[nt][1][i]));
+                else
+                    s[i] = sh[nt][0][i] + (sl[nt][0][i] + sm[nt][0][i]);
+            }
             if (!FULL) {
                 if (rowA >= nr) { s[0] = -INFINITY; s[1] = -INFINITY; }
                 if (rowB >= nr) { s[2] = -INFINITY; s[3] = -INFINITY; }
