@@ -481,7 +481,7 @@ def main():
 
     # ---- end to end through the host-buffer entry point --------------------------------
     e2e = None
-    if wname != "multi_step" and run.host is not None:
+    if wname != "multi_step" and run.host is not None and args.e2e_steps > 0:
         run.e2e_step()                                   # warm-up: staging buffers are allocated here
         torch.cuda.synchronize()
         barrier()
