@@ -218,6 +218,17 @@ def test_varlen_matches_oracle(D, hq, hkv):
     assert max_err(gpu_decode(q, K, V, s, seq_lens=lens, path=moa.PATH_GENERIC), ref) <= TOL
 
 
+@pytest.mark.parametrize("hq,hkv,d", [(4, 2, 128), (8, 1, 64)])
+def test_varlen_batch_larger_than_the_shared_memory_prefix(hq, hkv, d):
+    # more than 1024 batch items: the kernels scan the lengths in global memory instead of
+    # keeping a block prefix in shared memory
+    B, n_max = 1100, 40
+    q, K, V, s = make(740 + d, B, hq, hkv, n_max, d, d)
+    lens = (1 + (np.arange(B) * 7) % n_max).astype(np.int32)
+    ref = oracle.decode_varlen(q, K, V, lens, s)
+    assert max_err(gpu_decode(q, K, V, s, seq_lens=lens), ref) <= TOL
+
+
 @pytest.mark.parametrize("path", [moa.PATH_AUTO, moa.PATH_GENERIC])
 def test_out_of_range_length_sets_status_and_skips_the_item(path):
     B, hq, hkv, n_max, D = 3, 4, 2, 64, 128
