@@ -472,6 +472,7 @@ def main():
                                "partial merge)"}.get(moa.moa_last_path(), "?")
         roof = {"bound": "hbm", "kernel": kname, "achieved": ach, "peak": peak,
                 "peak_source": "of " + peak_kind, "unit": "GB/s", "frac": ach / peak,
+                "frac_of_nominal_8000": ach / 8000.0,
                 "kernel_us_per_launch": k_ms * 1e3,
                 "how": ("CUDA events around the %d back-to-back launches of the timed region / launches" % launches)
                 if single_launch else "CUDA event pair around every launch of the kernel (second pass)",
@@ -547,7 +548,12 @@ def main():
                                "decode_kernel_us": okern * 1e3 if okern else None,
                                "decode_kernel_GBps": (odec / (okern * 1e-3) / 1e9) if okern else None,
                                "decode_kernel_frac_of_peak": (odec / (okern * 1e-3) / 1e9 / peak) if okern else None,
+                               "frac_of_nominal_8000": ob / (oms * 1e-3) / 1e9 / 8000.0,
                                "l2": r.l2_note})
+                if name == "single_head":              # latency-bound: also with its lines resident in L2
+                    r.nsets = 1
+                    wms, _, _, _ = time_steps(r, 200, 10)
+                    others[-1]["us_per_step_l2_warm"] = wms * 1e3
                 del r
                 torch.cuda.empty_cache()
             except Exception as ex:                     # a secondary line must not lose the main one
