@@ -7,9 +7,10 @@
 // flat list dealt to persistent CTAs in equal contiguous ranges, every warp owns a private
 // ring of shared-memory stages filled by bulk asynchronous copies, split units are merged
 // by the CTA that delivers the last partial.  What differs is the arithmetic of a tile, and
-// that warps work in pairs: one warp owns the K tiles (scores, online softmax), its partner
-// the V tiles (weighted sum); probabilities and rescale factors pass from one to the other
-// through a double-buffered shared-memory slot guarded by two mbarriers each way.
+// that (at d = 128) warps work in pairs: one warp owns the K tiles (scores, online softmax),
+// its partner the V tiles (weighted sum); probabilities and rescale factors pass from one to
+// the other through a double-buffered shared-memory slot guarded by two mbarriers each way.
+// At d = 64 one warp does both halves of a tile, one after the other.
 // With 8 query heads per fetched row the FMA kernel is bound by instruction issue, not by
 // HBM; here a warp computes
 //     S^T [16 rows x 8 heads]   = K_tile [16 x d]  * Q^T [d x 8]        (m16n8k8, TF32)
