@@ -233,7 +233,7 @@ const char *moa_strerror(int code);
 #define MOA_PATH_GENERIC   1   /* any d_k, d_v, alignment: one CTA per (batch, query head) */
 #define MOA_PATH_STREAM    2   /* split-sequence streaming kernel on the FMA units, d in {32,64,128} */
 #define MOA_PATH_GROUPED   3   /* tcgen05 tensor-core kernel for large groups (g_s in {16,32,64}, dense) */
-#define MOA_PATH_MMA       4   /* streaming kernel with warp-level MMA, groups of 8 or 16 heads, d in {64,128} */
+#define MOA_PATH_MMA       4   /* streaming kernel with warp-level MMA, groups of 8 or 16 heads, d_k, d_v in {64,128} */
 int moa_set_option(int option, int value);
 int moa_last_path(void);
 

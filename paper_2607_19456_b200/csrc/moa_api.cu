@@ -95,7 +95,8 @@ static int validate_dims(int batch, int h_q, int h_kv, int n, int d_k, int d_v)
 // ---- streaming-kernel plan -------------------------------------------------------------
 struct StreamPlan {
     bool ok = false;
-    int D = 0;       // feature size
+    int D = 0;       // feature size (d_v; equal to d_k except in `mixed` plans)
+    int Dk = 0;      // d_k
     int G = 0;       // heads per (virtual) kv head handled by one CTA pass
     int share = 1;   // virtual kv heads per physical kv head (g_s = share * G when g_s > 8)
     int R = 0;       // rows per block of the chosen configuration
@@ -130,7 +131,21 @@ static bool mma_allowed() { return g_force_path != MOA_PATH_STREAM; }
 static StreamPlan plan_stream(int g_s, int d_k, int d_v)
 {
     StreamPlan p;
-    if (d_k != d_v || (d_k != 32 && d_k != 64 && d_k != 128)) return p;
+    p.Dk = d_k;
+    if (d_k != d_v) {
+        // Unequal row lengths: only the paired mode of the warp-MMA kernel handles them (every
+        // warp owns one operand), in groups of 8 heads.
+        if (!mma_allowed() || (d_k != 64 && d_k != 128) || (d_v != 64 && d_v != 128)) return p;
+        if (g_s > 8 && g_s % 8 != 0) return p;
+        p.D = d_v;
+        p.G = 8;
+        p.share = g_s > 8 ? g_s / 8 : 1;
+        p.mma = true;
+        p.R = 16;
+        p.ok = true;
+        return p;
+    }
+    if (d_k != 32 && d_k != 64 && d_k != 128) return p;
     p.D = d_k;
     p.G = stream_group(g_s, &p.share);
     p.mma = mma_allowed() && p.G == 8 && p.D >= 64;     // (the caller drops it for huge caches)
@@ -193,7 +208,7 @@ static cudaError_t launch_mma_cfg(const DecodeArgs &a, int num_ctas, cudaStream_
     // The caches as [d/32 column groups][rows][32 floats]: one box is a 16-row tile.
     const long long rows_total = (long long)a.batch * (a.h_kv / a.kv_share) * a.n_max;
     CUtensorMap mk, mv;
-    if (!make_rows_map(&mk, a.K, rows_total, C::D) || !make_rows_map(&mv, a.V, rows_total, C::D))
+    if (!make_rows_map(&mk, a.K, rows_total, C::DK) || !make_rows_map(&mv, a.V, rows_total, C::DV))
         return cudaErrorInvalidValue;
     static bool attr_set[kMaxDevices] = {};
     int dev = 0;
@@ -221,10 +236,14 @@ static cudaError_t launch_stream(const StreamPlan &p, const DecodeArgs &a, int n
                                  cudaStream_t st)
 {
     if (p.mma) {                         //                                     D   S  P  paired
-        if (p.D == 128 && p.G == 16) return launch_mma_cfg<MmaCfg<128, 3, 4, true, 2>>(a, num_ctas, st);
-        if (p.D == 128) return launch_mma_cfg<MmaCfg<128, 3, 4, true, 1>>(a, num_ctas, st);
-        if (p.G == 16) return launch_mma_cfg<MmaCfg<64, 2, 8, false, 2>>(a, num_ctas, st);
-        return launch_mma_cfg<MmaCfg<64, 2, 8, false, 1>>(a, num_ctas, st);
+        if (p.Dk != p.D) {               //                     d_k  d_v  S  P  paired NT
+            if (p.Dk == 128) return launch_mma_cfg<MmaCfg<128, 64, 3, 4, true, 1>>(a, num_ctas, st);
+            return launch_mma_cfg<MmaCfg<64, 128, 3, 4, true, 1>>(a, num_ctas, st);
+        }
+        if (p.D == 128 && p.G == 16) return launch_mma_cfg<MmaCfg<128, 128, 3, 4, true, 2>>(a, num_ctas, st);
+        if (p.D == 128) return launch_mma_cfg<MmaCfg<128, 128, 3, 4, true, 1>>(a, num_ctas, st);
+        if (p.G == 16) return launch_mma_cfg<MmaCfg<64, 64, 2, 8, false, 2>>(a, num_ctas, st);
+        return launch_mma_cfg<MmaCfg<64, 64, 2, 8, false, 1>>(a, num_ctas, st);
     }
     // The heavier configurations (many FMAs per fetched byte) run 16 warps per CTA: with
     // eight, two warps per scheduler cannot hide the shuffle and FMA latencies.  The lightest
@@ -417,6 +436,7 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
     StreamPlan plan = plan_stream(g_s, d_k, d_v);
     if (plan.mma && (long long)batch * h_kv * n_max > 0x7fffff00LL) {   // row coordinates are 32-bit
         plan.mma = false;
+        plan.ok = (d_k == d_v);
         plan.G = stream_group(g_s, &plan.share);
         plan.R = rows_per_block(plan.D, plan.G);
     }

@@ -44,9 +44,10 @@
 
 namespace moa {
 
-template <int D_, int S_, int P_, bool PAIRED_, int NT_>
+template <int DK_, int DV_, int S_, int P_, bool PAIRED_, int NT_>
 struct MmaCfg {
-    static constexpr int D = D_;              // d_k == d_v
+    static constexpr int DK = DK_, DV = DV_;  // they may differ in paired mode (each warp owns one operand)
+    static constexpr int D = DV;              // output row length (partials, merge buffers)
     static constexpr int NT = NT_;            // 8-head column tiles of the score matrix
     static constexpr int G = 8 * NT;          // query heads per (virtual) kv head
     static constexpr int S = S_;              // ring stages per warp
@@ -54,17 +55,19 @@ struct MmaCfg {
     static constexpr int P = P_;              // independent tile streams (pairs or single warps) per CTA
     static constexpr int W = PAIRED ? 2 * P : P;   // warps per CTA
     static constexpr int R = 16;              // rows per tile
-    static constexpr int LPR = D / 4;         // float4 per row
-    static constexpr int NJ = D / 16;         // K chunks a lane reads per row (2 k-steps each)
-    static constexpr int NU = D / 32;         // V chunks a lane reads per row (2 feature tiles each)
-    static constexpr int MT = D / 16;         // 16-feature output tiles
+    static constexpr int LPR = DV / 4;        // float4 per output row
+    static constexpr int NJ = DK / 16;        // K chunks a lane reads per row (2 k-steps each)
+    static constexpr int NU = DV / 32;        // V chunks a lane reads per row (2 feature tiles each)
+    static constexpr int MT = DV / 16;        // 16-feature output tiles
+    static constexpr int DMAX = DK > DV ? DK : DV;
     static constexpr int SUBT = R * 32;       // floats of one [16 rows][32 floats] sub-tile
-    static constexpr int STAGE_FLOATS = PAIRED ? R * D : 2 * R * D;   // one operand's tile / K tile + V tile
+    static constexpr int STAGE_FLOATS = PAIRED ? R * DMAX : 2 * R * D;   // one operand's tile / K tile + V tile
     static constexpr int PT_STRIDE = 20;      // floats between heads in a P^T hand-over buffer
     static constexpr int PBUF_FLOATS = G * PT_STRIDE + G;   // P^T [8 heads][16 rows] + alpha [8 heads]
     static constexpr int PS = D + 4;          // floats per partial: o[D], m, l, 2 pad
     static constexpr int THREADS = W * 32;
-    static_assert(D == 64 || D == 128, "row must be 256 or 512 bytes");
+    static_assert((DK == 64 || DK == 128) && (DV == 64 || DV == 128), "rows must be 256 or 512 bytes");
+    static_assert(PAIRED || DK == DV, "one warp per tile handles equal row lengths only");
     static_assert(NT == 1 || NT == 2, "8 or 16 heads");
     static_assert(G * LPR <= 4 * THREADS, "merge_unit_partials handles four items per thread");
     static_assert((STAGE_FLOATS * 4) % 1024 == 0, "swizzled sub-tiles need 1024-byte alignment");
@@ -130,7 +133,7 @@ template <class C>
 __global__ void __launch_bounds__(C::THREADS, 1)
 mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant__ CUtensorMap tmapV, const DecodeArgs a)
 {
-    constexpr int D = C::D, G = C::G, NT = C::NT, S = C::S, P = C::P, R = C::R, LPR = C::LPR, NJ = C::NJ, NU = C::NU,
+    constexpr int D = C::D, DK = C::DK, G = C::G, NT = C::NT, S = C::S, P = C::P, R = C::R, LPR = C::LPR, NJ = C::NJ, NU = C::NU,
                   MT = C::MT, SUBT = C::SUBT, PS = C::PS, PTS = C::PT_STRIDE;
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     unsigned char *const smem_m = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -179,6 +182,7 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
     float *my_pbuf = pbuf_all + (size_t)pair * 2 * C::PBUF_FLOATS;
     const uint32_t bar_pfull0 = smem_u32(&bars[C::W * S + 4 * pair]), bar_pfree0 = bar_pfull0 + 16u;
     const CUtensorMap *my_map = is_pv ? &tmapV : &tmapK;
+    const int my_d = is_pv ? D : DK;            // row length of this warp's operand
     const float *my_new = is_pv ? a.v_new : a.k_new;
     float *my_cache = is_pv ? a.Vw : a.Kw;
 
@@ -207,16 +211,16 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
             // A box is always transferred whole (rows past the end of the cache read as zero;
             // rows past the end of the unit belong to the next unit and are masked later).
             const uint32_t dst = smem_u32(my_ring + (size_t)stage * C::STAGE_FLOATS);
-            mbar_expect_tx(bar, (uint32_t)C::STAGE_FLOATS * 4u);
+            mbar_expect_tx(bar, PAIRED ? (uint32_t)R * my_d * 4u : (uint32_t)C::STAGE_FLOATS * 4u);
             tc::tma_load_3d(dst, my_map, 0, (int)row, 0, bar);
             if (!PAIRED) tc::tma_load_3d(dst + R * D * 4u, &tmapV, 0, (int)row, 0, bar);
         }
         // Fused append: the unit's last row is the token being appended.  The warp that fetches
         // the tile holding it also stores it into the cache (K by the score warp, V by the other);
         // the tile's copy of that row is replaced from k_new / v_new before use.
-        if (writes_new && row0 + R >= lc.len && lane < LPR) {
-            const size_t dst = (slab * (size_t)a.n_max + (size_t)(lc.len - 1)) * D + lane * 4;
-            *reinterpret_cast<float4 *>(my_cache + dst) = *reinterpret_cast<const float4 *>(my_new + slab * D + lane * 4);
+        if (writes_new && row0 + R >= lc.len && lane * 4 < my_d) {
+            const size_t dst = (slab * (size_t)a.n_max + (size_t)(lc.len - 1)) * my_d + lane * 4;
+            *reinterpret_cast<float4 *>(my_cache + dst) = *reinterpret_cast<const float4 *>(my_new + slab * my_d + lane * 4);
             if (!PAIRED)
                 *reinterpret_cast<float4 *>(a.Vw + dst) = *reinterpret_cast<const float4 *>(a.v_new + slab * D + lane * 4);
         }
@@ -313,10 +317,10 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
                 float *tile_base = my_ring + (size_t)stage * C::STAGE_FLOATS;
                 if ((a.k_new != nullptr) && (row0 + nr == cc.len)) {
                     // the appended token is this tile's last row: take it from k_new / v_new
-                    if (lane < LPR) {
+                    if (lane * 4 < my_d) {
                         const size_t cslab = (size_t)cc.b * h_stored + cc.h / a.kv_share;
                         *reinterpret_cast<float4 *>(tile_base + chunk_at(nr - 1, lane)) =
-                            *reinterpret_cast<const float4 *>(my_new + cslab * D + lane * 4);
+                            *reinterpret_cast<const float4 *>(my_new + cslab * my_d + lane * 4);
                         if (!PAIRED)
                             *reinterpret_cast<float4 *>(tile_base + R * D + chunk_at(nr - 1, lane)) =
                                 *reinterpret_cast<const float4 *>(a.v_new + cslab * D + lane * 4);
@@ -343,14 +347,14 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
     // State: Q^T fragments of head g (chunk t+4j of the scaled query row, split), running
     // maximum and this thread's share of the sum for heads 2t and 2t+1.
     auto score_begin = [&](ScoreState<NJ, NT> &st) {
-        const float *qb = a.q + ((size_t)cc.b * a.h_q + (size_t)cc.h * a.g_s) * D;
+        const float *qb = a.q + ((size_t)cc.b * a.h_q + (size_t)cc.h * a.g_s) * DK;
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
             const int hg = 8 * nt + g;
 #pragma unroll
             for (int j = 0; j < NJ; ++j) {
                 float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (hg < a.g_s) v = *reinterpret_cast<const float4 *>(qb + (size_t)hg * D + (t + 4 * j) * 4);
+                if (hg < a.g_s) v = *reinterpret_cast<const float4 *>(qb + (size_t)hg * DK + (t + 4 * j) * 4);
                 const Split4 s = split4(make_float4(v.x * a.qscale, v.y * a.qscale, v.z * a.qscale, v.w * a.qscale));
 #pragma unroll
                 for (int i = 0; i < 4; ++i) { st.qh[nt][j][i] = s.h[i]; st.ql[nt][j][i] = s.l[i]; }

@@ -115,6 +115,21 @@ def test_one_unit_split_across_more_ctas_than_one_merge_round_holds():
     assert max_err(gpu_decode(q, K, V, s, num_ctas=1000, expect_path=moa.PATH_MMA), ref) <= TOL
 
 
+@pytest.mark.parametrize("dk,dv", [(128, 64), (64, 128)])
+@pytest.mark.parametrize("gs", [1, 4, 8, 16])
+def test_unequal_key_and_value_row_lengths_on_the_fast_path(dk, dv, gs):
+    # d_k != d_v: the paired warp-MMA kernel (one warp per operand) takes them
+    hkv = 2
+    for n in (1, 17, 700, 3001):
+        q, K, V, s = make(4000 + dk + gs + n, 2, gs * hkv, hkv, n, dk, dv)
+        ref = oracle.decode(q, K, V, s)
+        assert max_err(gpu_decode(q, K, V, s, expect_path=moa.PATH_MMA), ref) <= TOL, (dk, dv, gs, n)
+    lens = np.array([3001, 5], np.int32)
+    assert max_err(gpu_decode(q, K, V, s, seq_lens=lens, expect_path=moa.PATH_MMA),
+                   oracle.decode_varlen(q, K, V, lens, s)) <= TOL
+    assert max_err(gpu_decode(q, K, V, s, path=moa.PATH_GENERIC), ref) <= TOL
+
+
 # ---------------------------------------------------------------------------------------
 # grouped tensor-core kernel (g_s in {16, 32, 64}, d = 128, dense cache)
 # ---------------------------------------------------------------------------------------
@@ -297,9 +312,11 @@ def test_append_out_of_range_position_is_skipped_and_reported():
 # multi-step decode: append then attend, token by token
 # ---------------------------------------------------------------------------------------
 @pytest.mark.parametrize("fused", [True, False])
-@pytest.mark.parametrize("D,hq,hkv", [(128, 8, 2), (64, 2, 1), (32, 8, 1), (16, 4, 4), (128, 8, 1), (64, 32, 2)])
+@pytest.mark.parametrize("D,hq,hkv", [(128, 8, 2), (64, 2, 1), (32, 8, 1), (16, 4, 4), (128, 8, 1), (64, 32, 2), ((128, 64), 8, 2),
+                                       ((64, 128), 4, 1)])
 def test_multistep_small(fused, D, hq, hkv):
-    w = mi.Workload("ms", 950 + D, 4, hq, hkv, 80, D, D, steps=40, len_lo=1, len_hi=40)
+    D, Dv = D if isinstance(D, tuple) else (D, D)
+    w = mi.Workload("ms", 950 + D + Dv, 4, hq, hkv, 80, D, Dv, steps=40, len_lo=1, len_hi=40)
     B, n_max = w.batch, w.n
     lens = w.start_lens()
     K, V = w.K(), w.V()
@@ -307,19 +324,19 @@ def test_multistep_small(fused, D, hq, hkv):
         K[b, :, lens[b]:] = 0
         V[b, :, lens[b]:] = 0
     gK, gV, glens = Guarded(K), Guarded(V), Guarded(lens)
-    gws, nbytes = workspace_for(B, hq, hkv, n_max, D, D)
-    gout = Guarded(shape=(B, hq, D))
+    gws, nbytes = workspace_for(B, hq, hkv, n_max, D, Dv)
+    gout = Guarded(shape=(B, hq, Dv))
     for t in range(w.steps):
         kn, vn, qt = w.k_new(t), w.v_new(t), w.q_step(t)
         gk, gv, gq = Guarded(kn), Guarded(vn), Guarded(qt)
         if fused:
             moa.moa_decode_step(gq.ptr, gK.ptr, gV.ptr, gk.ptr, gv.ptr, gout.ptr, glens.ptr, B, hq, hkv,
-                                n_max, D, D, w.scale, gws.ptr, nbytes)
+                                n_max, D, Dv, w.scale, gws.ptr, nbytes)
         else:
-            moa.moa_kv_append(gK.ptr, gV.ptr, gk.ptr, gv.ptr, glens.ptr, B, hkv, n_max, D, D)
+            moa.moa_kv_append(gK.ptr, gV.ptr, gk.ptr, gv.ptr, glens.ptr, B, hkv, n_max, D, Dv)
             moa.moa_lens_add(glens.ptr, B, 1)
             moa.moa_decode_attn_varlen(gq.ptr, gK.ptr, gV.ptr, gout.ptr, B, hq, hkv, glens.ptr, n_max,
-                                       D, D, w.scale, gws.ptr, nbytes)
+                                       D, Dv, w.scale, gws.ptr, nbytes)
         oracle.kv_append(K, V, kn, vn, lens)
         lens = lens + 1
         ref = oracle.decode_varlen(qt, K, V, lens, w.scale)
