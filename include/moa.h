@@ -133,8 +133,8 @@ int moa_lens_add(int32_t *lens, int batch, int delta, void *stream);
  * lens is a device int32[batch] that the call updates; all other arguments as above.
  * Requires lens[b] in [0, n_max-1]; otherwise the status bits above are set, the item
  * is skipped and its length is left unchanged.
- * For d_k == d_v in {32, 64, 128} and 16-byte-aligned pointers all three parts run in one
- * kernel launch (the streaming kernel takes the new row from k_new/v_new, stores it into
+ * For d_k == d_v in {32, 64, 128} (or d_k != d_v, both in {64, 128}) and 16-byte-aligned
+ * pointers all three parts run in one kernel launch (the streaming kernel takes the new row from k_new/v_new, stores it into
  * the cache, and the last CTA to finish advances the lengths); otherwise in three.
  * `workspace` as for moa_decode_attn_varlen.
  * The call allocates nothing and needs no host round trip, so a sequence of steps can be
