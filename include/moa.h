@@ -80,6 +80,18 @@ int moa_decode_attn_varlen(const float *q, const float *K, const float *V, float
                            void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * The same decode for `layers` independent caches of one shape (the per-token accounting of
+ * the paper's introduction counts one such call per transformer layer): q, K, V, out are
+ * HOST arrays of `layers` device pointers, each with the layout of moa_decode_attn.  The
+ * launches go to `stream` back to back; the first error is returned and later layers are
+ * not launched.  (In a real model the layers of one token depend on each other; this entry
+ * point is for measuring the attention traffic of a whole token in one call.)
+ */
+int moa_decode_attn_layers(const float *const *q, const float *const *K, const float *const *V,
+                           float *const *out, int layers, int batch, int h_q, int h_kv, int n,
+                           int d_k, int d_v, float scale, void *stream);
+
+/*
  * Sequence split across devices (the paper treats leading batch/head dimensions as
  * independent outer indices, section 2; a split of the *sequence* axis is not in the paper
  * and rests on the shift invariance of eq. (2), like the split inside one device).

@@ -44,6 +44,7 @@ def lib():
         L.moa_decode_attn_varlen.argtypes = [p, p, p, p, i, i, i, p, i, i, i, f, p, sz, p]
         L.moa_decode_attn_partial.argtypes = [p, p, p, p, i, i, i, i, i, i, f, p]
         L.moa_combine_partials.argtypes = [p, i, p, i, i, i, p]
+        L.moa_decode_attn_layers.argtypes = [p, p, p, p, i, i, i, i, i, i, i, f, p]
         L.moa_workspace_bytes.argtypes = [i, i, i, i, i, i]
         L.moa_workspace_bytes.restype = sz
         L.moa_kv_append.argtypes = [p, p, p, p, p, i, i, i, i, i, p]
@@ -125,6 +126,14 @@ def moa_combine_partials(partials, nparts, out, batch, h_q, d_v, stream=None):
     """Merge [nparts, batch, h_q, d_v + 4] triples into out [batch, h_q, d_v]."""
     _check(lib().moa_combine_partials(_ptr(partials), nparts, _ptr(out), batch, h_q, d_v, _stream(stream)),
            "moa_combine_partials")
+
+
+def moa_decode_attn_layers(q, K, V, out, batch, h_q, h_kv, n, d_k, d_v, scale, stream=None):
+    """q, K, V, out: sequences (one entry per layer) of tensors / addresses of one shape."""
+    layers = len(q)
+    arr = [(C.c_void_p * layers)(*[_ptr(x) for x in seq]) for seq in (q, K, V, out)]
+    _check(lib().moa_decode_attn_layers(arr[0], arr[1], arr[2], arr[3], layers, batch, h_q, h_kv, n, d_k, d_v,
+                                        scale, _stream(stream)), "moa_decode_attn_layers")
 
 
 def moa_workspace_bytes(batch, h_q, h_kv, n_max, d_k, d_v) -> int:

@@ -591,6 +591,19 @@ int moa_decode_attn_noalloc(const float *q, const float *K, const float *V, floa
     return rc;
 }
 
+int moa_decode_attn_layers(const float *const *q, const float *const *K, const float *const *V, float *const *out,
+                           int layers, int batch, int h_q, int h_kv, int n, int d_k, int d_v, float scale,
+                           void *stream)
+{
+    if (!q || !K || !V || !out || layers < 1) return MOA_ERR_INVALID;
+    for (int l = 0; l < layers; ++l) {
+        const int rc = decode_impl(q[l], K[l], V[l], out[l], batch, h_q, h_kv, nullptr, 0, n, d_k, d_v, scale,
+                                   nullptr, 0, true, static_cast<cudaStream_t>(stream));
+        if (rc != MOA_OK) return rc;
+    }
+    return MOA_OK;
+}
+
 int moa_decode_attn_partial(const float *q, const float *K, const float *V, float *partial, int batch,
                             int h_q, int h_kv, int n, int d_k, int d_v, float scale, void *stream)
 {

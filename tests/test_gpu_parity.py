@@ -403,6 +403,21 @@ def test_fused_step_at_capacity_skips_and_keeps_length():
 # ---------------------------------------------------------------------------------------
 # argument errors never launch anything
 # ---------------------------------------------------------------------------------------
+def test_layers_call_runs_every_layer():
+    L, B, hq, hkv, n, d = 3, 2, 8, 2, 500, 128
+    layers = [make(6000 + l, B, hq, hkv, n, d, d) for l in range(L)]
+    dq = [torch.from_numpy(x[0]).cuda() for x in layers]
+    dK = [torch.from_numpy(x[1]).cuda() for x in layers]
+    dV = [torch.from_numpy(x[2]).cuda() for x in layers]
+    outs = [torch.full((B, hq, d), float("nan"), device="cuda") for _ in range(L)]
+    moa.moa_decode_attn_layers(dq, dK, dV, outs, B, hq, hkv, n, d, d, layers[0][3])
+    torch.cuda.synchronize()
+    assert moa.moa_device_status() == 0
+    for l in range(L):
+        q, K, V, s = layers[l]
+        assert max_err(outs[l].cpu().numpy(), oracle.decode(q, K, V, s)) <= TOL
+
+
 def test_argument_errors():
     q, K, V, s = make(970, 1, 4, 2, 16, 128, 128)
     gq, gK, gV = Guarded(q), Guarded(K), Guarded(V)
