@@ -4,6 +4,7 @@
 #include <math.h>
 #include <stdint.h>
 #include <type_traits>
+#include <utility>
 
 #include "moa.h"
 #include "moa_device.cuh"
@@ -61,6 +62,25 @@ struct TimedLaunch {                      // RAII: event before / after the domi
     }
 };
 static inline void count_launch(int n = 1) { if (g_prof_on) g_prof_all += n; }
+
+// Launch with programmatic stream serialisation: the kernel may start while its predecessor
+// in the stream is still running and synchronises with it on the device (griddepcontrol.wait).
+template <class... KArgs, class... Args>
+static cudaError_t launch_dependent(void (*kernel)(KArgs...), int grid, int threads, size_t smem, cudaStream_t st,
+                                    Args &&...args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)threads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
 
 static int current_device(DeviceState **st)
 {
@@ -188,7 +208,7 @@ static cudaError_t launch_stream_cfg(const DecodeArgs &a, int num_ctas, cudaStre
     }
     {
         TimedLaunch t(st);
-        stream_decode_kernel<C><<<num_ctas, C::THREADS, C::SMEM_BYTES, st>>>(a);
+        launch_dependent(stream_decode_kernel<C>, num_ctas, C::THREADS, C::SMEM_BYTES, st, a);
     }
     count_launch();
     cudaError_t e = cudaGetLastError();
@@ -221,7 +241,7 @@ static cudaError_t launch_mma_cfg(const DecodeArgs &a, int num_ctas, cudaStream_
     }
     {
         TimedLaunch t(st);
-        mma_decode_kernel<C><<<num_ctas, C::THREADS, C::SMEM_BYTES, st>>>(mk, mv, a);
+        launch_dependent(mma_decode_kernel<C>, num_ctas, C::THREADS, C::SMEM_BYTES, st, mk, mv, a);
     }
     count_launch();
     cudaError_t e = cudaGetLastError();

@@ -67,6 +67,15 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
+// ---- programmatic dependent launch ------------------------------------------------------
+// The streaming kernels are launched so that the next kernel in the stream may be scheduled
+// while this one is still running (its CTAs take the SMs that this kernel's CTAs leave).
+// launch_dependents allows that; grid_dependency_wait blocks until the previous kernel in
+// the stream has completed and its writes are visible, and is placed before the first read
+// of anything that kernel may have written.  Both are no-ops for an ordinary launch.
+__device__ __forceinline__ void launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // Every spin in this library is bounded: after kWaitLimit unsuccessful polls the caller
 // gives up, raises MOA_STATUS_WAIT_TIMEOUT and leaves without touching the data.
 constexpr uint32_t kWaitLimit = 1u << 22;

@@ -160,9 +160,11 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
     const int rowA = (g >> 1) + 4 * (g & 1), rowB = rowA + 8;
     const int h_stored = a.h_kv / a.kv_share;
 
+    launch_dependents();
     if (tid < C::NBAR) mbar_init(smem_u32(&bars[tid]), 1);
     if (tid == 0) { tc::prefetch_tmap(&tmapK); tc::prefetch_tmap(&tmapV); }
     mbar_fence_init();
+    grid_dependency_wait();                   // lengths, cache rows, counters, partial slots of the previous step
     __syncthreads();
 
     const int *pref = nullptr;

@@ -108,8 +108,10 @@ __global__ void __launch_bounds__(C::THREADS, 1) stream_decode_kernel(const Deco
     const bool owner = (lane % LPR) < NV;     // first copy of the value inside the row group
     const int h_stored = a.h_kv / a.kv_share; // K/V heads as stored
 
+    launch_dependents();
     if (tid < W * S) mbar_init(smem_u32(&bars[tid]), 1);
     mbar_fence_init();
+    grid_dependency_wait();                   // lengths, cache rows, counters, partial slots of the previous step
     __syncthreads();
 
     const int *pref = nullptr;
