@@ -400,7 +400,7 @@ def run_reference(args, wname):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--steps", type=int, default=500)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=list(mi.WORKLOADS) + list(EXTRA_WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])

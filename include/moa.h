@@ -237,11 +237,14 @@ const char *moa_strerror(int code);
  *   MOA_OPT_NUM_CTAS   : 0 = one streaming CTA per SM, otherwise that many.
  *   MOA_OPT_GROUPED_HEADS : query heads per CTA of the tensor-core kernel (16, 32 or 64;
  *                        0 = automatic).  Larger groups are cut into neighbouring CTAs.
+ *   MOA_OPT_DEPENDENT_LAUNCH : 1 (default) = the streaming kernels are launched with
+ *                        programmatic stream serialisation, 0 = ordinary launches.
  * moa_last_path() reports which kernel family the last successful decode call used.
  */
 #define MOA_OPT_FORCE_PATH 1
 #define MOA_OPT_NUM_CTAS   2
 #define MOA_OPT_GROUPED_HEADS 3
+#define MOA_OPT_DEPENDENT_LAUNCH 4
 #define MOA_PATH_GENERIC   1   /* any d_k, d_v, alignment: one CTA per (batch, query head) */
 #define MOA_PATH_STREAM    2   /* split-sequence streaming kernel on the FMA units, d in {32,64,128} */
 #define MOA_PATH_GROUPED   3   /* tcgen05 tensor-core kernel for large groups (g_s in {16,32,64}, dense) */

@@ -63,6 +63,8 @@ struct TimedLaunch {                      // RAII: event before / after the domi
 };
 static inline void count_launch(int n = 1) { if (g_prof_on) g_prof_all += n; }
 
+static int g_dependent_launch = 1;   // MOA_OPT_DEPENDENT_LAUNCH
+
 // Launch with programmatic stream serialisation: the kernel may start while its predecessor
 // in the stream is still running and synchronises with it on the device (griddepcontrol.wait).
 template <class... KArgs, class... Args>
@@ -78,7 +80,7 @@ static cudaError_t launch_dependent(void (*kernel)(KArgs...), int grid, int thre
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = g_dependent_launch ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
@@ -879,6 +881,11 @@ int moa_set_option(int option, int value)
     if (option == MOA_OPT_GROUPED_HEADS) {
         if (value != 0 && value != 16 && value != 32 && value != 64) return MOA_ERR_INVALID;
         g_grouped_heads = value;
+        return MOA_OK;
+    }
+    if (option == MOA_OPT_DEPENDENT_LAUNCH) {
+        if (value != 0 && value != 1) return MOA_ERR_INVALID;
+        g_dependent_launch = value;
         return MOA_OK;
     }
     if (option == MOA_OPT_NUM_CTAS) {
