@@ -21,7 +21,12 @@ def run_dense_on_gpu(w):
     out = torch.full((w.batch, w.h_q, w.d_v), float("nan"), device="cuda")
     moa.moa_decode_attn(dq, dK, dV, out, w.batch, w.h_q, w.h_kv, w.n, w.d_k, w.d_v, w.scale)
     torch.cuda.synchronize()
-    assert moa.moa_last_path() == (moa.PATH_GROUPED if w.group >= 16 and w.d_k == 128 else moa.PATH_STREAM)
+    want = moa.PATH_STREAM
+    if w.group >= 32 and w.d_k == 128:
+        want = moa.PATH_GROUPED
+    elif w.group % 8 == 0 and w.d_k >= 64:
+        want = moa.PATH_MMA
+    assert moa.moa_last_path() == want
     assert moa.moa_device_status() == 0
     res = out.cpu().numpy()
     del dq, dK, dV, out
@@ -59,6 +64,17 @@ def test_dense_configs_full_size_sampled(name, count):
     q, res = run_dense_on_gpu(w)
     assert np.all(np.isfinite(res))
     assert check_units(w, q, res, sample_units(w, count, 5)) <= TOL
+
+
+@pytest.mark.parametrize("name,count", [("extra_group8_d128", 6), ("extra_group8_d64", 6), ("extra_group16_d128", 6),
+                                        ("extra_mha_d32", 12)])
+def test_extra_bench_shapes_full_size_sampled(name, count):
+    # the timing-only shapes of bench.py (warp-MMA kernel at 8 and 16 heads per row, d = 32)
+    import bench
+    w = bench.EXTRA_WORKLOADS[name]
+    q, res = run_dense_on_gpu(w)
+    assert np.all(np.isfinite(res))
+    assert check_units(w, q, res, sample_units(w, count, 6)) <= TOL
 
 
 def test_config5_multi_step_full():
