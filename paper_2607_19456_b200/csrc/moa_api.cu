@@ -306,7 +306,9 @@ struct GroupedPlan {
     int GH = 0;          // query heads per CTA (per virtual kv head)
     int share = 1;       // virtual kv heads per stored kv head
     int splits = 1, tiles_per_split = 1;
-    size_t ws_bytes = 0;
+    size_t ws_bytes = 0;        // partial slots
+    size_t tail_bytes = 0;      // scratch copies of every unit's last tile (ragged caches, fused step)
+    size_t ws_ragged() const { return (ws_bytes + 255) / 256 * 256 + tail_bytes; }
 };
 static int g_grouped_heads = 0;   // MOA_OPT_GROUPED_HEADS: 0 = automatic
 
@@ -333,6 +335,7 @@ static GroupedPlan plan_grouped(const DeviceState &s, int batch, int h_q, int h_
     p.splits = (int)splits;
     p.tiles_per_split = (tiles + p.splits - 1) / p.splits;
     p.ws_bytes = (size_t)units * p.share * p.splits * p.GH * 132 * sizeof(float);
+    p.tail_bytes = (size_t)units * 2 * 128 * 128 * sizeof(float);
     p.ok = true;
     return p;
 }
@@ -388,8 +391,8 @@ static bool make_rows_map(CUtensorMap *m, const float *base, long long rows_tota
 }
 
 template <int GH>
-static cudaError_t launch_grouped_cfg(const CUtensorMap &mk, const CUtensorMap &mv, const GroupedArgs &ga,
-                                      int grid, cudaStream_t st)
+static cudaError_t launch_grouped_cfg(const CUtensorMap &mk, const CUtensorMap &mv, const CUtensorMap &mkt,
+                                      const CUtensorMap &mvt, const GroupedArgs &ga, int grid, cudaStream_t st)
 {
     using C = GroupedCfg<GH>;
     static bool attr_set[kMaxDevices] = {};
@@ -403,7 +406,7 @@ static cudaError_t launch_grouped_cfg(const CUtensorMap &mk, const CUtensorMap &
     }
     {
         TimedLaunch t(st);
-        grouped_decode_kernel<C><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(mk, mv, ga);
+        grouped_decode_kernel<C><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(mk, mv, mkt, mvt, ga);
     }
     count_launch();
     cudaError_t e = cudaGetLastError();
@@ -468,11 +471,17 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
     }
     const bool fast_ok = plan.ok && aligned(q, 16) && aligned(K, 16) && aligned(V, 16) && aligned(out, 16);
     int path = fast_ok ? (plan.mma ? MOA_PATH_MMA : MOA_PATH_STREAM) : MOA_PATH_GENERIC;
-    // Large head groups over a dense cache go to the tensor cores.
+    // Large head groups go to the tcgen05 kernel; ragged caches and the fused step need scratch
+    // for the zero-padded copy of every unit's last tile on top of the partial slots.
     GroupedPlan gplan;
-    if (fast_ok && allow_grouped && fused == nullptr && seq_lens == nullptr)
+    const bool ragged = (seq_lens != nullptr) || (fused != nullptr);
+    if (fast_ok && allow_grouped && (fused == nullptr || (aligned(fused->k_new, 16) && aligned(fused->v_new, 16))))
         gplan = plan_grouped(*dev, batch, h_q, h_kv, n_max, d_k, d_v);
-    if (gplan.ok && (library_ws || (ws && ws_bytes >= gplan.ws_bytes))) path = MOA_PATH_GROUPED;
+    if (gplan.ok && ragged && (library_ws || seq_lens == nullptr)) gplan.ok = false;
+    // With per-sequence lengths this kernel's fixed (unit, split) grid is unbalanced; it still
+    // wins clearly for groups of 64, for 32 the flat decomposition of the warp-MMA kernel does.
+    if (gplan.ok && ragged && g_s != 64 && g_force_path != MOA_PATH_GROUPED) gplan.ok = false;
+    if (gplan.ok && (library_ws || (ws && ws_bytes >= (ragged ? gplan.ws_ragged() : gplan.ws_bytes)))) path = MOA_PATH_GROUPED;
     if (g_force_path == MOA_PATH_GENERIC) path = MOA_PATH_GENERIC;
     else if (g_force_path == MOA_PATH_STREAM) {
         if (!fast_ok) return MOA_ERR_UNSUPPORTED;
@@ -493,7 +502,7 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
     a.Kw = nullptr; a.Vw = nullptr; a.k_new = nullptr; a.v_new = nullptr; a.lens_rw = nullptr;
     a.tickets = nullptr;
     a.partial_out = partial_out;
-    if (fused != nullptr && path != MOA_PATH_STREAM && path != MOA_PATH_MMA) return MOA_ERR_UNSUPPORTED;
+    if (fused != nullptr && path == MOA_PATH_GENERIC) return MOA_ERR_UNSUPPORTED;
 
     cudaError_t e;
     if (path == MOA_PATH_GROUPED) {
@@ -517,10 +526,32 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
         ga.splits = gplan.splits; ga.tiles_per_split = gplan.tiles_per_split;
         ga.qscale = scale * kLog2e;
         ga.partial_out = partial_out;
+        ga.seq_lens = seq_lens; ga.len_bias = len_bias;
+        ga.tailK = nullptr; ga.tailV = nullptr;
+        CUtensorMap mkt = mk, mvt = mv;
+        if (ragged) {
+            // the last, partly filled tile of every unit, zero-padded (and the appended row of
+            // the fused step, which this kernel also stores into the cache)
+            ga.tailK = reinterpret_cast<float *>(static_cast<unsigned char *>(ws) + (gplan.ws_bytes + 255) / 256 * 256);
+            ga.tailV = ga.tailK + (size_t)units * 128 * 128;
+            if (!make_cache_map(&mkt, ga.tailK, units, 128, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
+                !make_cache_map(&mvt, ga.tailV, units, 128, 32, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B))
+                return MOA_ERR_CUDA;
+            grouped_tail_kernel<<<(int)units, 256, 0, st>>>(ga, K, V, fused ? fused->Kw : nullptr,
+                                                            fused ? fused->Vw : nullptr, fused ? fused->k_new : nullptr,
+                                                            fused ? fused->v_new : nullptr);
+            count_launch();
+            if (cudaGetLastError() != cudaSuccess) return MOA_ERR_CUDA;
+        }
         const int grid = (int)(units * gplan.share * gplan.splits);
-        if (gplan.GH == 16) e = launch_grouped_cfg<16>(mk, mv, ga, grid, st);
-        else if (gplan.GH == 32) e = launch_grouped_cfg<32>(mk, mv, ga, grid, st);
-        else e = launch_grouped_cfg<64>(mk, mv, ga, grid, st);
+        if (gplan.GH == 16) e = launch_grouped_cfg<16>(mk, mv, mkt, mvt, ga, grid, st);
+        else if (gplan.GH == 32) e = launch_grouped_cfg<32>(mk, mv, mkt, mvt, ga, grid, st);
+        else e = launch_grouped_cfg<64>(mk, mv, mkt, mvt, ga, grid, st);
+        if (e == cudaSuccess && fused != nullptr && fused->lens_rw != nullptr) {
+            lens_add_kernel<<<(batch + 127) / 128, 128, 0, st>>>(fused->lens_rw, batch, 1, n_max);
+            count_launch();
+            e = cudaGetLastError();
+        }
     } else if (path == MOA_PATH_STREAM || path == MOA_PATH_MMA) {
         const int num_ctas = stream_grid(*dev, plan, batch, h_kv, n_max);
         const size_t need = stream_ws_bytes(plan, num_ctas);
@@ -673,7 +704,7 @@ size_t moa_workspace_bytes(int batch, int h_q, int h_kv, int n_max, int d_k, int
     size_t need = stream_ws_bytes(plan, ctas);
     if (dev != nullptr || current_device(&dev) == MOA_OK) {
         const GroupedPlan gp = plan_grouped(*dev, batch, h_q, h_kv, n_max, d_k, d_v);
-        if (gp.ok && gp.ws_bytes > need) need = gp.ws_bytes;
+        if (gp.ok && gp.ws_ragged() > need) need = gp.ws_ragged();
     }
     return (need + 255) / 256 * 256;
 }

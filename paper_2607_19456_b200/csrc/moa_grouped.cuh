@@ -78,7 +78,60 @@ struct GroupedArgs {
     int tiles_per_split;
     float qscale;        // scale * log2(e)
     float *partial_out;  // nullptr, or [batch, h_q, 132]: unnormalised triples instead of `out`
+    // ---- ragged caches and the fused step (all null / zero for a dense decode) ----
+    const int32_t *seq_lens;   // device [batch] or nullptr: sequence b has seq_lens[b] + len_bias rows (n = capacity)
+    int len_bias;
+    float *tailK, *tailV;      // [stored units][128][128]: zero-padded copy of every unit's last tile, or nullptr
 };
+
+// Rows of sequence b as this kernel family sees them; 0 for an out-of-range length.
+__device__ __forceinline__ int grouped_len(const GroupedArgs &a, int b)
+{
+    if (a.seq_lens == nullptr) return a.n;
+    const int len = a.seq_lens[b] + a.len_bias;
+    return (len >= 1 && len <= a.n) ? len : 0;
+}
+
+// Ragged caches: rows past a sequence's length hold arbitrary bits (possibly NaN), and a zero
+// probability does not neutralise them inside a tensor-core product.  So the last, partly
+// filled tile of every unit is first copied into a scratch tile with its unused rows zeroed,
+// and the main kernel fetches that tile from there.  For the fused step the row being
+// appended (the unit's last row) is taken from k_new / v_new and also stored into the cache
+// (eqs. (4),(5)).  One block per stored (batch, kv head); the tile is 128 rows of 128 floats.
+__global__ void __launch_bounds__(256) grouped_tail_kernel(const GroupedArgs a, const float *K, const float *V, float *Kw,
+                                                           float *Vw, const float *k_new, const float *v_new)
+{
+    const int unit = blockIdx.x, b = unit / a.h_kv_stored;
+    const int len = grouped_len(a, b);
+    if (len == 0) {
+        if (threadIdx.x == 0 && (unit % a.h_kv_stored) == 0)
+            raise_status(MOA_STATUS_SEQLEN_RANGE | (k_new != nullptr ? MOA_STATUS_APPEND_RANGE : 0));
+        return;
+    }
+    const int row0 = ((len - 1) / 128) * 128, valid = len - row0;
+    const float4 *srcK = reinterpret_cast<const float4 *>(K + ((size_t)unit * a.n + row0) * 128);
+    const float4 *srcV = reinterpret_cast<const float4 *>(V + ((size_t)unit * a.n + row0) * 128);
+    float4 *dstK = reinterpret_cast<float4 *>(a.tailK + (size_t)unit * 128 * 128);
+    float4 *dstV = reinterpret_cast<float4 *>(a.tailV + (size_t)unit * 128 * 128);
+    const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int i = threadIdx.x; i < 128 * 32; i += blockDim.x) {
+        const int r = i >> 5, c = i & 31;
+        float4 k = zero, v = zero;
+        if (r < valid) {
+            if (k_new != nullptr && r == valid - 1) {
+                k = reinterpret_cast<const float4 *>(k_new + (size_t)unit * 128)[c];
+                v = reinterpret_cast<const float4 *>(v_new + (size_t)unit * 128)[c];
+                reinterpret_cast<float4 *>(Kw + ((size_t)unit * a.n + row0) * 128)[i] = k;
+                reinterpret_cast<float4 *>(Vw + ((size_t)unit * a.n + row0) * 128)[i] = v;
+            } else {
+                k = srcK[i];
+                v = srcV[i];
+            }
+        }
+        dstK[i] = k;
+        dstV[i] = v;
+    }
+}
 
 // Bounded mbarrier wait that also gives up when another role has already failed.
 __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int *abort_flag)
@@ -149,6 +202,7 @@ struct ChunkSeq {
 template <class C>
 __global__ void __launch_bounds__(C::THREADS, 1)
 grouped_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant__ CUtensorMap tmapV,
+                      const __grid_constant__ CUtensorMap tmapKt, const __grid_constant__ CUtensorMap tmapVt,
                       const GroupedArgs a)
 {
     constexpr int GH = C::GH, N1 = C::N1, NBUF = C::NBUF, PS = C::PS;
@@ -186,11 +240,15 @@ grouped_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_co
     const int sunit = blockIdx.x / (a.share * a.splits);          // stored (batch, kv head)
     const int b = sunit / a.h_kv_stored, h = (sunit % a.h_kv_stored) * a.share + sub;   // virtual head
     const int unit = sunit;                                         // tensor-map coordinate
-    const int tiles_total = (a.n + C::TILE - 1) / C::TILE;
-    const int tile0 = split * a.tiles_per_split;
+    const int len_b = grouped_len(a, b);           // 0: out-of-range length, the item is skipped
+    const int tiles_total = (len_b + C::TILE - 1) / C::TILE;
+    const int tiles_per_split = a.seq_lens ? (tiles_total + a.splits - 1) / a.splits : a.tiles_per_split;
+    const int tile0 = split * tiles_per_split;
     int T = tiles_total - tile0;
-    if (T > a.tiles_per_split) T = a.tiles_per_split;
+    if (T > tiles_per_split) T = tiles_per_split;
     if (T <= 0) return;                            // an empty split (uniform for the CTA)
+    // the unit's last tile comes from the zero-padded scratch copy when there is one
+    const int tail_t = (a.tailK != nullptr) ? tiles_total - 1 - tile0 : -1;
 
     // ---- set-up --------------------------------------------------------------------------
     if (tid == 0) {
@@ -209,6 +267,7 @@ grouped_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_co
         *acc_flag = 0u;
         tc::prefetch_tmap(&tmapK);
         tc::prefetch_tmap(&tmapV);
+        if (a.tailK != nullptr) { tc::prefetch_tmap(&tmapKt); tc::prefetch_tmap(&tmapVt); }
     }
     if (warp == 1) tc::tmem_alloc(smem_u32(tmem_slot), 512);
     // Q operand: rows 0..GH-1 hold hi(q*qscale), rows GH..2GH-1 the lo parts; K-major, 4
@@ -244,12 +303,13 @@ grouped_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_co
                 const uint32_t dst = sRing + (uint32_t)buf * C::CHUNK;
                 const uint32_t fb = bar_full(s.is_k, buf);
                 mbar_expect_tx(fb, C::CHUNK);
-                const int row = row_base + s.t * C::TILE;
+                const bool tail = (s.t == tail_t);
+                const int row = tail ? 0 : row_base + s.t * C::TILE;
                 if (s.is_k) {
-                    tc::tma_load_3d(dst, &tmapK, 32 * s.c, row, unit, fb);
+                    tc::tma_load_3d(dst, tail ? &tmapKt : &tmapK, 32 * s.c, row, unit, fb);
                 } else {
                     for (int dg = 0; dg < 4; ++dg)
-                        tc::tma_load_3d(dst + dg * 4096, &tmapV, 32 * dg, row + 32 * s.c, unit, fb);
+                        tc::tma_load_3d(dst + dg * 4096, tail ? &tmapVt : &tmapV, 32 * dg, row + 32 * s.c, unit, fb);
                 }
             }
         }
@@ -408,7 +468,7 @@ grouped_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_co
             ok = ok && wait_or_abort(bar_sfull(sb), (uint32_t)(t >> 1) & 1u, abort_flag);
             if (named_or(1, NS, !ok)) { ok = false; break; }     // leave together or not at all
             tc::fence_after_sync();
-            const bool valid = (row_base + t * C::TILE + row_in_tile) < a.n;
+            const bool valid = (row_base + t * C::TILE + row_in_tile) < len_b;
             // scores of this row against the current references; probabilities are formed at
             // once (they are only wrong if the reference has to be raised, which is rare)
             float vmax = -INFINITY;
@@ -603,8 +663,14 @@ __global__ void __launch_bounds__(128) grouped_combine_kernel(const GroupedArgs 
     const int b = (int)(wid / a.h_q), gq = (int)(wid % a.h_q);
     const int h = gq / GH, g = gq % GH;
     const int unit = b * a.h_kv + h;
-    const int tiles_total = (a.n + 127) / 128;
-    const int used = (tiles_total + a.tiles_per_split - 1) / a.tiles_per_split;   // non-empty splits
+    const int len_b = grouped_len(a, b);
+    if (len_b == 0) {                              // out-of-range length: report, leave out untouched
+        if (gq == 0 && lane == 0) raise_status(MOA_STATUS_SEQLEN_RANGE);
+        return;
+    }
+    const int tiles_total = (len_b + 127) / 128;
+    const int tiles_per_split = a.seq_lens ? (tiles_total + a.splits - 1) / a.splits : a.tiles_per_split;
+    const int used = (tiles_total + tiles_per_split - 1) / tiles_per_split;   // non-empty splits
     const float *base = a.ws + ((size_t)unit * a.splits * GH + g) * PS;
     const size_t stride = (size_t)GH * PS;
     float M = -INFINITY;

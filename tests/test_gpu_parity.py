@@ -244,9 +244,28 @@ def test_varlen_batch_larger_than_the_shared_memory_prefix(hq, hkv, d):
     assert max_err(gpu_decode(q, K, V, s, seq_lens=lens), ref) <= TOL
 
 
-@pytest.mark.parametrize("path", [moa.PATH_AUTO, moa.PATH_GENERIC])
-def test_out_of_range_length_sets_status_and_skips_the_item(path):
-    B, hq, hkv, n_max, D = 3, 4, 2, 64, 128
+@pytest.mark.parametrize("hq,hkv,d,want", [(8, 2, 128, moa.PATH_STREAM), (16, 2, 128, moa.PATH_MMA), (128, 2, 128, moa.PATH_GROUPED),
+                                           (64, 1, 128, moa.PATH_GROUPED), (32, 1, 128, moa.PATH_MMA), (6, 3, 40, moa.PATH_GENERIC)])
+def test_rows_past_the_length_may_hold_anything(hq, hkv, d, want):
+    # rows >= seq_lens[b] of a pre-allocated cache are never part of the result, whatever bits
+    # they hold (NaN here): a zero probability would not neutralise them inside a product
+    B, n_max = 4, 700
+    q, K, V, s = make(760 + hq + d, B, hq, hkv, n_max, d, d)
+    lens = np.array([1, 700, 129, 333], np.int32)
+    ref = oracle.decode_varlen(q, K, V, lens, s)
+    for b in range(B):
+        K[b, :, lens[b]:] = np.nan
+        V[b, :, lens[b]:] = np.nan
+    out = gpu_decode(q, K, V, s, seq_lens=lens, expect_path=want)
+    assert np.all(np.isfinite(out)) and max_err(out, ref) <= TOL
+    if hq // hkv == 32:                       # the tcgen05 kernel takes ragged groups of 32 only when forced
+        out = gpu_decode(q, K, V, s, seq_lens=lens, path=moa.PATH_GROUPED, expect_path=moa.PATH_GROUPED)
+        assert np.all(np.isfinite(out)) and max_err(out, ref) <= TOL
+
+
+@pytest.mark.parametrize("path,hq", [(moa.PATH_AUTO, 4), (moa.PATH_GENERIC, 4), (moa.PATH_AUTO, 16), (moa.PATH_AUTO, 128)])
+def test_out_of_range_length_sets_status_and_skips_the_item(path, hq):
+    B, hkv, n_max, D = 3, 2, 64, 128          # hq = 4: FMA kernel, 16: warp-MMA kernel, 128: tcgen05 kernel
     q, K, V, s = make(800, B, hq, hkv, n_max, D, D)
     lens = np.array([10, 0, 65], np.int32)
     gq, gK, gV = Guarded(q), Guarded(K), Guarded(V)
@@ -313,7 +332,7 @@ def test_append_out_of_range_position_is_skipped_and_reported():
 # ---------------------------------------------------------------------------------------
 @pytest.mark.parametrize("fused", [True, False])
 @pytest.mark.parametrize("D,hq,hkv", [(128, 8, 2), (64, 2, 1), (32, 8, 1), (16, 4, 4), (128, 8, 1), (64, 32, 2), ((128, 64), 8, 2),
-                                       ((64, 128), 4, 1)])
+                                       ((64, 128), 4, 1), (128, 64, 1), (128, 64, 2)])
 def test_multistep_small(fused, D, hq, hkv):
     D, Dv = D if isinstance(D, tuple) else (D, D)
     w = mi.Workload("ms", 950 + D + Dv, 4, hq, hkv, 80, D, Dv, steps=40, len_lo=1, len_hi=40)
@@ -350,7 +369,7 @@ def test_multistep_small(fused, D, hq, hkv):
 
 
 @pytest.mark.parametrize("ctas,misalign_new", [(0, 0), (4000, 0), (0, 1), (5, 0)])
-@pytest.mark.parametrize("D,hq,hkv", [(128, 32, 8), (64, 16, 1), (128, 6, 2), (32, 2, 2), (128, 16, 2)])
+@pytest.mark.parametrize("D,hq,hkv", [(128, 32, 8), (64, 16, 1), (128, 6, 2), (32, 2, 2), (128, 16, 2), (128, 64, 1)])
 def test_append_decode_single_call(ctas, misalign_new, D, hq, hkv):
     # one call appends at pos[b] and attends over pos[b]+1 rows; lengths are not modified.
     # ctas=4000 and a k_new that is only 4-byte aligned take the three-launch fallback.
