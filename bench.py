@@ -204,14 +204,8 @@ class DenseRun:
         q, K, V, out = self.ptrs[self.i % self.nsets]
         kn, vn, pos = self.aux
         self.i += 1
-        if w.group >= 16:
-            # large head groups: the tensor-core kernel serves dense caches through
-            # moa_decode_attn, so the step is an append launch followed by the decode launches
-            m.moa_kv_append(K, V, kn, vn, pos, w.batch, w.h_kv, w.n, w.d_k, w.d_v, self.stream)
-            m.moa_decode_attn(q, K, V, out, w.batch, w.h_q, w.h_kv, w.n, w.d_k, w.d_v, w.scale, self.stream)
-        else:
-            m.moa_append_decode(q, K, V, kn, vn, out, pos, w.batch, w.h_q, w.h_kv, w.n, w.d_k, w.d_v, w.scale,
-                                self.wsptr, self.ws_bytes, self.stream)
+        m.moa_append_decode(q, K, V, kn, vn, out, pos, w.batch, w.h_q, w.h_kv, w.n, w.d_k, w.d_v, w.scale,
+                            self.wsptr, self.ws_bytes, self.stream)
 
     def reset(self):
         self.i = 0
@@ -565,7 +559,9 @@ def main():
                 "vs_baseline": None, "dtype": "f32", "data": "synthetic",
                 "config": {"workload": wname, "batch_per_gpu": w.batch, "h_q": w.h_q, "h_kv": w.h_kv,
                            "n": w.n, "d_k": w.d_k, "d_v": w.d_v, "parallelism": "dp%d (batch-sharded, no collective)" % world,
-                           "step": "moa_append_decode: kv append at row n-1 + decode attention over n rows, one launch" if wname != "multi_step" else "moa_decode_step: append + attend over ragged lengths + length advance, one launch",
+                           "step": ("moa_decode_step: append + attend over ragged lengths + length advance, one launch" if wname == "multi_step"
+                                    else "moa_append_decode: kv append at row n-1 + decode attention over n rows, %d launch(es) per step"
+                                    % max(1, launches // max(1, args.steps))),
                            "l2": l2_note},
                 "us_per_step": ms * 1e3, "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
                 "roofline": roof, "cpu_baseline": cpu, "parity_max_abs_err_vs_oracle": parity,

@@ -537,7 +537,7 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
             if (!make_cache_map(&mkt, ga.tailK, units, 128, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
                 !make_cache_map(&mvt, ga.tailV, units, 128, 32, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B))
                 return MOA_ERR_CUDA;
-            grouped_tail_kernel<<<(int)units, 256, 0, st>>>(ga, K, V, fused ? fused->Kw : nullptr,
+            grouped_tail_kernel<<<(int)units * 8, 256, 0, st>>>(ga, K, V, fused ? fused->Kw : nullptr,
                                                             fused ? fused->Vw : nullptr, fused ? fused->k_new : nullptr,
                                                             fused ? fused->v_new : nullptr);
             count_launch();

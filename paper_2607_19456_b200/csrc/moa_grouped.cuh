@@ -97,14 +97,14 @@ __device__ __forceinline__ int grouped_len(const GroupedArgs &a, int b)
 // filled tile of every unit is first copied into a scratch tile with its unused rows zeroed,
 // and the main kernel fetches that tile from there.  For the fused step the row being
 // appended (the unit's last row) is taken from k_new / v_new and also stored into the cache
-// (eqs. (4),(5)).  One block per stored (batch, kv head); the tile is 128 rows of 128 floats.
+// (eqs. (4),(5)).  Eight blocks per stored (batch, kv head), 16 rows of 128 floats each.
 __global__ void __launch_bounds__(256) grouped_tail_kernel(const GroupedArgs a, const float *K, const float *V, float *Kw,
                                                            float *Vw, const float *k_new, const float *v_new)
 {
-    const int unit = blockIdx.x, b = unit / a.h_kv_stored;
+    const int unit = blockIdx.x >> 3, part = blockIdx.x & 7, b = unit / a.h_kv_stored;
     const int len = grouped_len(a, b);
     if (len == 0) {
-        if (threadIdx.x == 0 && (unit % a.h_kv_stored) == 0)
+        if (threadIdx.x == 0 && part == 0 && (unit % a.h_kv_stored) == 0)
             raise_status(MOA_STATUS_SEQLEN_RANGE | (k_new != nullptr ? MOA_STATUS_APPEND_RANGE : 0));
         return;
     }
@@ -114,7 +114,7 @@ __global__ void __launch_bounds__(256) grouped_tail_kernel(const GroupedArgs a, 
     float4 *dstK = reinterpret_cast<float4 *>(a.tailK + (size_t)unit * 128 * 128);
     float4 *dstV = reinterpret_cast<float4 *>(a.tailV + (size_t)unit * 128 * 128);
     const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int i = threadIdx.x; i < 128 * 32; i += blockDim.x) {
+    for (int i = part * 512 + threadIdx.x; i < (part + 1) * 512; i += blockDim.x) {
         const int r = i >> 5, c = i & 31;
         float4 k = zero, v = zero;
         if (r < valid) {
