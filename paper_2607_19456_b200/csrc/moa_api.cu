@@ -335,6 +335,8 @@ static GroupedPlan plan_grouped(const DeviceState &s, int batch, int h_q, int h_
     p.splits = (int)splits;
     p.tiles_per_split = (tiles + p.splits - 1) / p.splits;
     p.ws_bytes = (size_t)units * p.share * p.splits * p.GH * 132 * sizeof(float);
+    const size_t flat_slots = (size_t)(units > s.sm_count ? units : s.sm_count);   // one partial per CTA in flat mode
+    if (p.share == 1 && flat_slots * p.GH * 132 * sizeof(float) > p.ws_bytes) p.ws_bytes = flat_slots * p.GH * 132 * sizeof(float);
     p.tail_bytes = (size_t)units * 2 * 128 * 128 * sizeof(float);
     p.ok = true;
     return p;
@@ -478,9 +480,7 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
     if (fast_ok && allow_grouped && (fused == nullptr || (aligned(fused->k_new, 16) && aligned(fused->v_new, 16))))
         gplan = plan_grouped(*dev, batch, h_q, h_kv, n_max, d_k, d_v);
     if (gplan.ok && ragged && (library_ws || seq_lens == nullptr)) gplan.ok = false;
-    // With per-sequence lengths this kernel's fixed (unit, split) grid is unbalanced; it still
-    // wins clearly for groups of 64, for 32 the flat decomposition of the warp-MMA kernel does.
-    if (gplan.ok && ragged && g_s != 64 && g_force_path != MOA_PATH_GROUPED) gplan.ok = false;
+
     if (gplan.ok && (library_ws || (ws && ws_bytes >= (ragged ? gplan.ws_ragged() : gplan.ws_bytes)))) path = MOA_PATH_GROUPED;
     if (g_force_path == MOA_PATH_GENERIC) path = MOA_PATH_GENERIC;
     else if (g_force_path == MOA_PATH_STREAM) {
@@ -528,6 +528,7 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
         ga.partial_out = partial_out;
         ga.seq_lens = seq_lens; ga.len_bias = len_bias;
         ga.tailK = nullptr; ga.tailV = nullptr;
+        ga.flat = 0;
         CUtensorMap mkt = mk, mvt = mv;
         if (ragged) {
             // the last, partly filled tile of every unit, zero-padded (and the appended row of
@@ -543,7 +544,11 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
             count_launch();
             if (cudaGetLastError() != cudaSuccess) return MOA_ERR_CUDA;
         }
-        const int grid = (int)(units * gplan.share * gplan.splits);
+        int grid = (int)(units * gplan.share * gplan.splits);
+        if (ragged && gplan.share == 1) {          // CTAs follow the lengths, read on the device
+            grid = (int)(units > dev->sm_count ? units : dev->sm_count);
+            ga.flat = grid;
+        }
         if (gplan.GH == 16) e = launch_grouped_cfg<16>(mk, mv, mkt, mvt, ga, grid, st);
         else if (gplan.GH == 32) e = launch_grouped_cfg<32>(mk, mv, mkt, mvt, ga, grid, st);
         else e = launch_grouped_cfg<64>(mk, mv, mkt, mvt, ga, grid, st);

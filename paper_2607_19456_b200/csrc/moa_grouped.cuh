@@ -82,6 +82,8 @@ struct GroupedArgs {
     const int32_t *seq_lens;   // device [batch] or nullptr: sequence b has seq_lens[b] + len_bias rows (n = capacity)
     int len_bias;
     float *tailK, *tailV;      // [stored units][128][128]: zero-padded copy of every unit's last tile, or nullptr
+    int flat;                  // 0, or the grid size: ragged caches, CTAs are dealt to the units in proportion
+                               // to their lengths (see flat_share)
 };
 
 // Rows of sequence b as this kernel family sees them; 0 for an out-of-range length.
@@ -90,6 +92,51 @@ __device__ __forceinline__ int grouped_len(const GroupedArgs &a, int b)
     if (a.seq_lens == nullptr) return a.n;
     const int len = a.seq_lens[b] + a.len_bias;
     return (len >= 1 && len <= a.n) ? len : 0;
+}
+
+// Ragged caches, `flat` mode (share == 1): the grid's CTAs are dealt to the units in
+// proportion to their tile counts, every unit getting at least one:
+//     s_u = 1 + floor(extra * tiles_u / total),   extra = grid - units,   capped at tiles_u,
+// and CTA c works on split (c - first_u) of the unit u whose CTA range contains c; its
+// partial goes to slot c.  Every CTA and the combine kernel recompute this from the lengths.
+struct FlatShare {
+    int unit, first, count;    // unit == -1: a CTA past the last unit's range
+};
+// Warp-collective (all 32 lanes, same arguments); every lane gets the answer.
+__device__ __forceinline__ FlatShare flat_share(const GroupedArgs &a, int grid, int want_cta, int want_unit, int lane)
+{
+    const int units = a.batch * a.h_kv_stored;
+    long long total = 0;
+    for (int b = lane; b < a.batch; b += 32) total += (long long)((grouped_len(a, b) + 127) / 128) * a.h_kv_stored;
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) total += __shfl_xor_sync(0xffffffffu, total, off);
+    const long long extra = grid > units ? grid - units : 0;
+    int first = 0;
+    for (int base = 0; base < units; base += 32) {
+        const int u = base + lane;
+        int cnt = 0;
+        if (u < units) {
+            const int tiles = (grouped_len(a, u / a.h_kv_stored) + 127) / 128;
+            long long c = 1 + (total > 0 ? extra * tiles / total : 0);
+            if (c > tiles) c = tiles > 0 ? tiles : 1;
+            cnt = (int)c;
+        }
+        int incl = cnt;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, incl, off);
+            if (lane >= off) incl += t;
+        }
+        const int mine = first + incl - cnt;
+        const bool hit = u < units && (u == want_unit || (want_cta >= mine && want_cta < mine + cnt));
+        const unsigned m = __ballot_sync(0xffffffffu, hit);
+        if (m != 0u) {
+            const int src = __ffs(m) - 1;
+            return FlatShare{base + src, __shfl_sync(0xffffffffu, mine, src), __shfl_sync(0xffffffffu, cnt, src)};
+        }
+        first += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    return FlatShare{-1, first, 0};
 }
 
 // Ragged caches: rows past a sequence's length hold arbitrary bits (possibly NaN), and a zero
@@ -235,14 +282,25 @@ grouped_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_co
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     // CTA order: the virtual heads that share one stored K/V head are neighbours, so they run
     // at the same time and the second reader of a chunk finds it in L2.
-    const int sub = blockIdx.x % a.share;
-    const int split = (blockIdx.x / a.share) % a.splits;
-    const int sunit = blockIdx.x / (a.share * a.splits);          // stored (batch, kv head)
+    int sub = blockIdx.x % a.share;
+    int split = (blockIdx.x / a.share) % a.splits;
+    int sunit = blockIdx.x / (a.share * a.splits);                // stored (batch, kv head)
+    int splits_u = a.splits;
+    if (a.flat) {                                  // warp 0 walks the lengths, all take its answer
+        int *s_share = reinterpret_cast<int *>(lred);    // (the reduction scratch is not in use yet)
+        if (warp == 0) {
+            const FlatShare f = flat_share(a, (int)gridDim.x, (int)blockIdx.x, -1, lane);
+            if (lane == 0) { s_share[0] = f.unit; s_share[1] = f.first; s_share[2] = f.count; }
+        }
+        __syncthreads();
+        if (s_share[0] < 0) return;
+        sub = 0; sunit = s_share[0]; split = (int)blockIdx.x - s_share[1]; splits_u = s_share[2];
+    }
     const int b = sunit / a.h_kv_stored, h = (sunit % a.h_kv_stored) * a.share + sub;   // virtual head
     const int unit = sunit;                                         // tensor-map coordinate
     const int len_b = grouped_len(a, b);           // 0: out-of-range length, the item is skipped
     const int tiles_total = (len_b + C::TILE - 1) / C::TILE;
-    const int tiles_per_split = a.seq_lens ? (tiles_total + a.splits - 1) / a.splits : a.tiles_per_split;
+    const int tiles_per_split = a.seq_lens ? (tiles_total + splits_u - 1) / splits_u : a.tiles_per_split;
     const int tile0 = split * tiles_per_split;
     int T = tiles_total - tile0;
     if (T > tiles_per_split) T = tiles_per_split;
@@ -590,7 +648,8 @@ grouped_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_co
                 if (lane == 0) lred[q4 * GH + h0 + g] = v;
             }
             named_sync(1, NS);
-            float *slot = a.ws + ((((size_t)b * a.h_kv + h) * a.splits + split) * GH) * PS;
+            float *slot = a.flat ? a.ws + ((size_t)blockIdx.x * GH) * PS
+                                 : a.ws + ((((size_t)b * a.h_kv + h) * a.splits + split) * GH) * PS;
             const int d = row_in_tile;               // TMEM lane of O^T = output feature
 #pragma unroll
             for (int j = 0; j < NP; ++j) {
@@ -669,9 +728,16 @@ __global__ void __launch_bounds__(128) grouped_combine_kernel(const GroupedArgs 
         return;
     }
     const int tiles_total = (len_b + 127) / 128;
-    const int tiles_per_split = a.seq_lens ? (tiles_total + a.splits - 1) / a.splits : a.tiles_per_split;
+    int splits_u = a.splits;
+    size_t first_slot = (size_t)unit * a.splits;
+    if (a.flat) {
+        const FlatShare f = flat_share(a, a.flat, -1, unit, lane);      // a.flat holds the grid size
+        splits_u = f.count;
+        first_slot = (size_t)f.first;
+    }
+    const int tiles_per_split = a.seq_lens ? (tiles_total + splits_u - 1) / splits_u : a.tiles_per_split;
     const int used = (tiles_total + tiles_per_split - 1) / tiles_per_split;   // non-empty splits
-    const float *base = a.ws + ((size_t)unit * a.splits * GH + g) * PS;
+    const float *base = a.ws + (first_slot * GH + g) * PS;
     const size_t stride = (size_t)GH * PS;
     float M = -INFINITY;
     for (int s0 = 0; s0 < used; s0 += 32) {
