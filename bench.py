@@ -301,6 +301,9 @@ def time_steps(run, steps, warmup, sampler=None, bracket=False):
     e1.record()
     torch.cuda.synchronize()
     kern_ms, kern_n, launches = moa.moa_profile_read()
+    LAST_BRACKETED.clear()
+    if bracket and kern_n:
+        LAST_BRACKETED.extend(moa.moa_profile_launch_ms(i) * 1e3 for i in range(int(kern_n)))
     moa.moa_profile(0)
     clocks = sampler.stop() if sampler else None
     barrier()
@@ -309,6 +312,7 @@ def time_steps(run, steps, warmup, sampler=None, bracket=False):
 
 
 _DIST = {"on": False}
+LAST_BRACKETED = []      # per-launch event times (us) of the last bracketed pass
 
 
 def barrier():
@@ -471,6 +475,8 @@ def main():
                 "how": ("CUDA events around the %d back-to-back launches of the timed region / launches" % launches)
                 if single_launch else "CUDA event pair around every launch of the kernel (second pass)",
                 "kernel_us_per_launch_event_bracketed": (kern_ms * 1e3 if kern_ms else None),
+                "kernel_us_event_bracketed_min_median_max": (
+                    [min(LAST_BRACKETED), statistics.median(LAST_BRACKETED), max(LAST_BRACKETED)] if LAST_BRACKETED else None),
                 "algorithmic_bytes_per_launch": decode_bytes,
                 "traffic": NCU_TRAFFIC_BYTES.get(wname)}
 
@@ -543,6 +549,9 @@ def main():
                                "decode_kernel_GBps": (odec / (okern * 1e-3) / 1e9) if okern else None,
                                "decode_kernel_frac_of_peak": (odec / (okern * 1e-3) / 1e9 / peak) if okern else None,
                                "frac_of_nominal_8000": ob / (oms * 1e-3) / 1e9 / 8000.0,
+                               "decode_kernel_us_min_median_max": (
+                                   [min(LAST_BRACKETED), statistics.median(LAST_BRACKETED), max(LAST_BRACKETED)]
+                                   if LAST_BRACKETED else None),
                                "l2": r.l2_note})
                 if name == "single_head":              # latency-bound: also with its lines resident in L2
                     r.nsets = 1

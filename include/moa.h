@@ -263,12 +263,14 @@ int moa_last_path(void);
  * moa_profile_read synchronises the device and reports the summed event time of the
  * timed decode-kernel launches in milliseconds, how many of them were timed, and the
  * total number of kernels launched since moa_profile(1).  Any pointer may be NULL.
- * moa_profile(0) stops counting.
+ * moa_profile_launch_ms reports the event time of the index-th timed launch (for a median
+ * or a histogram).  moa_profile(0) stops counting.
  */
 #define MOA_PROFILE_MAX_EVENTS 8192
 int moa_profile(int enable);
 int moa_profile_read(double *decode_kernel_ms, long long *decode_kernel_launches,
                      long long *all_kernel_launches);
+int moa_profile_launch_ms(long long index, double *ms);
 
 #ifdef __cplusplus
 }

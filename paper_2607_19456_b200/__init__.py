@@ -61,6 +61,7 @@ def lib():
         L.moa_profile.argtypes = [i]
         L.moa_profile_read.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_longlong),
                                        C.POINTER(C.c_longlong)]
+        L.moa_profile_launch_ms.argtypes = [C.c_longlong, C.POINTER(C.c_double)]
         _lib = L
     return _lib
 
@@ -206,3 +207,10 @@ def moa_profile_read():
     ms, n, a = C.c_double(0), C.c_longlong(0), C.c_longlong(0)
     _check(lib().moa_profile_read(C.byref(ms), C.byref(n), C.byref(a)), "moa_profile_read")
     return ms.value, n.value, a.value
+
+
+def moa_profile_launch_ms(index: int) -> float:
+    """Event time of the index-th timed decode-kernel launch, in milliseconds."""
+    ms = C.c_double(0)
+    _check(lib().moa_profile_launch_ms(int(index), C.byref(ms)), "moa_profile_launch_ms")
+    return ms.value

@@ -964,4 +964,18 @@ int moa_profile_read(double *decode_kernel_ms, long long *decode_kernel_launches
     return MOA_OK;
 }
 
+int moa_profile_launch_ms(long long index, double *ms)
+{
+    if (!ms || index < 0 || index >= g_prof_timed) return MOA_ERR_INVALID;
+    if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return MOA_ERR_CUDA; }
+    float t = 0.f;
+    if (!g_prof_ev || !g_prof_ev[2 * index] || !g_prof_ev[2 * index + 1] ||
+        cudaEventElapsedTime(&t, g_prof_ev[2 * index], g_prof_ev[2 * index + 1]) != cudaSuccess) {
+        cudaGetLastError();
+        return MOA_ERR_CUDA;
+    }
+    *ms = t;
+    return MOA_OK;
+}
+
 }  // extern "C"
