@@ -263,6 +263,23 @@ def test_rows_past_the_length_may_hold_anything(hq, hkv, d, want):
         assert np.all(np.isfinite(out)) and max_err(out, ref) <= TOL
 
 
+def test_ragged_groups_cut_into_two_ctas_of_32_heads():
+    # MOA_OPT_GROUPED_HEADS = 32 on groups of 64: two neighbouring CTAs per tile range, the
+    # fixed (unit, split) grid instead of the length-proportional one
+    B, hq, hkv, n_max = 3, 64, 1, 1500
+    q, K, V, s = make(770, B, hq, hkv, n_max, 128, 128)
+    lens = np.array([1500, 7, 640], np.int32)
+    ref = oracle.decode_varlen(q, K, V, lens, s)
+    for b in range(B):
+        V[b, :, lens[b]:] = np.nan
+    moa.moa_set_option(moa.OPT_GROUPED_HEADS, 32)
+    try:
+        out = gpu_decode(q, K, V, s, seq_lens=lens, expect_path=moa.PATH_GROUPED)
+    finally:
+        moa.moa_set_option(moa.OPT_GROUPED_HEADS, 0)
+    assert np.all(np.isfinite(out)) and max_err(out, ref) <= TOL
+
+
 @pytest.mark.parametrize("path,hq", [(moa.PATH_AUTO, 4), (moa.PATH_GENERIC, 4), (moa.PATH_AUTO, 16), (moa.PATH_AUTO, 128)])
 def test_out_of_range_length_sets_status_and_skips_the_item(path, hq):
     B, hkv, n_max, D = 3, 2, 64, 128          # hq = 4: FMA kernel, 16: warp-MMA kernel, 128: tcgen05 kernel
