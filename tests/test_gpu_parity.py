@@ -454,6 +454,21 @@ def test_layers_call_runs_every_layer():
         assert max_err(outs[l].cpu().numpy(), oracle.decode(q, K, V, s)) <= TOL
 
 
+@pytest.mark.parametrize("hq,hkv,d", [(4, 2, 128), (16, 2, 128), (64, 1, 128), (6, 3, 40)])
+def test_non_finite_inputs_do_not_hang_or_raise_status(hq, hkv, d):
+    # values are unspecified for non-finite inputs, but every kernel family must finish, keep its
+    # bounded waits unexpired and leave the rows of the untouched batch item exact
+    B, n = 2, 900
+    q, K, V, s = make(8800 + hq, B, hq, hkv, n, d, d)
+    ref = oracle.decode(q[1:], K[1:], V[1:], s)
+    K[0, 0, 5, 3] = np.inf
+    K[0, 0, 700, 1] = np.nan
+    V[0, 0, 17, 2] = -np.inf
+    q[0, 0, 0] = np.nan
+    out = gpu_decode(q, K, V, s)               # asserts a clear status word and intact guards
+    assert max_err(out[1:], ref) <= TOL
+
+
 def test_argument_errors():
     q, K, V, s = make(970, 1, 4, 2, 16, 128, 128)
     gq, gK, gV = Guarded(q), Guarded(K), Guarded(V)
