@@ -172,6 +172,9 @@ static StreamPlan plan_stream(int g_s, int d_k, int d_v)
     p.G = stream_group(g_s, &p.share);
     p.mma = mma_allowed() && p.G == 8 && p.D >= 64;     // (the caller drops it for huge caches)
     if (p.mma && g_s % 16 == 0) { p.G = 16; p.share = g_s / 16; }   // two 8-head tiles per fetched row
+    if (mma_allowed() && p.D >= 64 && g_s > 8 && g_s < 16) {         // 9..15 heads: one padded 16-head group
+        p.G = 16; p.share = 1; p.mma = true;
+    }
     p.R = p.mma ? 16 : rows_per_block(p.D, p.G);
     p.ok = true;
     return p;

@@ -52,6 +52,8 @@ def automatic_path(D, gs):
     """The kernel family the library picks for a dense, aligned call."""
     if D == 128 and gs in (32, 64):
         return moa.PATH_GROUPED
+    if 8 < gs < 16 and D >= 64:
+        return moa.PATH_MMA                  # one padded group of 16 heads
     if gs <= 8:
         G = 1
         while G < gs:
