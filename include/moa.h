@@ -169,6 +169,42 @@ int moa_append_decode(const float *q, float *K, float *V, const float *k_new,
                       void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * Caches that are not densely packed (section 5.3 pre-allocates the cache once; a serving
+ * stack often carves K and V out of one larger allocation, keeps the heads innermost, or
+ * shares one prefix between batch items).  Element (b, h, i, t) of K lives at
+ *   K + b*k_strides[0] + h*k_strides[1] + i*k_strides[2] + t
+ * and likewise for V with v_strides; both are HOST arrays of three element counts
+ * {batch stride, kv-head stride, row stride}.  The feature axis is always contiguous.
+ * Strides must be >= 0 and at most 2^40, the row stride at least the row length; a zero batch or head
+ * stride (the same rows read for every item) is allowed for caches that are only read.
+ * q, out, k_new, v_new stay dense.  The computation is Algorithm 1 on the addressed rows;
+ * seq_lens (device int32[batch]) may be NULL: every sequence then has n_max rows.
+ *   - every stride a multiple of 4, row stride == row length: the kernels of the dense
+ *     calls (the tcgen05 kernel excepted, its groups run on the warp-MMA kernel);
+ *   - every stride a multiple of 4, larger row stride, d_k and d_v in {64, 128}: the
+ *     warp-MMA kernel (its tiled copies take any stride), groups padded to 8 heads;
+ *   - anything else: the catch-all kernel.
+ * `workspace` as for moa_decode_attn_varlen (moa_workspace_bytes covers these calls);
+ * moa_decode_attn_strided also accepts workspace == NULL and then uses (and may grow)
+ * the library-owned workspace like moa_decode_attn.
+ * moa_kv_append_strided and moa_decode_step_strided are moa_kv_append and moa_decode_step
+ * on such a cache; they refuse zero batch/head strides (MOA_ERR_INVALID).
+ */
+int moa_decode_attn_strided(const float *q, const float *K, const float *V, float *out,
+                            const int32_t *seq_lens, int batch, int h_q, int h_kv, int n_max,
+                            int d_k, int d_v, float scale, const long long *k_strides,
+                            const long long *v_strides, void *workspace,
+                            size_t workspace_bytes, void *stream);
+int moa_kv_append_strided(float *K, float *V, const float *k_new, const float *v_new,
+                          const int32_t *pos, int batch, int h_kv, int n_max, int d_k, int d_v,
+                          const long long *k_strides, const long long *v_strides, void *stream);
+int moa_decode_step_strided(const float *q, float *K, float *V, const float *k_new,
+                            const float *v_new, float *out, int32_t *lens, int batch, int h_q,
+                            int h_kv, int n_max, int d_k, int d_v, float scale,
+                            const long long *k_strides, const long long *v_strides,
+                            void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * Host-buffer convenience call: q, K, V, out are HOST pointers (pinned memory gives
  * full copy bandwidth).  Copies the inputs to library-owned device staging buffers,
  * runs moa_decode_attn and copies `out` back; synchronises before returning.

@@ -51,6 +51,10 @@ def lib():
         L.moa_lens_add.argtypes = [p, i, i, p]
         L.moa_decode_step.argtypes = [p, p, p, p, p, p, p, i, i, i, i, i, i, f, p, sz, p]
         L.moa_append_decode.argtypes = [p, p, p, p, p, p, p, i, i, i, i, i, i, f, p, sz, p]
+        ll3 = C.POINTER(C.c_longlong)
+        L.moa_decode_attn_strided.argtypes = [p, p, p, p, p, i, i, i, i, i, i, f, ll3, ll3, p, sz, p]
+        L.moa_kv_append_strided.argtypes = [p, p, p, p, p, i, i, i, i, i, ll3, ll3, p]
+        L.moa_decode_step_strided.argtypes = [p, p, p, p, p, p, p, i, i, i, i, i, i, f, ll3, ll3, p, sz, p]
         L.moa_decode_attn_host.argtypes = [p, p, p, p, i, i, i, i, i, i, f]
         L.moa_device_status.argtypes = [p, C.POINTER(C.c_int)]
         L.moa_min_bytes.argtypes = [i, i, i, C.c_longlong, i, i]
@@ -164,6 +168,38 @@ def moa_append_decode(q, K, V, k_new, v_new, out, pos, batch, h_q, h_kv, n_max, 
                                    _ptr(pos), batch, h_q, h_kv, n_max, d_k, d_v, scale,
                                    _ptr(workspace), workspace_bytes, _stream(stream)),
            "moa_append_decode")
+
+
+def _strides3(st):
+    """(batch, head, row) element strides as a host array of three long long."""
+    if len(st) != 3:
+        raise ValueError("strides are (batch, kv head, row) element counts")
+    return (C.c_longlong * 3)(*[int(x) for x in st])
+
+
+def moa_decode_attn_strided(q, K, V, out, seq_lens, batch, h_q, h_kv, n_max, d_k, d_v, scale, k_strides,
+                            v_strides, workspace=None, workspace_bytes=0, stream=None):
+    """K, V: base addresses (tensors or ints) of caches whose element (b, h, i, t) sits at
+    base + b*strides[0] + h*strides[1] + i*strides[2] + t; seq_lens may be None."""
+    _check(lib().moa_decode_attn_strided(_ptr(q), _ptr(K), _ptr(V), _ptr(out), _ptr(seq_lens), batch, h_q,
+                                         h_kv, n_max, d_k, d_v, scale, _strides3(k_strides),
+                                         _strides3(v_strides), _ptr(workspace), workspace_bytes,
+                                         _stream(stream)), "moa_decode_attn_strided")
+
+
+def moa_kv_append_strided(K, V, k_new, v_new, pos, batch, h_kv, n_max, d_k, d_v, k_strides, v_strides,
+                          stream=None):
+    _check(lib().moa_kv_append_strided(_ptr(K), _ptr(V), _ptr(k_new), _ptr(v_new), _ptr(pos), batch, h_kv,
+                                       n_max, d_k, d_v, _strides3(k_strides), _strides3(v_strides),
+                                       _stream(stream)), "moa_kv_append_strided")
+
+
+def moa_decode_step_strided(q, K, V, k_new, v_new, out, lens, batch, h_q, h_kv, n_max, d_k, d_v, scale,
+                            k_strides, v_strides, workspace, workspace_bytes, stream=None):
+    _check(lib().moa_decode_step_strided(_ptr(q), _ptr(K), _ptr(V), _ptr(k_new), _ptr(v_new), _ptr(out),
+                                         _ptr(lens), batch, h_q, h_kv, n_max, d_k, d_v, scale,
+                                         _strides3(k_strides), _strides3(v_strides), _ptr(workspace),
+                                         workspace_bytes, _stream(stream)), "moa_decode_step_strided")
 
 
 def moa_decode_attn_host(q, K, V, out, batch, h_q, h_kv, n, d_k, d_v, scale):

@@ -114,6 +114,45 @@ static int validate_dims(int batch, int h_q, int h_kv, int n, int d_k, int d_v)
     return MOA_OK;
 }
 
+// ---- cache layout ------------------------------------------------------------------------
+struct Layout {
+    CacheStrides k, v;      // element strides: batch item, kv head, row
+    bool dense;             // exactly [batch, h_kv, n_max, d]
+    bool rows_contig;       // row stride == row length for both caches
+    bool vec4;              // every stride a multiple of 4 elements (16 bytes)
+};
+
+static Layout dense_layout(int h_kv, int n_max, int d_k, int d_v)
+{
+    Layout l;
+    l.k = {(long long)h_kv * n_max * d_k, (long long)n_max * d_k, (long long)d_k};
+    l.v = {(long long)h_kv * n_max * d_v, (long long)n_max * d_v, (long long)d_v};
+    l.dense = l.rows_contig = true;
+    l.vec4 = (d_k % 4 == 0) && (d_v % 4 == 0);
+    return l;
+}
+
+// Layout from caller-supplied strides {batch, head, row}; false if they are unusable.
+static bool strided_layout(const long long *ks, const long long *vs, int h_kv, int n_max, int d_k, int d_v, Layout *out)
+{
+    if (!ks || !vs) return false;
+    for (int i = 0; i < 3; ++i)
+        if (ks[i] < 0 || vs[i] < 0 || ks[i] > (1LL << 40) || vs[i] > (1LL << 40)) return false;
+    if (ks[2] < d_k || vs[2] < d_v) return false;        // rows may not overlap
+    Layout l;
+    l.k = {ks[0], ks[1], ks[2]};
+    l.v = {vs[0], vs[1], vs[2]};
+    const Layout d = dense_layout(h_kv, n_max, d_k, d_v);
+    l.dense = l.k.sb == d.k.sb && l.k.sh == d.k.sh && l.k.sr == d.k.sr && l.v.sb == d.v.sb && l.v.sh == d.v.sh &&
+              l.v.sr == d.v.sr;
+    l.rows_contig = (l.k.sr == d_k) && (l.v.sr == d_v);
+    l.vec4 = true;
+    for (int i = 0; i < 3; ++i)
+        if (ks[i] % 4 != 0 || vs[i] % 4 != 0) l.vec4 = false;
+    *out = l;
+    return true;
+}
+
 // ---- streaming-kernel plan -------------------------------------------------------------
 struct StreamPlan {
     bool ok = false;
@@ -150,18 +189,22 @@ static int rows_per_block(int D, int G)
 // size (and with it the whole decomposition) differs.  MOA_PATH_STREAM forces the FMA kernel.
 static bool mma_allowed() { return g_force_path != MOA_PATH_STREAM; }
 
-static StreamPlan plan_stream(int g_s, int d_k, int d_v)
+static StreamPlan plan_stream(int g_s, int d_k, int d_v, bool rows_contig = true)
 {
     StreamPlan p;
     p.Dk = d_k;
-    if (d_k != d_v) {
+    if (d_k != d_v || !rows_contig || (g_force_path == MOA_PATH_MMA && d_k >= 64)) {
         // Unequal row lengths: only the paired mode of the warp-MMA kernel handles them (every
-        // warp owns one operand), in groups of 8 heads.
+        // warp owns one operand), in groups of 8 heads.  Rows that are not contiguous in memory
+        // (a row stride larger than the row) need tiled copies, which only that kernel issues:
+        // small groups are padded to 8 heads, which costs no extra memory traffic.
         if (!mma_allowed() || (d_k != 64 && d_k != 128) || (d_v != 64 && d_v != 128)) return p;
-        if (g_s > 8 && g_s % 8 != 0) return p;
+        if (g_s > 8 && g_s % 8 != 0 && !(d_k == d_v && g_s < 16)) return p;
         p.D = d_v;
         p.G = 8;
         p.share = g_s > 8 ? g_s / 8 : 1;
+        if (d_k == d_v && g_s > 8 && g_s < 16) { p.G = 16; p.share = 1; }
+        else if (d_k == d_v && g_s % 16 == 0) { p.G = 16; p.share = g_s / 16; }
         p.mma = true;
         p.R = 16;
         p.ok = true;
@@ -170,7 +213,7 @@ static StreamPlan plan_stream(int g_s, int d_k, int d_v)
     if (d_k != 32 && d_k != 64 && d_k != 128) return p;
     p.D = d_k;
     p.G = stream_group(g_s, &p.share);
-    p.mma = mma_allowed() && p.G == 8 && p.D >= 64;     // (the caller drops it for huge caches)
+    p.mma = mma_allowed() && p.G == 8 && p.D >= 64;
     if (p.mma && g_s % 16 == 0) { p.G = 16; p.share = g_s / 16; }   // two 8-head tiles per fetched row
     if (mma_allowed() && p.D >= 64 && g_s > 8 && g_s < 16) {         // 9..15 heads: one padded 16-head group
         p.G = 16; p.share = 1; p.mma = true;
@@ -229,15 +272,16 @@ static cudaError_t launch_stream_cfg(const DecodeArgs &a, int num_ctas, cudaStre
     return cudaGetLastError();
 }
 
-static bool make_rows_map(CUtensorMap *m, const float *base, long long rows_total, int D);
+static bool make_rows_map(CUtensorMap *m, const float *base, int D, int n_max, int heads, int batch,
+                          const CacheStrides &cs);
 
 template <class C>
 static cudaError_t launch_mma_cfg(const DecodeArgs &a, int num_ctas, cudaStream_t st)
 {
-    // The caches as [d/32 column groups][rows][32 floats]: one box is a 16-row tile.
-    const long long rows_total = (long long)a.batch * (a.h_kv / a.kv_share) * a.n_max;
     CUtensorMap mk, mv;
-    if (!make_rows_map(&mk, a.K, rows_total, C::DK) || !make_rows_map(&mv, a.V, rows_total, C::DV))
+    const int h_stored = a.h_kv / a.kv_share;
+    if (!make_rows_map(&mk, a.K, C::DK, a.n_max, h_stored, a.batch, CacheStrides{a.k_sb, a.k_sh, a.k_sr}) ||
+        !make_rows_map(&mv, a.V, C::DV, a.n_max, h_stored, a.batch, CacheStrides{a.v_sb, a.v_sh, a.v_sr}))
         return cudaErrorInvalidValue;
     static bool attr_set[kMaxDevices] = {};
     int dev = 0;
@@ -380,17 +424,22 @@ static bool make_cache_map(CUtensorMap *m, const float *base, long long units, i
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Tensor map over a cache seen as rows of D floats: dimensions (32 floats, rows, D/32 column
-// groups), so that one box of 16 rows lands as D/32 swizzled [16 rows][128 bytes] sub-tiles.
-static bool make_rows_map(CUtensorMap *m, const float *base, long long rows_total, int D)
+// Tensor map over a cache [batch][stored kv heads][n_max rows][D floats] with arbitrary element
+// strides, seen as (32 floats, row, D/32 column groups, head, batch item): one box of 16 rows
+// lands as D/32 swizzled [16 rows][128 bytes] sub-tiles; rows past n_max read as zero.
+static bool make_rows_map(CUtensorMap *m, const float *base, int D, int n_max, int heads, int batch,
+                          const CacheStrides &cs)
 {
     TmapEncodeFn enc = tmap_encoder();
     if (!enc) return false;
-    cuuint64_t dims[3] = {32, (cuuint64_t)rows_total, (cuuint64_t)(D / 32)};
-    cuuint64_t strides[2] = {(cuuint64_t)D * 4, 128};
-    cuuint32_t box[3] = {32, 16, (cuuint32_t)(D / 32)};
-    cuuint32_t estr[3] = {1, 1, 1};
-    return enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(base), dims, strides, box, estr,
+    cuuint64_t dims[5] = {32, (cuuint64_t)n_max, (cuuint64_t)(D / 32), (cuuint64_t)heads, (cuuint64_t)batch};
+    cuuint64_t strides[4] = {(cuuint64_t)cs.sr * 4, 128, (cuuint64_t)cs.sh * 4, (cuuint64_t)cs.sb * 4};
+    // a dimension of extent 1 is never stepped along: give it a harmless legal stride
+    if (heads == 1 && strides[2] == 0) strides[2] = 16;
+    if (batch == 1 && strides[3] == 0) strides[3] = 16;
+    cuuint32_t box[5] = {32, 16, (cuuint32_t)(D / 32), 1, 1};
+    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 5, const_cast<float *>(base), dims, strides, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -451,7 +500,7 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
                        int h_q, int h_kv, const int32_t *seq_lens, int len_bias, int n_max,
                        int d_k, int d_v, float scale, void *ws, size_t ws_bytes,
                        bool library_ws, cudaStream_t st, const FusedStep *fused = nullptr,
-                       bool allow_grouped = true, float *partial_out = nullptr)
+                       bool allow_grouped = true, float *partial_out = nullptr, const Layout *layp = nullptr)
 {
     if (!q || !K || !V || (!out && !partial_out)) return MOA_ERR_INVALID;
     if (partial_out != nullptr) out = partial_out;      // (alignment checks below apply to it)
@@ -467,20 +516,22 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
     if (rc != MOA_OK) return rc;
 
     const int g_s = h_q / h_kv;
-    StreamPlan plan = plan_stream(g_s, d_k, d_v);
-    if (plan.mma && (long long)batch * h_kv * n_max > 0x7fffff00LL) {   // row coordinates are 32-bit
-        plan.mma = false;
-        plan.ok = (d_k == d_v);
-        plan.G = stream_group(g_s, &plan.share);
-        plan.R = rows_per_block(plan.D, plan.G);
+    const Layout lay = layp ? *layp : dense_layout(h_kv, n_max, d_k, d_v);
+    StreamPlan plan = plan_stream(g_s, d_k, d_v, lay.rows_contig);
+    bool fast_ok = plan.ok && lay.vec4 && aligned(q, 16) && aligned(K, 16) && aligned(V, 16) && aligned(out, 16);
+    if (fast_ok && plan.mma && !lay.dense) {
+        // strides a tensor map cannot express (zero, or beyond its range): catch-all kernel
+        CUtensorMap probe;
+        if (!make_rows_map(&probe, K, plan.Dk, n_max, h_kv, batch, lay.k) ||
+            !make_rows_map(&probe, V, plan.D, n_max, h_kv, batch, lay.v))
+            fast_ok = false;
     }
-    const bool fast_ok = plan.ok && aligned(q, 16) && aligned(K, 16) && aligned(V, 16) && aligned(out, 16);
     int path = fast_ok ? (plan.mma ? MOA_PATH_MMA : MOA_PATH_STREAM) : MOA_PATH_GENERIC;
     // Large head groups go to the tcgen05 kernel; ragged caches and the fused step need scratch
     // for the zero-padded copy of every unit's last tile on top of the partial slots.
     GroupedPlan gplan;
     const bool ragged = (seq_lens != nullptr) || (fused != nullptr);
-    if (fast_ok && allow_grouped && (fused == nullptr || (aligned(fused->k_new, 16) && aligned(fused->v_new, 16))))
+    if (fast_ok && allow_grouped && lay.dense && (fused == nullptr || (aligned(fused->k_new, 16) && aligned(fused->v_new, 16))))
         gplan = plan_grouped(*dev, batch, h_q, h_kv, n_max, d_k, d_v);
     if (gplan.ok && ragged && (library_ws || seq_lens == nullptr)) gplan.ok = false;
 
@@ -501,6 +552,8 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
     a.seq_lens = seq_lens; a.len_bias = len_bias;
     a.batch = batch; a.h_q = h_q; a.h_kv = h_kv; a.g_s = g_s; a.kv_share = 1;
     a.n_max = n_max; a.d_k = d_k; a.d_v = d_v;
+    a.k_sb = lay.k.sb; a.k_sh = lay.k.sh; a.k_sr = lay.k.sr;
+    a.v_sb = lay.v.sb; a.v_sh = lay.v.sh; a.v_sr = lay.v.sr;
     a.qscale = scale * kLog2e;
     a.Kw = nullptr; a.Vw = nullptr; a.k_new = nullptr; a.v_new = nullptr; a.lens_rw = nullptr;
     a.tickets = nullptr;
@@ -710,6 +763,8 @@ size_t moa_workspace_bytes(int batch, int h_q, int h_kv, int n_max, int d_k, int
     int ctas = g_num_ctas;
     if (ctas <= 0) ctas = (current_device(&dev) == MOA_OK) ? dev->sm_count : 256;
     size_t need = stream_ws_bytes(plan, ctas);
+    const StreamPlan tiled = plan_stream(h_q / h_kv, d_k, d_v, false);   // caches with a row stride
+    if (tiled.ok && stream_ws_bytes(tiled, ctas) > need) need = stream_ws_bytes(tiled, ctas);
     if (dev != nullptr || current_device(&dev) == MOA_OK) {
         const GroupedPlan gp = plan_grouped(*dev, batch, h_q, h_kv, n_max, d_k, d_v);
         if (gp.ok && gp.ws_ragged() > need) need = gp.ws_ragged();
@@ -717,8 +772,8 @@ size_t moa_workspace_bytes(int batch, int h_q, int h_kv, int n_max, int d_k, int
     return (need + 255) / 256 * 256;
 }
 
-int moa_kv_append(float *K, float *V, const float *k_new, const float *v_new, const int32_t *pos,
-                  int batch, int h_kv, int n_max, int d_k, int d_v, void *stream)
+static int kv_append_impl(float *K, float *V, const float *k_new, const float *v_new, const int32_t *pos,
+                          int batch, int h_kv, int n_max, int d_k, int d_v, const Layout &lay, void *stream)
 {
     if (!K || !V || !k_new || !v_new || !pos) return MOA_ERR_INVALID;
     if (batch < 1 || h_kv < 1 || n_max < 1 || d_k < 1 || d_v < 1) return MOA_ERR_INVALID;
@@ -733,9 +788,34 @@ int moa_kv_append(float *K, float *V, const float *k_new, const float *v_new, co
     kv_append_kernel<<<(int)blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(
         reinterpret_cast<uint32_t *>(K), reinterpret_cast<uint32_t *>(V),
         reinterpret_cast<const uint32_t *>(k_new), reinterpret_cast<const uint32_t *>(v_new), pos,
-        batch, h_kv, n_max, d_k, d_v);
+        batch, h_kv, n_max, d_k, d_v, lay.k, lay.v);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? MOA_OK : MOA_ERR_CUDA;
+}
+
+int moa_kv_append(float *K, float *V, const float *k_new, const float *v_new, const int32_t *pos,
+                  int batch, int h_kv, int n_max, int d_k, int d_v, void *stream)
+{
+    if (batch < 1 || h_kv < 1 || n_max < 1 || d_k < 1 || d_v < 1) return MOA_ERR_INVALID;
+    return kv_append_impl(K, V, k_new, v_new, pos, batch, h_kv, n_max, d_k, d_v,
+                          dense_layout(h_kv, n_max, d_k, d_v), stream);
+}
+
+// A cache that is written must not alias itself: strides of zero are refused here.
+static bool writable_layout(const Layout &l, int batch, int h_kv)
+{
+    return (batch == 1 || (l.k.sb > 0 && l.v.sb > 0)) && (h_kv == 1 || (l.k.sh > 0 && l.v.sh > 0));
+}
+
+int moa_kv_append_strided(float *K, float *V, const float *k_new, const float *v_new, const int32_t *pos,
+                          int batch, int h_kv, int n_max, int d_k, int d_v, const long long *k_strides,
+                          const long long *v_strides, void *stream)
+{
+    if (batch < 1 || h_kv < 1 || n_max < 1 || d_k < 1 || d_v < 1) return MOA_ERR_INVALID;
+    Layout lay;
+    if (!strided_layout(k_strides, v_strides, h_kv, n_max, d_k, d_v, &lay) || !writable_layout(lay, batch, h_kv))
+        return MOA_ERR_INVALID;
+    return kv_append_impl(K, V, k_new, v_new, pos, batch, h_kv, n_max, d_k, d_v, lay, stream);
 }
 
 int moa_lens_add(int32_t *lens, int batch, int delta, void *stream)
@@ -754,7 +834,7 @@ int moa_lens_add(int32_t *lens, int batch, int delta, void *stream)
 static int step_impl(const float *q, float *K, float *V, const float *k_new, const float *v_new,
                      float *out, int32_t *lens_rw, const int32_t *lens, int batch, int h_q, int h_kv,
                      int n_max, int d_k, int d_v, float scale, void *workspace, size_t workspace_bytes,
-                     void *stream, bool advance)
+                     void *stream, bool advance, const Layout *layp = nullptr)
 {
     if (!q || !K || !V || !k_new || !v_new || !out || !lens) return MOA_ERR_INVALID;
     int rc = validate_dims(batch, h_q, h_kv, n_max, d_k, d_v);
@@ -767,8 +847,15 @@ static int step_impl(const float *q, float *K, float *V, const float *k_new, con
     rc = current_device(&dev);
     if (rc != MOA_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const StreamPlan plan = plan_stream(h_q / h_kv, d_k, d_v);
-    const bool fast_ok = plan.ok && aligned(q, 16) && aligned(K, 16) && aligned(V, 16) && aligned(out, 16);
+    const Layout lay = layp ? *layp : dense_layout(h_kv, n_max, d_k, d_v);
+    const StreamPlan plan = plan_stream(h_q / h_kv, d_k, d_v, lay.rows_contig);
+    bool fast_ok = plan.ok && lay.vec4 && aligned(q, 16) && aligned(K, 16) && aligned(V, 16) && aligned(out, 16);
+    if (fast_ok && plan.mma && !lay.dense) {
+        CUtensorMap probe;
+        if (!make_rows_map(&probe, K, plan.Dk, n_max, h_kv, batch, lay.k) ||
+            !make_rows_map(&probe, V, plan.D, n_max, h_kv, batch, lay.v))
+            fast_ok = false;
+    }
     const bool stream_path = fast_ok && g_force_path != MOA_PATH_GENERIC;
     if ((g_force_path == MOA_PATH_STREAM || g_force_path == MOA_PATH_MMA) && !fast_ok) return MOA_ERR_UNSUPPORTED;
     if (stream_path) {          // validate the scratch before anything is written
@@ -781,13 +868,13 @@ static int step_impl(const float *q, float *K, float *V, const float *k_new, con
         FusedStep f;
         f.Kw = K; f.Vw = V; f.k_new = k_new; f.v_new = v_new; f.lens_rw = advance ? lens_rw : nullptr;
         return decode_impl(q, K, V, out, batch, h_q, h_kv, lens, 1, n_max, d_k, d_v, scale, workspace,
-                           workspace_bytes, false, st, &f);
+                           workspace_bytes, false, st, &f, true, nullptr, &lay);
     }
     // Otherwise the same thing as three launches.
-    rc = moa_kv_append(K, V, k_new, v_new, lens, batch, h_kv, n_max, d_k, d_v, stream);
+    rc = kv_append_impl(K, V, k_new, v_new, lens, batch, h_kv, n_max, d_k, d_v, lay, stream);
     if (rc != MOA_OK) return rc;
     rc = decode_impl(q, K, V, out, batch, h_q, h_kv, lens, 1, n_max, d_k, d_v, scale, workspace,
-                     workspace_bytes, false, st);
+                     workspace_bytes, false, st, nullptr, true, nullptr, &lay);
     if (rc != MOA_OK || !advance) return rc;
     lens_add_kernel<<<(batch + 127) / 128, 128, 0, st>>>(lens_rw, batch, 1, n_max);
     count_launch();
@@ -808,6 +895,32 @@ int moa_append_decode(const float *q, float *K, float *V, const float *k_new, co
 {
     return step_impl(q, K, V, k_new, v_new, out, nullptr, pos, batch, h_q, h_kv, n_max, d_k, d_v, scale,
                      workspace, workspace_bytes, stream, false);
+}
+
+int moa_decode_attn_strided(const float *q, const float *K, const float *V, float *out, const int32_t *seq_lens,
+                            int batch, int h_q, int h_kv, int n_max, int d_k, int d_v, float scale,
+                            const long long *k_strides, const long long *v_strides, void *workspace,
+                            size_t workspace_bytes, void *stream)
+{
+    if (validate_dims(batch, h_q, h_kv, n_max, d_k, d_v) == MOA_ERR_INVALID) return MOA_ERR_INVALID;
+    Layout lay;
+    if (!strided_layout(k_strides, v_strides, h_kv, n_max, d_k, d_v, &lay)) return MOA_ERR_INVALID;
+    return decode_impl(q, K, V, out, batch, h_q, h_kv, seq_lens, 0, n_max, d_k, d_v, scale, workspace,
+                       workspace_bytes, workspace == nullptr, static_cast<cudaStream_t>(stream), nullptr, true,
+                       nullptr, &lay);
+}
+
+int moa_decode_step_strided(const float *q, float *K, float *V, const float *k_new, const float *v_new, float *out,
+                            int32_t *lens, int batch, int h_q, int h_kv, int n_max, int d_k, int d_v, float scale,
+                            const long long *k_strides, const long long *v_strides, void *workspace,
+                            size_t workspace_bytes, void *stream)
+{
+    if (validate_dims(batch, h_q, h_kv, n_max, d_k, d_v) == MOA_ERR_INVALID) return MOA_ERR_INVALID;
+    Layout lay;
+    if (!strided_layout(k_strides, v_strides, h_kv, n_max, d_k, d_v, &lay) || !writable_layout(lay, batch, h_kv))
+        return MOA_ERR_INVALID;
+    return step_impl(q, K, V, k_new, v_new, out, lens, lens, batch, h_q, h_kv, n_max, d_k, d_v, scale,
+                     workspace, workspace_bytes, stream, true, &lay);
 }
 
 int moa_decode_attn_host(const float *q, const float *K, const float *V, float *out, int batch,

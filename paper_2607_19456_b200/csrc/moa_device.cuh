@@ -126,8 +126,12 @@ struct DecodeArgs {
     int h_kv;                 // kv heads as the kernels count them (virtual heads, see kv_share)
     int g_s;                  // query heads per (virtual) kv head
     int kv_share;             // consecutive virtual kv heads that read the same stored K/V head
-    int n_max;                // row capacity = stride between heads
+    int n_max;                // row capacity of every (batch, kv head) slab
     int d_k, d_v;
+    // Element strides of the caches: batch item, stored kv head, row.  The dense layout is
+    // (h_kv * n_max * d, n_max * d, d); the 1-D bulk copies need a row stride of exactly d.
+    long long k_sb, k_sh, k_sr;
+    long long v_sb, v_sh, v_sr;
     float qscale;             // scale * log2(e): scores live in the log2 domain
     // ---- fused step (all null/zero for a plain decode) ----
     float *Kw, *Vw;           // writable K / V when the new row is appended by the decode kernel

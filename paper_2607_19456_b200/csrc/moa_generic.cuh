@@ -28,8 +28,8 @@ __global__ void __launch_bounds__(kGenericWarps * 32) generic_decode_kernel(cons
     const int len = seq_len_of(a, b);
     if (len == 0) return;                               // out-of-range length: untouched
     const int h = g / a.g_s;
-    const float *Kg = a.K + ((size_t)b * a.h_kv + h) * (size_t)a.n_max * a.d_k;
-    const float *Vg = a.V + ((size_t)b * a.h_kv + h) * (size_t)a.n_max * a.d_v;
+    const float *Kg = a.K + (size_t)b * a.k_sb + (size_t)h * a.k_sh;
+    const float *Vg = a.V + (size_t)b * a.v_sb + (size_t)h * a.v_sh;
     const float *qg = a.q + ((size_t)b * a.h_q + g) * a.d_k;
 
     for (int j = threadIdx.x; j < a.d_k; j += blockDim.x) sq[j] = qg[j] * a.qscale;
@@ -41,7 +41,7 @@ __global__ void __launch_bounds__(kGenericWarps * 32) generic_decode_kernel(cons
     float m = -INFINITY, l = 0.f;
 
     for (int row = warp; row < len; row += kGenericWarps) {
-        const float *kr = Kg + (size_t)row * a.d_k;
+        const float *kr = Kg + (size_t)row * a.k_sr;
         float dot = 0.f;
         for (int j = lane; j < a.d_k; j += 32) dot = fmaf(sq[j], kr[j], dot);
 #pragma unroll
@@ -51,7 +51,7 @@ __global__ void __launch_bounds__(kGenericWarps * 32) generic_decode_kernel(cons
         const float p = exp2_diff(dot, m_new);
         l = fmaf(l, alpha, p);
         m = m_new;
-        const float *vr = Vg + (size_t)row * a.d_v;
+        const float *vr = Vg + (size_t)row * a.v_sr;
 #pragma unroll
         for (int i = 0; i < kGenericDvSlots; ++i) {
             const int d = lane + 32 * i;
@@ -117,27 +117,31 @@ __global__ void check_lens_kernel(const int32_t *lens, int bias, int batch, int 
     }
 }
 
+// Element strides of one cache: batch item, kv head, row.
+struct CacheStrides { long long sb, sh, sr; };
+
 // Cache append, eqs. (4),(5): one thread per 32-bit word of the new K row and V row of
 // one (batch, kv head); words are moved as raw bit patterns.
 __global__ void __launch_bounds__(256) kv_append_kernel(uint32_t *K, uint32_t *V,
                                                         const uint32_t *k_new,
                                                         const uint32_t *v_new,
                                                         const int32_t *pos, int batch, int h_kv,
-                                                        int n_max, int d_k, int d_v)
+                                                        int n_max, int d_k, int d_v,
+                                                        CacheStrides ks, CacheStrides vs)
 {
     const int per = d_k + d_v;
     const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= (long long)batch * h_kv * per) return;
     const int w = (int)(t % per);
     const long long slab = t / per;                     // b * h_kv + h
-    const int b = (int)(slab / h_kv);
+    const int b = (int)(slab / h_kv), h = (int)(slab % h_kv);
     const int p = pos[b];
     if (p < 0 || p >= n_max) {
-        if (w == 0 && slab % h_kv == 0) raise_status(MOA_STATUS_APPEND_RANGE);
+        if (w == 0 && h == 0) raise_status(MOA_STATUS_APPEND_RANGE);
         return;
     }
-    if (w < d_k) K[((size_t)slab * n_max + p) * d_k + w] = k_new[(size_t)slab * d_k + w];
-    else V[((size_t)slab * n_max + p) * d_v + (w - d_k)] = v_new[(size_t)slab * d_v + (w - d_k)];
+    if (w < d_k) K[(size_t)b * ks.sb + (size_t)h * ks.sh + (size_t)p * ks.sr + w] = k_new[(size_t)slab * d_k + w];
+    else V[(size_t)b * vs.sb + (size_t)h * vs.sh + (size_t)p * vs.sr + (w - d_k)] = v_new[(size_t)slab * d_v + (w - d_k)];
 }
 
 // lens[b] += delta.  With `guard_n_max` > 0 the increment is applied only to lengths in

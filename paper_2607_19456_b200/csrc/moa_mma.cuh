@@ -187,15 +187,17 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
     const int my_d = is_pv ? D : DK;            // row length of this warp's operand
     const float *my_new = is_pv ? a.v_new : a.k_new;
     float *my_cache = is_pv ? a.Vw : a.Kw;
+    const long long my_sb = is_pv ? a.v_sb : a.k_sb, my_sh = is_pv ? a.v_sh : a.k_sh, my_sr = is_pv ? a.v_sr : a.k_sr;
 
     // ---- load side: this pair's tiles are c0+pair, c0+pair+P, ... ------------------------
     long long jl = c0 + pair;
     int kl = 0;
     Cursor lc = cursor_at<R>(a, (jl < c1) ? jl : c0, pref);
     size_t slab = 0;                           // stored (batch, kv head) of the unit under lc
+    int hs = 0;                                // its stored kv head
     bool writes_new = false;                   // this virtual head stores the appended row
     auto load_unit_changed = [&]() {
-        const int hs = lc.h / a.kv_share;
+        hs = lc.h / a.kv_share;
         slab = (size_t)lc.b * h_stored + hs;
         writes_new = (a.k_new != nullptr) && (lc.h == hs * a.kv_share);
     };
@@ -206,25 +208,26 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
             load_unit_changed();
         }
         const int row0 = (int)(jl - lc.first) * R;
-        const size_t row = slab * (size_t)a.n_max + row0;
         if (lane == 0) {
             const int stage = kl % S;
             const uint32_t bar = my_bar0 + 8u * stage;
-            // A box is always transferred whole (rows past the end of the cache read as zero;
-            // rows past the end of the unit belong to the next unit and are masked later).
+            // A box is always transferred whole: rows past the slab's capacity read as zero, rows
+            // past the live length are masked later.
             const uint32_t dst = smem_u32(my_ring + (size_t)stage * C::STAGE_FLOATS);
             mbar_expect_tx(bar, PAIRED ? (uint32_t)R * my_d * 4u : (uint32_t)C::STAGE_FLOATS * 4u);
-            tc::tma_load_3d(dst, my_map, 0, (int)row, 0, bar);
-            if (!PAIRED) tc::tma_load_3d(dst + R * D * 4u, &tmapV, 0, (int)row, 0, bar);
+            tc::tma_load_5d(dst, my_map, 0, row0, 0, hs, lc.b, bar);
+            if (!PAIRED) tc::tma_load_5d(dst + R * D * 4u, &tmapV, 0, row0, 0, hs, lc.b, bar);
         }
         // Fused append: the unit's last row is the token being appended.  The warp that fetches
         // the tile holding it also stores it into the cache (K by the score warp, V by the other);
         // the tile's copy of that row is replaced from k_new / v_new before use.
         if (writes_new && row0 + R >= lc.len && lane * 4 < my_d) {
-            const size_t dst = (slab * (size_t)a.n_max + (size_t)(lc.len - 1)) * my_d + lane * 4;
+            const size_t dst = (size_t)lc.b * my_sb + (size_t)hs * my_sh + (size_t)(lc.len - 1) * my_sr + lane * 4;
             *reinterpret_cast<float4 *>(my_cache + dst) = *reinterpret_cast<const float4 *>(my_new + slab * my_d + lane * 4);
-            if (!PAIRED)
-                *reinterpret_cast<float4 *>(a.Vw + dst) = *reinterpret_cast<const float4 *>(a.v_new + slab * D + lane * 4);
+            if (!PAIRED) {
+                const size_t dstv = (size_t)lc.b * a.v_sb + (size_t)hs * a.v_sh + (size_t)(lc.len - 1) * a.v_sr + lane * 4;
+                *reinterpret_cast<float4 *>(a.Vw + dstv) = *reinterpret_cast<const float4 *>(a.v_new + slab * D + lane * 4);
+            }
         }
         jl += P;
         ++kl;

@@ -141,8 +141,10 @@ __global__ void __launch_bounds__(C::THREADS, 1) stream_decode_kernel(const Deco
         // k_new / v_new (never from the cache), and this warp also stores it into the cache.
         const bool has_new = (a.k_new != nullptr) && (row0 + nr == lc.len);
         const int nr_cache = has_new ? nr - 1 : nr;
-        const size_t slab = (size_t)lc.b * h_stored + lc.h / a.kv_share;
-        const size_t row = slab * (size_t)a.n_max + row0;
+        const int hs = lc.h / a.kv_share;      // stored kv head
+        const size_t slab = (size_t)lc.b * h_stored + hs;
+        const float *Ksrc = a.K + (size_t)lc.b * a.k_sb + (size_t)hs * a.k_sh + (size_t)row0 * D;
+        const float *Vsrc = a.V + (size_t)lc.b * a.v_sb + (size_t)hs * a.v_sh + (size_t)row0 * D;
         if (lane == 0) {
             const int stage = kl % S;
             const uint32_t bar = my_bar0 + 8u * stage;
@@ -150,8 +152,8 @@ __global__ void __launch_bounds__(C::THREADS, 1) stream_decode_kernel(const Deco
             const uint32_t bytes = (uint32_t)nr_cache * D * 4u;
             mbar_expect_tx(bar, 2u * (uint32_t)nr * D * 4u);
             if (nr_cache > 0) {
-                bulk_g2s(dst, a.K + row * D, bytes, bar);
-                bulk_g2s(dst + R * D * 4u, a.V + row * D, bytes, bar);
+                bulk_g2s(dst, Ksrc, bytes, bar);
+                bulk_g2s(dst + R * D * 4u, Vsrc, bytes, bar);
             }
             if (has_new) {
                 bulk_g2s(dst + bytes, a.k_new + slab * D, D * 4u, bar);
@@ -159,10 +161,10 @@ __global__ void __launch_bounds__(C::THREADS, 1) stream_decode_kernel(const Deco
             }
         }
         if (has_new && (lc.h % a.kv_share) == 0 && lane < LPR) {
-            const size_t dst_row = (row + nr_cache) * D + lane * 4;
-            *reinterpret_cast<float4 *>(a.Kw + dst_row) =
+            const size_t in_unit = (size_t)nr_cache * D + lane * 4;
+            *reinterpret_cast<float4 *>(a.Kw + (Ksrc - a.K) + in_unit) =
                 *reinterpret_cast<const float4 *>(a.k_new + slab * D + lane * 4);
-            *reinterpret_cast<float4 *>(a.Vw + dst_row) =
+            *reinterpret_cast<float4 *>(a.Vw + (Vsrc - a.V) + in_unit) =
                 *reinterpret_cast<const float4 *>(a.v_new + slab * D + lane * 4);
         }
         jl += W;
