@@ -12,6 +12,7 @@
 #include "moa_stream.cuh"
 #include "moa_mma.cuh"
 #include "moa_grouped.cuh"
+#include "moa_grouped64.cuh"
 
 namespace moa {
 
@@ -471,6 +472,36 @@ static cudaError_t launch_grouped_cfg(const CUtensorMap &mk, const CUtensorMap &
     return cudaGetLastError();
 }
 
+static int g_grouped_operands = 0;   // MOA_OPT_GROUPED_OPERANDS
+
+// Groups of 64 heads with Q and P in tensor memory; same arguments and partial format as
+// the shared-memory-operand kernel, so the combine kernel is shared.
+static cudaError_t launch_grouped64(const CUtensorMap &mk, const CUtensorMap &mv, const CUtensorMap &mkt,
+                                    const CUtensorMap &mvt, const GroupedArgs &ga, int grid, cudaStream_t st)
+{
+    using C = Grouped64Cfg;
+    static bool attr_set[kMaxDevices] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (!attr_set[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(grouped64_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)C::SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        attr_set[dev] = true;
+    }
+    {
+        TimedLaunch t(st);
+        grouped64_decode_kernel<<<grid, C::THREADS, C::SMEM_BYTES, st>>>(mk, mv, mkt, mvt, ga);
+    }
+    count_launch();
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const long long warps = (long long)ga.batch * ga.h_q;
+    grouped_combine_kernel<64><<<(int)((warps + 3) / 4), 128, 0, st>>>(ga);
+    count_launch();
+    return cudaGetLastError();
+}
+
 static cudaError_t launch_generic(const DecodeArgs &a, cudaStream_t st)
 {
     const size_t smem = sizeof(float) * ((size_t)a.d_k + (size_t)kGenericWarps * a.d_v + 2 * kGenericWarps);
@@ -607,6 +638,7 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
         }
         if (gplan.GH == 16) e = launch_grouped_cfg<16>(mk, mv, mkt, mvt, ga, grid, st);
         else if (gplan.GH == 32) e = launch_grouped_cfg<32>(mk, mv, mkt, mvt, ga, grid, st);
+        else if (gplan.share == 1 && g_grouped_operands == 0) e = launch_grouped64(mk, mv, mkt, mvt, ga, grid, st);
         else e = launch_grouped_cfg<64>(mk, mv, mkt, mvt, ga, grid, st);
         if (e == cudaSuccess && fused != nullptr && fused->lens_rw != nullptr) {
             lens_add_kernel<<<(batch + 127) / 128, 128, 0, st>>>(fused->lens_rw, batch, 1, n_max);
@@ -1033,6 +1065,11 @@ int moa_set_option(int option, int value)
     if (option == MOA_OPT_GROUPED_HEADS) {
         if (value != 0 && value != 16 && value != 32 && value != 64) return MOA_ERR_INVALID;
         g_grouped_heads = value;
+        return MOA_OK;
+    }
+    if (option == MOA_OPT_GROUPED_OPERANDS) {
+        if (value != 0 && value != 1) return MOA_ERR_INVALID;
+        g_grouped_operands = value;
         return MOA_OK;
     }
     if (option == MOA_OPT_DEPENDENT_LAUNCH) {

@@ -1,0 +1,470 @@
+// moa_grouped64.cuh -- tensor-core decode kernel for groups of 64 query heads per K/V head
+// (MQA), with the small operands (Q, P) resident in tensor memory.
+//
+// Steps I and III of Algorithm 1 (eqs. (1),(3)) per tile of 128 cached rows, heads on the
+// M axis:
+//     S[heads x rows] = Q[heads x d] * K_tile^T,      O[heads x d] += P[heads x rows] * V_tile
+// on tcgen05.mma (kind::tf32) with the three-term split x = hi + lo that keeps fp32 accuracy.
+// The A operand is read from tensor memory: its 128 lanes hold, for every head, one lane with
+// the hi part and one lane with the lo part of that head's row ("stacked" operand), so that
+//     [Q_hi; Q_lo] * K_hi^T  gives  Q_hi*K_hi  in the hi lanes and  Q_lo*K_hi  in the lo lanes,
+//     [Q_hi; Q_lo] * K_lo^T  gives  Q_hi*K_lo  in the hi lanes (and the negligible lo*lo term),
+// and likewise for [P_hi; P_lo] and V.  Only the streamed operand (K and V chunks, the B
+// operand) lives in shared memory, where it is read once as loaded (the tensor core keeps
+// exactly the hi part of an fp32 word) and once after an in-place conversion to its lo part.
+// Compared with both operands in shared memory this halves the operand traffic of every
+// product and frees 128 KB for the chunk ring, which is what bounds that arrangement.
+//
+// Lanes: quadrant w (lanes 32w..32w+31) holds heads 16w..16w+15; lane 32w+j (j < 16) the hi
+// part of head 16w+j, lane 32w+16+j its lo part.  A thread of the softmax group owns one
+// lane, so the two parts of a head meet by one shuffle inside a warp.
+//
+// Tensor memory (512 columns): Q (128), two score/probability regions (128 each; the
+// probabilities of a tile overwrite its scores), O (128).  The tensor core accumulates with
+// truncation, so chains are kept short: the scores of a tile are a chain of 32 steps, and the
+// weighted sum of every tile starts from zero and is folded into fp32 running values held in
+// registers (online softmax, eq. (2) with a running maximum per head).
+//
+// A thread that issues tcgen05.mma cannot look at a barrier without draining the tensor pipe
+// (measured: one shared-memory read between two products costs ~170 cycles of tensor time),
+// so the issuer asks once per batch, on barriers that collect a whole batch: all four chunks
+// of a group landed -> 16 hi products; the first two conversions done -> 8 lo products; the
+// other two -> 8 more.  Nothing the
+// softmax group does is on the tensor core's critical path: while it works on tile t the
+// tensor core multiplies tile t+1's K chunks and tile t-1's V chunks.
+//
+// Roles (736 threads): warp 0 TMA producer, warp 1 MMA issuer (and owner of the tensor
+// memory allocation), warp 22 batch scheduler, warps 4-19 softmax (warp w: lane quadrant w % 4, columns 32 * ((w-4)/4)
+// .. +31 of a 128-column region), warps 2, 3, 20, 21 turn chunks into their lo parts.  Every
+// hand-off is an mbarrier; every wait is bounded.
+#pragma once
+
+#include "moa_grouped.cuh"
+
+namespace moa {
+
+// Bounded wait for the roles that are not on the tensor core's critical path: try_wait lets
+// the hardware suspend the thread, so a waiting warp takes no issue slots from the issuer.
+__device__ __forceinline__ bool wait_suspended(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+{
+    for (uint32_t it = 0; it < kWaitLimit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 15u) == 15u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    raise_status(MOA_STATUS_WAIT_TIMEOUT);
+    return false;
+}
+
+__device__ __forceinline__ uint4 lds_volatile_v4(uint32_t addr)
+{
+    uint4 v;
+    asm volatile("ld.volatile.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void sts_volatile_v4(uint32_t addr, uint32_t x, uint32_t y, uint32_t z, uint32_t w)
+{
+    asm volatile("st.volatile.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+}
+
+struct Grouped64Cfg {
+    static constexpr int GH = 64;
+    static constexpr int D = 128;
+    static constexpr int TILE = 128;
+    static constexpr int NBUF = 13;                // 16 KB chunk buffers
+    static constexpr int NG = 4;                   // groups of four chunks with barriers of their own (> NBUF / 4)
+    static constexpr int CHUNK = 16384;
+    static constexpr int THREADS = 736;            // 23 warps
+    static constexpr int QN = 4;                   // batch descriptors queued between scheduler and issuer
+    static constexpr int CONV_WARPS = 4;
+    static constexpr int SOFT_WARPS = 16;
+    static constexpr int PS = D + 4;
+    static constexpr uint32_t OFF_RING = 0;
+    static constexpr uint32_t OFF_MX = OFF_RING + NBUF * CHUNK;     // [2 tiles][4 column quarters][64 heads] tile maxima
+    static constexpr uint32_t OFF_LX = OFF_MX + 2 * 4 * 64 * 4;     // [4 column quarters][64 heads] sums
+    static constexpr uint32_t OFF_BAR = OFF_LX + 4 * 64 * 4;
+    static constexpr int NBAR = 2 * NBUF + 2 * NG + 2 + 2 + 1 + 1;
+    static constexpr uint32_t OFF_TMEM = OFF_BAR + NBAR * 8;
+    static constexpr uint32_t OFF_ABORT = OFF_TMEM + 4;
+    static constexpr uint32_t OFF_SHARE = OFF_ABORT + 4;            // flat mode: unit, first CTA, CTA count
+    static constexpr uint32_t OFF_QCNT = OFF_SHARE + 16;            // batches published / batches taken
+    static constexpr uint32_t OFF_QUEUE = (OFF_QCNT + 8 + 15) / 16 * 16;   // [QN][16] words
+    static constexpr size_t SMEM_BYTES = OFF_QUEUE + QN * 64;
+};
+
+__global__ void __launch_bounds__(Grouped64Cfg::THREADS, 1)
+grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant__ CUtensorMap tmapV,
+                        const __grid_constant__ CUtensorMap tmapKt, const __grid_constant__ CUtensorMap tmapVt,
+                        const GroupedArgs a)
+{
+    using C = Grouped64Cfg;
+    constexpr int GH = C::GH, NBUF = C::NBUF, NG = C::NG, PS = C::PS;
+    extern __shared__ __align__(1024) unsigned char smem_g64[];
+    unsigned char *const smem = smem_g64;
+    float *mx = reinterpret_cast<float *>(smem + C::OFF_MX);
+    float *lx = reinterpret_cast<float *>(smem + C::OFF_LX);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + C::OFF_BAR);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + C::OFF_TMEM);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + C::OFF_ABORT);
+    int *s_share = reinterpret_cast<int *>(smem + C::OFF_SHARE);
+    volatile int *q_ready = reinterpret_cast<volatile int *>(smem + C::OFF_QCNT);
+    volatile int *q_taken = q_ready + 1;
+    const uint32_t queue = smem_u32(smem) + C::OFF_QUEUE;       // 64 bytes per batch
+
+    const uint32_t sRing = smem_u32(smem) + C::OFF_RING;
+    // Per ring buffer (every role sees every use of every buffer, so one parity bit per use):
+    auto bar_hi = [&](int b) { return smem_u32(&bars[b]); };                 // the chunk's hi product is complete
+    auto bar_empty = [&](int b) { return smem_u32(&bars[NBUF + b]); };       // its lo product is complete
+    // Per group of four chunks (group g uses slot g % NG; the ring holds fewer than NG groups):
+    auto bar_gfull = [&](int g) { return smem_u32(&bars[2 * NBUF + g]); };            // all four chunks landed
+    auto bar_glo = [&](int g) { return smem_u32(&bars[2 * NBUF + NG + g]); };         // all four lo parts in place
+    auto bar_sfull = [&](int s) { return smem_u32(&bars[2 * NBUF + 2 * NG + s]); };   // scores of a tile complete
+    auto bar_pfull = [&](int s) { return smem_u32(&bars[2 * NBUF + 2 * NG + 2 + s]); };   // probabilities stored
+    const uint32_t bar_ofull = smem_u32(&bars[2 * NBUF + 2 * NG + 4]);                // weighted sum of a tile complete
+    const uint32_t bar_ofree = smem_u32(&bars[2 * NBUF + 2 * NG + 5]);                // ... and folded
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    int split = (int)blockIdx.x % a.splits;
+    int sunit = (int)blockIdx.x / a.splits;                       // stored (batch, kv head)
+    int splits_u = a.splits;
+    if (a.flat) {                                  // warp 0 walks the lengths, all take its answer
+        if (warp == 0) {
+            const FlatShare f = flat_share(a, (int)gridDim.x, (int)blockIdx.x, -1, lane);
+            if (lane == 0) { s_share[0] = f.unit; s_share[1] = f.first; s_share[2] = f.count; }
+        }
+        __syncthreads();
+        if (s_share[0] < 0) return;
+        sunit = s_share[0]; split = (int)blockIdx.x - s_share[1]; splits_u = s_share[2];
+    }
+    const int b = sunit / a.h_kv_stored, h = sunit % a.h_kv_stored;
+    const int unit = sunit;                                         // tensor-map coordinate
+    const int len_b = grouped_len(a, b);           // 0: out-of-range length, the item is skipped
+    const int tiles_total = (len_b + C::TILE - 1) / C::TILE;
+    const int tiles_per_split = a.seq_lens ? (tiles_total + splits_u - 1) / splits_u : a.tiles_per_split;
+    const int tile0 = split * tiles_per_split;
+    int T = tiles_total - tile0;
+    if (T > tiles_per_split) T = tiles_per_split;
+    if (T <= 0) return;                            // an empty split (uniform for the CTA)
+    const int tail_t = (a.tailK != nullptr) ? tiles_total - 1 - tile0 : -1;
+    const int row_base = tile0 * C::TILE;
+
+    // ---- set-up --------------------------------------------------------------------------
+    if (tid == 0) {
+        for (int i = 0; i < NBUF; ++i) { mbar_init(bar_hi(i), 1); mbar_init(bar_empty(i), 1); }
+        for (int g = 0; g < NG; ++g) {
+            mbar_init(bar_gfull(g), 4);            // one arrival (with its byte count) per chunk
+            mbar_init(bar_glo(g), 4 * C::CONV_WARPS);
+        }
+        for (int i = 0; i < 2; ++i) { mbar_init(bar_sfull(i), 1); mbar_init(bar_pfull(i), C::SOFT_WARPS); }
+        mbar_init(bar_ofull, 1); mbar_init(bar_ofree, C::SOFT_WARPS);
+        mbar_fence_init();
+        *abort_flag = 0;
+        *q_ready = 0; *q_taken = 0;
+        tc::prefetch_tmap(&tmapK);
+        tc::prefetch_tmap(&tmapV);
+        if (a.tailK != nullptr) { tc::prefetch_tmap(&tmapKt); tc::prefetch_tmap(&tmapVt); }
+    }
+    if (warp == 1) tc::tmem_alloc(smem_u32(tmem_slot), 512);
+    tc::fence_before_sync();
+    __syncthreads();
+    tc::fence_after_sync();
+    const uint32_t tmem = *tmem_slot;
+    const uint32_t tQ = tmem, tO = tmem + 384u;
+    auto tSP_of = [tmem](int t) -> uint32_t { return tmem + 128u + (uint32_t)(t & 1) * 128u; };
+
+    // softmax-group coordinates (also used for the Q operand, which that group writes)
+    const bool is_soft = warp >= 4 && warp < 20;
+    const int qd = warp & 3;                       // lane quadrant
+    const int sub = (warp - 4) >> 2;               // which 32 columns of a 128-column region
+    const int col0 = 32 * sub;
+    const uint32_t lane_addr = (uint32_t)(qd * 32) << 16;
+    const int head = 16 * qd + (lane & 15);
+    const bool is_lo = (lane & 16) != 0;
+    if (is_soft) {
+        // Q operand: this lane's part (hi or lo) of (scale * log2 e) * q[head], columns = features
+        const float *qb = a.q + ((size_t)b * a.h_q + (size_t)h * GH + head) * 128 + col0;
+        uint32_t v[32];
+#pragma unroll
+        for (int i = 0; i < 32; i += 4) {
+            const float4 x4 = *reinterpret_cast<const float4 *>(qb + i);
+            const float xs[4] = {x4.x * a.qscale, x4.y * a.qscale, x4.z * a.qscale, x4.w * a.qscale};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float hi = tf32_hi(xs[k]);
+                v[i + k] = __float_as_uint(is_lo ? xs[k] - hi : hi);
+            }
+        }
+        tc::tmem_st32(tQ + lane_addr + col0, v);
+        tc::tmem_st_wait();
+    }
+    tc::fence_before_sync();
+    __syncthreads();
+    tc::fence_after_sync();
+
+    if (warp == 0) {
+        // ================= TMA producer =================
+        if (lane == 0) {
+            for (ChunkSeq s(T); !s.done; s.next()) {
+                const int buf = s.seq % NBUF, use = s.seq / NBUF;
+                if (use > 0 && !wait_suspended(bar_empty(buf), (uint32_t)(use - 1) & 1u, abort_flag)) break;
+                const uint32_t dst = sRing + (uint32_t)buf * C::CHUNK;
+                const uint32_t fb = bar_gfull((s.seq >> 2) % NG);
+                mbar_expect_tx(fb, C::CHUNK);
+                const bool tail = (s.t == tail_t);
+                const int row = tail ? 0 : row_base + s.t * C::TILE;
+                if (s.is_k) {
+                    tc::tma_load_3d(dst, tail ? &tmapKt : &tmapK, 32 * s.c, row, unit, fb);
+                } else {
+                    for (int dg = 0; dg < 4; ++dg)
+                        tc::tma_load_3d(dst + dg * 4096, tail ? &tmapVt : &tmapV, 32 * dg, row + 32 * s.c, unit, fb);
+                }
+            }
+        }
+    } else if (warp == 22) {
+        // ================= batch scheduler (one thread) =================
+        // The thread that issues tcgen05.mma has about 64 cycles between two products before the
+        // tensor pipe runs dry, so everything else the issue needs is done here: the order of the
+        // batches, their descriptors and barrier addresses, and the waiting.  Batches of 16
+        // products, in the order
+        //     K_hi(0) K_lo(0)  [K_hi(t+1) V_hi(t) K_lo(t+1) V_lo(t)] for t = 0..T-2  V_hi(T-1) V_lo(T-1):
+        // between the hi and the lo batch of a group runs a batch of the other operand, which is
+        // the time the converters have.  A batch is published (16 words) once its barriers are
+        // complete; the queue holds QN of them.
+        if (lane == 0) {
+            const uint32_t idesc_k = tc::idesc_tf32(128, 128, false, false);   // B = K chunk, K-major
+            const uint32_t idesc_v = tc::idesc_tf32(128, 128, false, true);    // B = V chunk, MN-major
+            // descriptor words: [addr>>4 | lbo>>4 << 16] and [sbo>>4 | version << 14 | layout << 29]
+            const uint32_t k_hiword = 64u | (1u << 14) | (2u << 29), v_hiword = 32u | (1u << 14) | (1u << 29);
+            const uint32_t k_base = (sRing >> 4) | (1u << 16), v_base = (sRing >> 4) | (256u << 16);
+            const int nbatch = 4 * T;
+            bool ok = true;
+            for (int i = 0; ok && i < nbatch; ++i) {
+                bool is_k, is_hi;
+                int t;
+                if (i < 2) { is_k = true; t = 0; is_hi = (i == 0); }
+                else {
+                    const int jj = i - 2, r = jj & 3;
+                    t = jj >> 2;
+                    if (t >= T - 1) { is_k = false; t = T - 1; is_hi = (r == 0); }
+                    else { is_k = (r == 0 || r == 2); is_hi = (r < 2); if (is_k) t += 1; }
+                }
+                const int g = is_k ? (t == 0 ? 0 : 2 * t - 1) : (t < T - 1 ? 2 * t + 2 : 2 * T - 1);
+                const int gs = g % NG;
+                const uint32_t gpar = (uint32_t)(g / NG) & 1u;
+                uint32_t w[16];
+                w[0] = is_k ? tSP_of(t) : tO;                       // D
+                w[1] = is_k ? tQ : tSP_of(t);                       // A
+                w[2] = is_k ? k_hiword : v_hiword;
+                w[3] = is_k ? 2u : 64u;                             // descriptor step per k-step
+                w[4] = is_k ? idesc_k : idesc_v;
+                w[5] = is_hi ? 0u : 1u;                             // accumulate flag of the first product
+                w[6] = is_hi ? 0u : (is_k ? bar_sfull(t & 1) : bar_ofull);   // barrier of the whole tile product
+                w[7] = 0u;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const int buf = (4 * g + c) % NBUF;
+                    w[8 + c] = (is_k ? k_base : v_base) + (uint32_t)buf * (C::CHUNK >> 4);
+                    w[12 + c] = is_hi ? bar_hi(buf) : bar_empty(buf);
+                }
+                // what the batch needs: hi products the four chunks (a weighted sum also the tile's
+                // probabilities and the fold of the previous tile's weighted sum, which the softmax
+                // group does after storing the probabilities); lo products the four conversions
+                if (is_hi) {
+                    ok = wait_or_abort(bar_gfull(gs), gpar, abort_flag);
+                    if (ok && !is_k)
+                        ok = (t > 0) ? wait_or_abort(bar_ofree, (uint32_t)(t - 1) & 1u, abort_flag)
+                                     : wait_or_abort(bar_pfull(0), 0u, abort_flag);
+                } else {
+                    ok = wait_or_abort(bar_glo(gs), gpar, abort_flag);
+                }
+                for (uint32_t it = 0; ok && *q_taken + C::QN <= i; ++it)       // a free queue slot
+                    if (it >= kWaitLimit || ((it & 255u) == 255u && *abort_flag)) {
+                        if (it >= kWaitLimit) { *abort_flag = 1; raise_status(MOA_STATUS_WAIT_TIMEOUT); }
+                        ok = false;
+                    }
+                if (!ok) break;
+                const uint32_t slot = queue + (uint32_t)(i % C::QN) * 64u;
+                sts_volatile_v4(slot, w[0], w[1], w[2], w[3]);
+                sts_volatile_v4(slot + 16u, w[4], w[5], w[6], w[7]);
+                sts_volatile_v4(slot + 32u, w[8], w[9], w[10], w[11]);
+                sts_volatile_v4(slot + 48u, w[12], w[13], w[14], w[15]);
+                __threadfence_block();
+                *q_ready = i + 1;
+            }
+        }
+    } else if (warp == 1) {
+        // ================= MMA issuer (one thread) =================
+        if (lane == 0) {
+            const int nbatch = 4 * T;
+            int have = 0;
+            bool ok = true;
+            uint4 n0, n1, n2, n3;                  // the next batch, fetched ahead
+            bool fetched = false;
+            for (int i = 0; ok && i < nbatch; ++i) {
+                if (!fetched) {
+                    for (uint32_t it = 0; have <= i; ++it) {
+                        have = *q_ready;
+                        if (it >= kWaitLimit || ((it & 255u) == 255u && *abort_flag)) {
+                            if (it >= kWaitLimit) { *abort_flag = 1; raise_status(MOA_STATUS_WAIT_TIMEOUT); }
+                            ok = false;
+                            break;
+                        }
+                    }
+                    if (!ok) break;
+                    __threadfence_block();
+                    const uint32_t slot = queue + (uint32_t)(i % C::QN) * 64u;
+                    n0 = lds_volatile_v4(slot); n1 = lds_volatile_v4(slot + 16u);
+                    n2 = lds_volatile_v4(slot + 32u); n3 = lds_volatile_v4(slot + 48u);
+                    *q_taken = i + 1;
+                }
+                const uint32_t d = n0.x, a0 = n0.y, hiword = n0.z, step = n0.w, idesc = n1.x, acc0 = n1.y, final_bar = n1.z;
+                const uint32_t bdesc[4] = {n2.x, n2.y, n2.z, n2.w}, done[4] = {n3.x, n3.y, n3.z, n3.w};
+                fetched = false;
+                tc::fence_after_sync();
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    if (c == 3 && i + 1 < nbatch) {    // fetch the next batch while this chunk is multiplied
+                        have = *q_ready;
+                        if (have > i + 1) {
+                            __threadfence_block();
+                            const uint32_t slot = queue + (uint32_t)((i + 1) % C::QN) * 64u;
+                            n0 = lds_volatile_v4(slot); n1 = lds_volatile_v4(slot + 16u);
+                            n2 = lds_volatile_v4(slot + 32u); n3 = lds_volatile_v4(slot + 48u);
+                            *q_taken = i + 2;
+                            fetched = true;
+                        }
+                    }
+#pragma unroll
+                    for (uint32_t ks = 0; ks < 4; ++ks)
+                        tc::mma_tf32_ts(d, a0 + 32u * c + 8u * ks, tc::pack64(bdesc[c] + ks * step, hiword), idesc,
+                                        (c == 0 && ks == 0) ? acc0 : 1u);
+                    tc::mma_commit(done[c]);
+                }
+                if (final_bar != 0u) tc::mma_commit(final_bar);
+            }
+        }
+    } else if (is_soft) {
+        // ================= softmax group: thread = (lane of the stacked operand, 32 columns) ==========
+        float Om[32];                              // running weighted sum: this lane's part, features col0..col0+31
+#pragma unroll
+        for (int i = 0; i < 32; ++i) Om[i] = 0.f;
+        float m_run = -INFINITY, l_run = 0.f, alpha_prev = 0.f;
+        bool ok = true;
+        auto fold = [&](float alpha) {             // Om = alpha * Om + (weighted sum of the last tile)
+            uint32_t o[32];
+            tc::tmem_ld32(tO + lane_addr + col0, o);
+            tc::tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) Om[i] = fmaf(Om[i], alpha, __uint_as_float(o[i]));
+        };
+        for (int t = 0; t < T; ++t) {
+            ok = ok && wait_suspended(bar_sfull(t & 1), (uint32_t)(t >> 1) & 1u, abort_flag);
+            if (named_or(1 + qd, 128, !ok)) { ok = false; break; }    // the four warps of a quadrant leave together
+            tc::fence_after_sync();
+            const uint32_t tSP = tSP_of(t) + lane_addr + col0;
+            const int row0 = row_base + t * C::TILE + col0;
+            // scores of this lane's head against 32 cached rows: the two lanes of a head hold the
+            // terms of its hi and of its lo query part; each adds the other's
+            uint32_t x[32];
+            tc::tmem_ld32(tSP, x);
+            tc::tmem_ld_wait();
+            float vmax = -INFINITY;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const float mine = __uint_as_float(x[i]);
+                float sc = mine + __shfl_xor_sync(0xffffffffu, mine, 16);
+                if (row0 + i >= len_b) sc = -INFINITY;
+                vmax = fmaxf(vmax, sc);
+                x[i] = __float_as_uint(sc);
+            }
+            // maximum over the tile: the other columns belong to the other warps of the quadrant
+            float *mxt = mx + (t & 1) * 256;
+            if (!is_lo) mxt[sub * 64 + head] = vmax;
+            named_sync(1 + qd, 128);
+            const float m_new = fmaxf(fmaxf(m_run, mxt[head]), fmaxf(fmaxf(mxt[64 + head], mxt[128 + head]), mxt[192 + head]));
+            const float alpha = exp2_diff(m_run, m_new);
+            m_run = m_new;
+            // probabilities, this lane's part, over the scores
+            float lsum = 0.f;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const float p = fast_exp2(__uint_as_float(x[i]) - m_new);
+                lsum += p;
+                const float ph = tf32_hi(p);
+                x[i] = __float_as_uint(is_lo ? p - ph : ph);
+            }
+            tc::tmem_st32(tSP, x);
+            tc::tmem_st_wait();
+            tc::fence_before_sync();
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive(bar_pfull(t & 1));
+            l_run = fmaf(l_run, alpha, lsum);
+            // fold the previous tile's weighted sum into the running values
+            if (t > 0) {
+                ok = wait_suspended(bar_ofull, (uint32_t)(t - 1) & 1u, abort_flag);
+                if (ok) {
+                    tc::fence_after_sync();
+                    fold(alpha_prev);
+                    tc::fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) tc::mbar_arrive(bar_ofree);
+                }
+            }
+            alpha_prev = alpha;
+        }
+        // ---- epilogue: last fold, then this split's partial (m, l, o) per head
+        if (ok) ok = wait_suspended(bar_ofull, (uint32_t)(T - 1) & 1u, abort_flag);
+        if (named_or(1 + qd, 128, !ok)) ok = false;
+        if (ok) {
+            tc::fence_after_sync();
+            fold(alpha_prev);
+            if (!is_lo) lx[sub * 64 + head] = l_run;
+            named_sync(1 + qd, 128);
+            float *slot = (a.flat ? a.ws + ((size_t)blockIdx.x * GH) * PS
+                                  : a.ws + ((((size_t)b * a.h_kv + h) * a.splits + split) * GH) * PS) + (size_t)head * PS;
+#pragma unroll
+            for (int i = 0; i < 32; i += 4) {
+                float4 v;
+                v.x = Om[i] + __shfl_xor_sync(0xffffffffu, Om[i], 16);
+                v.y = Om[i + 1] + __shfl_xor_sync(0xffffffffu, Om[i + 1], 16);
+                v.z = Om[i + 2] + __shfl_xor_sync(0xffffffffu, Om[i + 2], 16);
+                v.w = Om[i + 3] + __shfl_xor_sync(0xffffffffu, Om[i + 3], 16);
+                if (!is_lo) *reinterpret_cast<float4 *>(slot + col0 + i) = v;
+            }
+            if (sub == 0 && !is_lo) {
+                slot[128] = m_run;
+                slot[129] = (lx[head] + lx[64 + head]) + (lx[128 + head] + lx[192 + head]);
+            }
+        }
+    } else {
+        // ================= converters: chunk -> its lo part, in place =================
+        constexpr int TT = C::CONV_WARPS * 32;                         // 128 threads
+        constexpr int PER = (C::CHUNK / 16) / TT;                      // float4 every thread handles
+        const int ct = ((warp < 4) ? warp - 2 : warp - 18) * 32 + lane;
+        bool ok = true;
+        for (ChunkSeq s(T); ok && !s.done; s.next()) {
+            const int buf = s.seq % NBUF, use = s.seq / NBUF;
+            ok = wait_suspended(bar_hi(buf), (uint32_t)use & 1u, abort_flag);
+            if (!ok) break;
+            float4 *p = reinterpret_cast<float4 *>(smem + C::OFF_RING + (uint32_t)buf * C::CHUNK);
+            float4 v[PER];
+#pragma unroll
+            for (int i = 0; i < PER; ++i) v[i] = p[ct + i * TT];
+#pragma unroll
+            for (int i = 0; i < PER; ++i) {
+                v[i].x -= tf32_hi(v[i].x); v[i].y -= tf32_hi(v[i].y);
+                v[i].z -= tf32_hi(v[i].z); v[i].w -= tf32_hi(v[i].w);
+                p[ct + i * TT] = v[i];
+            }
+            tc::fence_async_smem();
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive(bar_glo((s.seq >> 2) % NG));
+        }
+    }
+
+    tc::fence_before_sync();
+    __syncthreads();
+    if (warp == 1) tc::tmem_dealloc(tmem, 512);
+}
+
+}  // namespace moa
