@@ -363,20 +363,25 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
             tc::fence_after_sync();
             const uint32_t tSP = tSP_of(t) + lane_addr + col0;
             const int row0 = row_base + t * C::TILE + col0;
-            // scores of this lane's head against 32 cached rows: the two lanes of a head hold the
-            // terms of its hi and of its lo query part; each adds the other's
+            // Scores of this lane's head against 32 cached rows.  The two lanes of a head hold the
+            // terms of its hi and of its lo query part; they share the work: the hi lane takes
+            // columns 0..15, the lo lane columns 16..31, each gets the other lane's terms for its
+            // columns by shuffle and hands back the part of the probabilities the other lane stores.
             uint32_t x[32];
             tc::tmem_ld32(tSP, x);
             tc::tmem_ld_wait();
+            float sc[16];
             float vmax = -INFINITY;
+            const int rowc = row0 + (is_lo ? 16 : 0);
+            const bool full_tile = (row0 + 32 <= len_b);
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                const float mine = __uint_as_float(x[i]);
-                float sc = mine + __shfl_xor_sync(0xffffffffu, mine, 16);
-                if (row0 + i >= len_b) sc = -INFINITY;
-                vmax = fmaxf(vmax, sc);
-                x[i] = __float_as_uint(sc);
+            for (int i = 0; i < 16; ++i) {
+                const float other = __shfl_xor_sync(0xffffffffu, __uint_as_float(is_lo ? x[i] : x[16 + i]), 16);
+                sc[i] = __uint_as_float(is_lo ? x[16 + i] : x[i]) + other;
+                if (!full_tile && rowc + i >= len_b) sc[i] = -INFINITY;
+                vmax = fmaxf(vmax, sc[i]);
             }
+            vmax = fmaxf(vmax, __shfl_xor_sync(0xffffffffu, vmax, 16));
             // maximum over the tile: the other columns belong to the other warps of the quadrant
             float *mxt = mx + (t & 1) * 256;
             if (!is_lo) mxt[sub * 64 + head] = vmax;
@@ -384,14 +389,17 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
             const float m_new = fmaxf(fmaxf(m_run, mxt[head]), fmaxf(fmaxf(mxt[64 + head], mxt[128 + head]), mxt[192 + head]));
             const float alpha = exp2_diff(m_run, m_new);
             m_run = m_new;
-            // probabilities, this lane's part, over the scores
+            // probabilities of this lane's 16 columns, split; the lane keeps its own part (hi or lo)
+            // and receives that part for the other 16 columns
             float lsum = 0.f;
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                const float p = fast_exp2(__uint_as_float(x[i]) - m_new);
+            for (int i = 0; i < 16; ++i) {
+                const float p = fast_exp2(sc[i] - m_new);
                 lsum += p;
-                const float ph = tf32_hi(p);
-                x[i] = __float_as_uint(is_lo ? p - ph : ph);
+                const float ph = tf32_hi(p), pl = p - ph;
+                const float got = __shfl_xor_sync(0xffffffffu, is_lo ? ph : pl, 16);
+                x[i] = __float_as_uint(is_lo ? got : ph);              // columns 0..15: own (hi lane) or received (lo lane)
+                x[16 + i] = __float_as_uint(is_lo ? pl : got);         // columns 16..31
             }
             tc::tmem_st32(tSP, x);
             tc::tmem_st_wait();
@@ -418,7 +426,8 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
         if (ok) {
             tc::fence_after_sync();
             fold(alpha_prev);
-            if (!is_lo) lx[sub * 64 + head] = l_run;
+            const float l_pair = l_run + __shfl_xor_sync(0xffffffffu, l_run, 16);   // each lane summed 16 of the 32 columns
+            if (!is_lo) lx[sub * 64 + head] = l_pair;
             named_sync(1 + qd, 128);
             float *slot = (a.flat ? a.ws + ((size_t)blockIdx.x * GH) * PS
                                   : a.ws + ((((size_t)b * a.h_kv + h) * a.splits + split) * GH) * PS) + (size_t)head * PS;
