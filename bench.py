@@ -43,7 +43,7 @@ L2_BYTES_ASSUMED = 126 * 1024 * 1024
 # from are kept as text under profiles/.  None = not captured.
 NCU_TRAFFIC_BYTES = {
     "gqa": 1074650112 + 3750144,        # profiles/stream_decode_kernel_gqa.md (full-size launch)
-    "mqa_long": 537828864 + 5385984,    # profiles/grouped_decode_kernel_mqa_long.md (full-size launch)
+    "mqa_long": 537066496 + 314112,     # profiles/grouped64_decode_kernel_mqa_long.md (full-size launch)
     "extra_group8_d128": 1075588864 + 4157440,   # profiles/mma_decode_kernel_group8_d128.md (full-size launch)
 }
 
@@ -483,7 +483,7 @@ def main():
         ach = decode_bytes / (k_ms * 1e-3) / 1e9
         kname = {moa.PATH_GENERIC: "generic_decode_kernel",
                  moa.PATH_STREAM: "stream_decode_kernel (FMA; scores, online softmax, weighted sum, append, partial merge)",
-                 moa.PATH_GROUPED: "grouped_decode_kernel (tcgen05)",
+                 moa.PATH_GROUPED: "grouped64_decode_kernel / grouped_decode_kernel (tcgen05)",
                  moa.PATH_MMA: "mma_decode_kernel (warp-level TF32 MMA; scores, online softmax, weighted sum, append, "
                                "partial merge)"}.get(moa.moa_last_path(), "?")
         roof = {"bound": "hbm", "kernel": kname, "achieved": ach, "peak": peak,

@@ -467,7 +467,7 @@ static cudaError_t launch_grouped_cfg(const CUtensorMap &mk, const CUtensorMap &
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     const long long warps = (long long)ga.batch * ga.h_q;
-    grouped_combine_kernel<GH><<<(int)((warps + 3) / 4), 128, 0, st>>>(ga);
+    grouped_combine_kernel<GH><<<(int)warps, 128, 0, st>>>(ga);
     count_launch();
     return cudaGetLastError();
 }
@@ -497,7 +497,7 @@ static cudaError_t launch_grouped64(const CUtensorMap &mk, const CUtensorMap &mv
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     const long long warps = (long long)ga.batch * ga.h_q;
-    grouped_combine_kernel<64><<<(int)((warps + 3) / 4), 128, 0, st>>>(ga);
+    grouped_combine_kernel<64><<<(int)warps, 128, 0, st>>>(ga);
     count_launch();
     return cudaGetLastError();
 }

@@ -709,22 +709,26 @@ grouped_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_co
     if (warp == 1) tc::tmem_dealloc(tmem, 512);
 }
 
-// Merge the per-split partials of the grouped kernel.  One warp per (batch, query head).
-// The (m, l) pairs of up to 32 splits are read by the lanes in parallel; the weighted-sum
-// rows are then accumulated split by split, in split order, with independent loads.
+// Merge the per-split partials of the grouped kernels.  One block of four warps per (batch,
+// query head): warp w accumulates the splits w, w+4, ... (in that order) against the global
+// maximum, which every warp first reads from all splits in parallel; the four sums are then
+// added in warp order, so the result is reproducible.  A split row is 132 floats
+// (o[128], m, l, 2 pad); with many splits per unit the merge is a chain of dependent L2
+// reads, which is why it is cut four ways.
 template <int GH>
 __global__ void __launch_bounds__(128) grouped_combine_kernel(const GroupedArgs a)
 {
     constexpr int PS = 132;
-    const int lane = threadIdx.x & 31;
-    const long long wid = (long long)blockIdx.x * 4 + (threadIdx.x >> 5);
-    if (wid >= (long long)a.batch * a.h_q) return;
+    __shared__ float4 s_acc[4][32];
+    __shared__ float s_l[4];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long wid = blockIdx.x;
     const int b = (int)(wid / a.h_q), gq = (int)(wid % a.h_q);
     const int h = gq / GH, g = gq % GH;
     const int unit = b * a.h_kv + h;
     const int len_b = grouped_len(a, b);
     if (len_b == 0) {                              // out-of-range length: report, leave out untouched
-        if (gq == 0 && lane == 0) raise_status(MOA_STATUS_SEQLEN_RANGE);
+        if (gq == 0 && threadIdx.x == 0) raise_status(MOA_STATUS_SEQLEN_RANGE);
         return;
     }
     const int tiles_total = (len_b + 127) / 128;
@@ -748,21 +752,26 @@ __global__ void __launch_bounds__(128) grouped_combine_kernel(const GroupedArgs 
     }
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float L = 0.f;
-    for (int s0 = 0; s0 < used; s0 += 32) {
-        const bool mine = s0 + lane < used;
-        const float f_mine = mine ? exp2_diff(base[(size_t)(s0 + lane) * stride + 128], M) : 0.f;
-        float lf = mine ? base[(size_t)(s0 + lane) * stride + 129] * f_mine : 0.f;
-#pragma unroll
-        for (int off = 16; off >= 1; off >>= 1) lf += __shfl_xor_sync(0xffffffffu, lf, off);
-        L += lf;
-        const int cnt = (used - s0 < 32) ? used - s0 : 32;
 #pragma unroll 4
-        for (int j = 0; j < cnt; ++j) {
-            const float f = __shfl_sync(0xffffffffu, f_mine, j);
-            const float4 t = *reinterpret_cast<const float4 *>(base + (size_t)(s0 + j) * stride + lane * 4);
-            acc.x = fmaf(t.x, f, acc.x); acc.y = fmaf(t.y, f, acc.y);
-            acc.z = fmaf(t.z, f, acc.z); acc.w = fmaf(t.w, f, acc.w);
-        }
+    for (int sp = warp; sp < used; sp += 4) {
+        const float *row = base + (size_t)sp * stride;
+        const float f = exp2_diff(row[128], M);
+        L = fmaf(row[129], f, L);
+        const float4 t = *reinterpret_cast<const float4 *>(row + lane * 4);
+        acc.x = fmaf(t.x, f, acc.x); acc.y = fmaf(t.y, f, acc.y);
+        acc.z = fmaf(t.z, f, acc.z); acc.w = fmaf(t.w, f, acc.w);
+    }
+    s_acc[warp][lane] = acc;
+    if (lane == 0) s_l[warp] = L;
+    __syncthreads();
+    if (warp != 0) return;
+    acc = s_acc[0][lane];
+    L = s_l[0];
+#pragma unroll
+    for (int w = 1; w < 4; ++w) {
+        const float4 t = s_acc[w][lane];
+        acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
+        L += s_l[w];
     }
     if (a.partial_out != nullptr) {
         float *dst = a.partial_out + ((size_t)b * a.h_q + gq) * 132;
