@@ -83,7 +83,7 @@ struct Grouped64Cfg {
     static constexpr uint32_t OFF_MX = OFF_RING + NBUF * CHUNK;     // [2 tiles][4 column quarters][64 heads] tile maxima
     static constexpr uint32_t OFF_LX = OFF_MX + 2 * 4 * 64 * 4;     // [4 column quarters][64 heads] sums
     static constexpr uint32_t OFF_BAR = OFF_LX + 4 * 64 * 4;
-    static constexpr int NBAR = 2 * NBUF + 2 * NG + 2 + 2 + 1 + 1;
+    static constexpr int NBAR = 2 * NBUF + 2 * NG + 2 + 1;
     static constexpr uint32_t OFF_TMEM = OFF_BAR + NBAR * 8;
     static constexpr uint32_t OFF_ABORT = OFF_TMEM + 4;
     static constexpr uint32_t OFF_SHARE = OFF_ABORT + 4;            // flat mode: unit, first CTA, CTA count
@@ -118,11 +118,17 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
     // Per group of four chunks (group g uses slot g % NG; the ring holds fewer than NG groups):
     auto bar_gfull = [&](int g) { return smem_u32(&bars[2 * NBUF + g]); };            // all four chunks landed
     auto bar_glo = [&](int g) { return smem_u32(&bars[2 * NBUF + NG + g]); };         // all four lo parts in place
-    auto bar_sfull = [&](int s) { return smem_u32(&bars[2 * NBUF + 2 * NG + s]); };   // scores of a tile complete
-    auto bar_pfull = [&](int s) { return smem_u32(&bars[2 * NBUF + 2 * NG + 2 + s]); };   // probabilities stored
-    const uint32_t bar_ofull = smem_u32(&bars[2 * NBUF + 2 * NG + 4]);                // weighted sum of a tile complete
-    const uint32_t bar_ofree = smem_u32(&bars[2 * NBUF + 2 * NG + 5]);                // ... and folded
+    auto bar_pfull = [&](int s) { return smem_u32(&bars[2 * NBUF + 2 * NG + s]); };   // probabilities stored
+    const uint32_t bar_ofree = smem_u32(&bars[2 * NBUF + 2 * NG + 2]);                // weighted sum of a tile folded
 
+    // "The product of a whole tile is complete" is the completion of the lo product of the last
+    // chunk of its group (a second tcgen05.commit at the end of a batch costs the issuer about
+    // 250 cycles of tensor time, measured).  Group index of the K / V chunks of tile t in ring
+    // order; ring buffer and use count of a group's last chunk.
+    auto group_k = [](int t) { return t == 0 ? 0 : 2 * t - 1; };
+    auto group_v = [](int t, int tiles) { return t < tiles - 1 ? 2 * t + 2 : 2 * tiles - 1; };
+    auto bar_group_done = [&](int g) { return bar_empty((4 * g + 3) % NBUF); };
+    auto par_group_done = [](int g) { return (uint32_t)((4 * g + 3) / Grouped64Cfg::NBUF) & 1u; };
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     int split = (int)blockIdx.x % a.splits;
     int sunit = (int)blockIdx.x / a.splits;                       // stored (batch, kv head)
@@ -155,8 +161,8 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
             mbar_init(bar_gfull(g), 4);            // one arrival (with its byte count) per chunk
             mbar_init(bar_glo(g), 4 * C::CONV_WARPS);
         }
-        for (int i = 0; i < 2; ++i) { mbar_init(bar_sfull(i), 1); mbar_init(bar_pfull(i), C::SOFT_WARPS); }
-        mbar_init(bar_ofull, 1); mbar_init(bar_ofree, C::SOFT_WARPS);
+        for (int i = 0; i < 2; ++i) mbar_init(bar_pfull(i), C::SOFT_WARPS);
+        mbar_init(bar_ofree, C::SOFT_WARPS);
         mbar_fence_init();
         *abort_flag = 0;
         *q_ready = 0; *q_taken = 0;
@@ -258,7 +264,7 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
                 w[3] = is_k ? 2u : 64u;                             // descriptor step per k-step
                 w[4] = is_k ? idesc_k : idesc_v;
                 w[5] = is_hi ? 0u : 1u;                             // accumulate flag of the first product
-                w[6] = is_hi ? 0u : (is_k ? bar_sfull(t & 1) : bar_ofull);   // barrier of the whole tile product
+                w[6] = 0u;
                 w[7] = 0u;
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
@@ -317,7 +323,7 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
                     n2 = lds_volatile_v4(slot + 32u); n3 = lds_volatile_v4(slot + 48u);
                     *q_taken = i + 1;
                 }
-                const uint32_t d = n0.x, a0 = n0.y, hiword = n0.z, step = n0.w, idesc = n1.x, acc0 = n1.y, final_bar = n1.z;
+                const uint32_t d = n0.x, a0 = n0.y, hiword = n0.z, step = n0.w, idesc = n1.x, acc0 = n1.y;
                 const uint32_t bdesc[4] = {n2.x, n2.y, n2.z, n2.w}, done[4] = {n3.x, n3.y, n3.z, n3.w};
                 fetched = false;
                 tc::fence_after_sync();
@@ -340,7 +346,6 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
                                         (c == 0 && ks == 0) ? acc0 : 1u);
                     tc::mma_commit(done[c]);
                 }
-                if (final_bar != 0u) tc::mma_commit(final_bar);
             }
         }
     } else if (is_soft) {
@@ -358,7 +363,7 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
             for (int i = 0; i < 32; ++i) Om[i] = fmaf(Om[i], alpha, __uint_as_float(o[i]));
         };
         for (int t = 0; t < T; ++t) {
-            ok = ok && wait_suspended(bar_sfull(t & 1), (uint32_t)(t >> 1) & 1u, abort_flag);
+            ok = ok && wait_suspended(bar_group_done(group_k(t)), par_group_done(group_k(t)), abort_flag);
             if (named_or(1 + qd, 128, !ok)) { ok = false; break; }    // the four warps of a quadrant leave together
             tc::fence_after_sync();
             const uint32_t tSP = tSP_of(t) + lane_addr + col0;
@@ -409,7 +414,7 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
             l_run = fmaf(l_run, alpha, lsum);
             // fold the previous tile's weighted sum into the running values
             if (t > 0) {
-                ok = wait_suspended(bar_ofull, (uint32_t)(t - 1) & 1u, abort_flag);
+                ok = wait_suspended(bar_group_done(group_v(t - 1, T)), par_group_done(group_v(t - 1, T)), abort_flag);
                 if (ok) {
                     tc::fence_after_sync();
                     fold(alpha_prev);
@@ -421,7 +426,7 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
             alpha_prev = alpha;
         }
         // ---- epilogue: last fold, then this split's partial (m, l, o) per head
-        if (ok) ok = wait_suspended(bar_ofull, (uint32_t)(T - 1) & 1u, abort_flag);
+        if (ok) ok = wait_suspended(bar_group_done(group_v(T - 1, T)), par_group_done(group_v(T - 1, T)), abort_flag);
         if (named_or(1 + qd, 128, !ok)) ok = false;
         if (ok) {
             tc::fence_after_sync();
