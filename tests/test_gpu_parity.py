@@ -487,3 +487,18 @@ def test_argument_errors():
                                     None, 0, st) == moa.ERR_WORKSPACE
     torch.cuda.synchronize()
     assert np.all(gout.host() == -7.0)
+
+
+def test_both_kernels_for_groups_of_64_heads():
+    # tensor-memory operands (default) and shared-memory operands (on request), same inputs
+    q, K, V, s = make(2110, 2, 64, 1, 3333, 128, 128)
+    ref = oracle.decode(q, K, V, s)
+    lens = np.array([3333, 130], np.int32)
+    ref_v = oracle.decode_varlen(q, K, V, lens, s)
+    for operands in (0, 1):
+        moa.moa_set_option(moa.OPT_GROUPED_OPERANDS, operands)
+        try:
+            assert max_err(gpu_decode(q, K, V, s, expect_path=moa.PATH_GROUPED), ref) <= TOL, operands
+            assert max_err(gpu_decode(q, K, V, s, seq_lens=lens, expect_path=moa.PATH_GROUPED), ref_v) <= TOL, operands
+        finally:
+            moa.moa_set_option(moa.OPT_GROUPED_OPERANDS, 0)
