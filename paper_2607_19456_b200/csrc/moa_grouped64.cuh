@@ -159,7 +159,7 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
         for (int i = 0; i < NBUF; ++i) { mbar_init(bar_hi(i), 1); mbar_init(bar_empty(i), 1); }
         for (int g = 0; g < NG; ++g) {
             mbar_init(bar_gfull(g), 4);            // one arrival (with its byte count) per chunk
-            mbar_init(bar_glo(g), 4 * C::CONV_WARPS);
+            mbar_init(bar_glo(g), 4);              // one warp per chunk
         }
         for (int i = 0; i < 2; ++i) mbar_init(bar_pfull(i), C::SOFT_WARPS);
         mbar_init(bar_ofree, C::SOFT_WARPS);
@@ -170,7 +170,7 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
         tc::prefetch_tmap(&tmapV);
         if (a.tailK != nullptr) { tc::prefetch_tmap(&tmapKt); tc::prefetch_tmap(&tmapVt); }
     }
-    if (warp == 1) tc::tmem_alloc(smem_u32(tmem_slot), 512);
+    if (warp == 3) tc::tmem_alloc(smem_u32(tmem_slot), 512);
     tc::fence_before_sync();
     __syncthreads();
     tc::fence_after_sync();
@@ -298,7 +298,7 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
                 *q_ready = i + 1;
             }
         }
-    } else if (warp == 1) {
+    } else if (warp == 3) {
         // ================= MMA issuer (one thread) =================
         if (lane == 0) {
             const int nbatch = 4 * T;
@@ -452,23 +452,32 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
         }
     } else {
         // ================= converters: chunk -> its lo part, in place =================
-        constexpr int TT = C::CONV_WARPS * 32;                         // 128 threads
+        // Each of the four converter warps takes every fourth chunk, so that four conversions are in flight: a
+        // conversion is a chain of barrier wait, 16 KB of loads, 16 KB of stores and barrier
+        // arrival, and one team alone (about 750 cycles per chunk, 8 chunks per tile) was what the
+        // lo batches waited for.
+        constexpr int TT = 32;                                         // threads of a team
         constexpr int PER = (C::CHUNK / 16) / TT;                      // float4 every thread handles
-        const int ct = ((warp < 4) ? warp - 2 : warp - 18) * 32 + lane;
+        const int team = (warp < 4) ? warp - 1 : warp - 18;           // warps 1, 2, 20, 21
+        const int ct = lane;
         bool ok = true;
         for (ChunkSeq s(T); ok && !s.done; s.next()) {
+            if ((s.seq & 3) != team) continue;
             const int buf = s.seq % NBUF, use = s.seq / NBUF;
             ok = wait_suspended(bar_hi(buf), (uint32_t)use & 1u, abort_flag);
             if (!ok) break;
             float4 *p = reinterpret_cast<float4 *>(smem + C::OFF_RING + (uint32_t)buf * C::CHUNK);
-            float4 v[PER];
 #pragma unroll
-            for (int i = 0; i < PER; ++i) v[i] = p[ct + i * TT];
+            for (int part = 0; part < 4; ++part) {
+                float4 v[PER / 4];
 #pragma unroll
-            for (int i = 0; i < PER; ++i) {
-                v[i].x -= tf32_hi(v[i].x); v[i].y -= tf32_hi(v[i].y);
-                v[i].z -= tf32_hi(v[i].z); v[i].w -= tf32_hi(v[i].w);
-                p[ct + i * TT] = v[i];
+                for (int i = 0; i < PER / 4; ++i) v[i] = p[ct + (part * (PER / 4) + i) * TT];
+#pragma unroll
+                for (int i = 0; i < PER / 4; ++i) {
+                    v[i].x -= tf32_hi(v[i].x); v[i].y -= tf32_hi(v[i].y);
+                    v[i].z -= tf32_hi(v[i].z); v[i].w -= tf32_hi(v[i].w);
+                    p[ct + (part * (PER / 4) + i) * TT] = v[i];
+                }
             }
             tc::fence_async_smem();
             __syncwarp();
@@ -478,7 +487,7 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
 
     tc::fence_before_sync();
     __syncthreads();
-    if (warp == 1) tc::tmem_dealloc(tmem, 512);
+    if (warp == 3) tc::tmem_dealloc(tmem, 512);
 }
 
 }  // namespace moa
