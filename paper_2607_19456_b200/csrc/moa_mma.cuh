@@ -187,18 +187,22 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
     const int my_d = is_pv ? D : DK;            // row length of this warp's operand
     const float *my_new = is_pv ? a.v_new : a.k_new;
     float *my_cache = is_pv ? a.Vw : a.Kw;
-    const long long my_sb = is_pv ? a.v_sb : a.k_sb, my_sh = is_pv ? a.v_sh : a.k_sh, my_sr = is_pv ? a.v_sr : a.k_sr;
 
     // ---- load side: this pair's tiles are c0+pair, c0+pair+P, ... ------------------------
     long long jl = c0 + pair;
     int kl = 0;
     Cursor lc = cursor_at<R>(a, (jl < c1) ? jl : c0, pref);
-    size_t slab = 0;                           // stored (batch, kv head) of the unit under lc
+    // The 16-head configuration is at the register limit: what only the fused append needs is
+    // recomputed there instead of being carried through the loop (the other configurations are
+    // 5 % faster with the values carried).
+    constexpr bool LEAN = (C::NT == 2);
+    const long long sb_keep = is_pv ? a.v_sb : a.k_sb, sh_keep = is_pv ? a.v_sh : a.k_sh, sr_keep = is_pv ? a.v_sr : a.k_sr;
+    size_t slab_keep = 0;                      // stored (batch, kv head) of the unit under lc
     int hs = 0;                                // its stored kv head
     bool writes_new = false;                   // this virtual head stores the appended row
     auto load_unit_changed = [&]() {
         hs = lc.h / a.kv_share;
-        slab = (size_t)lc.b * h_stored + hs;
+        if (!LEAN) slab_keep = (size_t)lc.b * h_stored + hs;
         writes_new = (a.k_new != nullptr) && (lc.h == hs * a.kv_share);
     };
     load_unit_changed();
@@ -222,6 +226,9 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
         // the tile holding it also stores it into the cache (K by the score warp, V by the other);
         // the tile's copy of that row is replaced from k_new / v_new before use.
         if (writes_new && row0 + R >= lc.len && lane * 4 < my_d) {
+            const size_t slab = LEAN ? (size_t)lc.b * h_stored + hs : slab_keep;   // (b, stored kv head) of the dense new rows
+            const long long my_sb = LEAN ? (is_pv ? a.v_sb : a.k_sb) : sb_keep, my_sh = LEAN ? (is_pv ? a.v_sh : a.k_sh) : sh_keep,
+                            my_sr = LEAN ? (is_pv ? a.v_sr : a.k_sr) : sr_keep;
             const size_t dst = (size_t)lc.b * my_sb + (size_t)hs * my_sh + (size_t)(lc.len - 1) * my_sr + lane * 4;
             *reinterpret_cast<float4 *>(my_cache + dst) = *reinterpret_cast<const float4 *>(my_new + slab * my_d + lane * 4);
             if (!PAIRED) {
