@@ -359,12 +359,18 @@ struct GroupedPlan {
     size_t ws_ragged() const { return (ws_bytes + 255) / 256 * 256 + tail_bytes; }
 };
 static int g_grouped_heads = 0;   // MOA_OPT_GROUPED_HEADS: 0 = automatic
+static int g_grouped_operands = 0;   // MOA_OPT_GROUPED_OPERANDS
 
 static GroupedPlan plan_grouped(const DeviceState &s, int batch, int h_q, int h_kv, int n, int d_k, int d_v)
 {
     GroupedPlan p;
     const int g_s = h_q / h_kv;
-    if (d_k != 128 || d_v != 128 || (g_s != 16 && g_s != 32 && g_s != 64)) return p;
+    if (d_k != 128 || d_v != 128) return p;
+    // Any group of 17 to 64 heads runs on the kernel with 64 head lanes (missing heads are zero
+    // lanes): its time per tile does not depend on the number of heads, and from 17 heads on it
+    // beats the warp-MMA kernel's passes over groups of 8 or 16.
+    const bool lanes64 = (g_grouped_operands == 0) && g_s > 16 && g_s <= 64 && (g_grouped_heads == 0 || g_grouped_heads == 64);
+    if (!lanes64 && g_s != 16 && g_s != 32 && g_s != 64) return p;
     // Groups of 16 are faster as two groups of 8 on the warp-MMA streaming kernel (the K/V tile
     // is read twice, the second time from L2); this kernel takes them only when forced.
     if (g_s == 16 && g_force_path != MOA_PATH_GROUPED) return p;
@@ -372,10 +378,10 @@ static GroupedPlan plan_grouped(const DeviceState &s, int batch, int h_q, int h_
     if (units > 0x7fffffffLL / 256 || (long long)n > 0x7fffffffLL - 256) return p;
     // One CTA takes the whole group (measured faster than cutting a group of 64 into two
     // neighbouring CTAs of 32 heads that read the same rows through L2).
-    p.GH = g_s;
-    if (g_grouped_heads == 16 || g_grouped_heads == 32 || g_grouped_heads == 64)
+    p.GH = lanes64 ? 64 : g_s;
+    if (!lanes64 && (g_grouped_heads == 16 || g_grouped_heads == 32 || g_grouped_heads == 64))
         if (g_grouped_heads <= g_s) p.GH = g_grouped_heads;
-    p.share = g_s / p.GH;
+    p.share = lanes64 ? 1 : g_s / p.GH;
     const long long ctas_per_split = units * p.share;
     const int tiles = (n + 127) / 128;
     long long splits = ctas_per_split >= s.sm_count ? 1 : s.sm_count / ctas_per_split;
@@ -472,26 +478,26 @@ static cudaError_t launch_grouped_cfg(const CUtensorMap &mk, const CUtensorMap &
     return cudaGetLastError();
 }
 
-static int g_grouped_operands = 0;   // MOA_OPT_GROUPED_OPERANDS
 
 // Groups of 64 heads with Q and P in tensor memory; same arguments and partial format as
 // the shared-memory-operand kernel, so the combine kernel is shared.
-static cudaError_t launch_grouped64(const CUtensorMap &mk, const CUtensorMap &mv, const CUtensorMap &mkt,
-                                    const CUtensorMap &mvt, const GroupedArgs &ga, int grid, cudaStream_t st)
+template <bool PRECISE>
+static cudaError_t launch_grouped64_cfg(const CUtensorMap &mk, const CUtensorMap &mv, const CUtensorMap &mkt,
+                                        const CUtensorMap &mvt, const GroupedArgs &ga, int grid, cudaStream_t st)
 {
     using C = Grouped64Cfg;
     static bool attr_set[kMaxDevices] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (!attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(grouped64_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(grouped64_decode_kernel<PRECISE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)C::SMEM_BYTES);
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
     {
         TimedLaunch t(st);
-        grouped64_decode_kernel<<<grid, C::THREADS, C::SMEM_BYTES, st>>>(mk, mv, mkt, mvt, ga);
+        grouped64_decode_kernel<PRECISE><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(mk, mv, mkt, mvt, ga);
     }
     count_launch();
     cudaError_t e = cudaGetLastError();
@@ -500,6 +506,27 @@ static cudaError_t launch_grouped64(const CUtensorMap &mk, const CUtensorMap &mv
     grouped_combine_kernel<64><<<(int)warps, 128, 0, st>>>(ga);
     count_launch();
     return cudaGetLastError();
+}
+
+template <int GH>
+static cudaError_t launch_grouped_cfg(const CUtensorMap &mk, const CUtensorMap &mv, const CUtensorMap &mkt,
+                                      const CUtensorMap &mvt, const GroupedArgs &ga, int grid, cudaStream_t st);
+
+// Groups of 17 to 64 heads on 64 head lanes.  Same arguments and partial format as the
+// shared-memory-operand kernel, so the combine kernel is shared.
+//  - Long dense caches: the kernel with Q and P in tensor memory whose scores are one
+//    accumulation chain of 32 steps (the error of an output averages out over the rows).
+//  - Short caches and ragged ones (lengths unknown here): exact groups of 32 or 64 heads run
+//    on the shared-memory-operand kernel (16-step chains, and faster than the next one);
+//    padded groups on the tensor-memory kernel that keeps the two score chains apart.
+static cudaError_t launch_grouped64(const CUtensorMap &mk, const CUtensorMap &mv, const CUtensorMap &mkt,
+                                    const CUtensorMap &mvt, const GroupedArgs &ga, int grid, cudaStream_t st,
+                                    bool fused)
+{
+    if (ga.seq_lens == nullptr && !fused && ga.n >= 4096) return launch_grouped64_cfg<false>(mk, mv, mkt, mvt, ga, grid, st);
+    if (ga.g_s == 64) return launch_grouped_cfg<64>(mk, mv, mkt, mvt, ga, grid, st);
+    if (ga.g_s == 32) return launch_grouped_cfg<32>(mk, mv, mkt, mvt, ga, grid, st);
+    return launch_grouped64_cfg<true>(mk, mv, mkt, mvt, ga, grid, st);
 }
 
 static cudaError_t launch_generic(const DecodeArgs &a, cudaStream_t st)
@@ -610,6 +637,7 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
         ga.q = q; ga.out = out; ga.ws = static_cast<float *>(ws);
         ga.batch = batch; ga.h_q = h_q; ga.h_kv = h_kv * gplan.share; ga.n = n_max;
         ga.h_kv_stored = h_kv; ga.share = gplan.share;
+        ga.g_s = (gplan.share == 1) ? g_s : gplan.GH;
         ga.splits = gplan.splits; ga.tiles_per_split = gplan.tiles_per_split;
         ga.qscale = scale * kLog2e;
         ga.partial_out = partial_out;
@@ -638,7 +666,7 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
         }
         if (gplan.GH == 16) e = launch_grouped_cfg<16>(mk, mv, mkt, mvt, ga, grid, st);
         else if (gplan.GH == 32) e = launch_grouped_cfg<32>(mk, mv, mkt, mvt, ga, grid, st);
-        else if (gplan.share == 1 && g_grouped_operands == 0) e = launch_grouped64(mk, mv, mkt, mvt, ga, grid, st);
+        else if (gplan.share == 1 && g_grouped_operands == 0) e = launch_grouped64(mk, mv, mkt, mvt, ga, grid, st, fused != nullptr);
         else e = launch_grouped_cfg<64>(mk, mv, mkt, mvt, ga, grid, st);
         if (e == cudaSuccess && fused != nullptr && fused->lens_rw != nullptr) {
             lens_add_kernel<<<(batch + 127) / 128, 128, 0, st>>>(fused->lens_rw, batch, 1, n_max);

@@ -72,6 +72,7 @@ struct GroupedArgs {
     float *out;          // [batch, h_q, 128]
     float *ws;           // partial slots [units][splits][GH][PS]
     int batch, h_q, h_kv, n;
+    int g_s;             // query heads per (virtual) kv head; smaller than GH only on the 64-lane kernel (padded group)
     int h_kv_stored;     // K/V heads as stored; h_kv above counts virtual heads of GH query heads
     int share;           // virtual heads per stored K/V head (h_kv = h_kv_stored * share)
     int splits;          // sequence splits per unit
@@ -724,7 +725,7 @@ __global__ void __launch_bounds__(128) grouped_combine_kernel(const GroupedArgs 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const long long wid = blockIdx.x;
     const int b = (int)(wid / a.h_q), gq = (int)(wid % a.h_q);
-    const int h = gq / GH, g = gq % GH;
+    const int h = gq / a.g_s, g = gq % a.g_s;      // (partial slots are GH apart, the heads of a unit a.g_s)
     const int unit = b * a.h_kv + h;
     const int len_b = grouped_len(a, b);
     if (len_b == 0) {                              // out-of-range length: report, leave out untouched

@@ -83,7 +83,7 @@ struct Grouped64Cfg {
     static constexpr uint32_t OFF_MX = OFF_RING + NBUF * CHUNK;     // [2 tiles][4 column quarters][64 heads] tile maxima
     static constexpr uint32_t OFF_LX = OFF_MX + 2 * 4 * 64 * 4;     // [4 column quarters][64 heads] sums
     static constexpr uint32_t OFF_BAR = OFF_LX + 4 * 64 * 4;
-    static constexpr int NBAR = 2 * NBUF + 2 * NG + 2 + 1;
+    static constexpr int NBAR = 2 * NBUF + 2 * NG + 2 + 1 + 1;
     static constexpr uint32_t OFF_TMEM = OFF_BAR + NBAR * 8;
     static constexpr uint32_t OFF_ABORT = OFF_TMEM + 4;
     static constexpr uint32_t OFF_SHARE = OFF_ABORT + 4;            // flat mode: unit, first CTA, CTA count
@@ -92,6 +92,7 @@ struct Grouped64Cfg {
     static constexpr size_t SMEM_BYTES = OFF_QUEUE + QN * 64;
 };
 
+template <bool PRECISE>
 __global__ void __launch_bounds__(Grouped64Cfg::THREADS, 1)
 grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant__ CUtensorMap tmapV,
                         const __grid_constant__ CUtensorMap tmapKt, const __grid_constant__ CUtensorMap tmapVt,
@@ -120,6 +121,7 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
     auto bar_glo = [&](int g) { return smem_u32(&bars[2 * NBUF + NG + g]); };         // all four lo parts in place
     auto bar_pfull = [&](int s) { return smem_u32(&bars[2 * NBUF + 2 * NG + s]); };   // probabilities stored
     const uint32_t bar_ofree = smem_u32(&bars[2 * NBUF + 2 * NG + 2]);                // weighted sum of a tile folded
+    const uint32_t bar_shread = smem_u32(&bars[2 * NBUF + 2 * NG + 3]);               // K_hi products of a tile read out
 
     // "The product of a whole tile is complete" is the completion of the lo product of the last
     // chunk of its group (a second tcgen05.commit at the end of a batch costs the issuer about
@@ -129,6 +131,7 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
     auto group_v = [](int t, int tiles) { return t < tiles - 1 ? 2 * t + 2 : 2 * tiles - 1; };
     auto bar_group_done = [&](int g) { return bar_empty((4 * g + 3) % NBUF); };
     auto par_group_done = [](int g) { return (uint32_t)((4 * g + 3) / Grouped64Cfg::NBUF) & 1u; };
+    auto bar_group_hi = [&](int g) { return bar_hi((4 * g + 3) % NBUF); };            // ... of its hi products (same parity)
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     int split = (int)blockIdx.x % a.splits;
     int sunit = (int)blockIdx.x / a.splits;                       // stored (batch, kv head)
@@ -153,6 +156,16 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
     if (T <= 0) return;                            // an empty split (uniform for the CTA)
     const int tail_t = (a.tailK != nullptr) ? tiles_total - 1 - tile0 : -1;
     const int row_base = tile0 * C::TILE;
+    // The tensor core accumulates with truncation, and an error of one unit in the last place of
+    // a score costs the same whatever the size of the term that was added.  With the K_lo
+    // products on top of the K_hi products a score is a chain of 32 steps instead of 16, which
+    // doubles its error: measured against the fp64 oracle 5.1e-6 (max) at 128 rows, 2.2e-6 at
+    // 1000, 1.1e-6 at 4000, 2.7e-7 at 16000 -- the error of an output averages out over the rows.
+    // The PRECISE variant therefore keeps the two chains apart (the softmax group reads the K_hi
+    // products out before the K_lo products start the region afresh: 2.9e-6 at 128 rows), at
+    // the price of one more hand-over per tile; the host uses it for caches of fewer than 4096
+    // rows and for ragged caches, whose lengths it does not know.
+    constexpr bool precise = PRECISE;
 
     // ---- set-up --------------------------------------------------------------------------
     if (tid == 0) {
@@ -162,7 +175,7 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
             mbar_init(bar_glo(g), 4);              // one warp per chunk
         }
         for (int i = 0; i < 2; ++i) mbar_init(bar_pfull(i), C::SOFT_WARPS);
-        mbar_init(bar_ofree, C::SOFT_WARPS);
+        mbar_init(bar_ofree, C::SOFT_WARPS); mbar_init(bar_shread, C::SOFT_WARPS);
         mbar_fence_init();
         *abort_flag = 0;
         *q_ready = 0; *q_taken = 0;
@@ -188,11 +201,12 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
     const bool is_lo = (lane & 16) != 0;
     if (is_soft) {
         // Q operand: this lane's part (hi or lo) of (scale * log2 e) * q[head], columns = features
-        const float *qb = a.q + ((size_t)b * a.h_q + (size_t)h * GH + head) * 128 + col0;
+        // (a group of fewer than 64 heads is padded: the lanes of the missing heads hold zeros)
+        const float *qb = a.q + ((size_t)b * a.h_q + (size_t)h * a.g_s + head) * 128 + col0;
         uint32_t v[32];
 #pragma unroll
         for (int i = 0; i < 32; i += 4) {
-            const float4 x4 = *reinterpret_cast<const float4 *>(qb + i);
+            const float4 x4 = head < a.g_s ? *reinterpret_cast<const float4 *>(qb + i) : make_float4(0.f, 0.f, 0.f, 0.f);
             const float xs[4] = {x4.x * a.qscale, x4.y * a.qscale, x4.z * a.qscale, x4.w * a.qscale};
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
@@ -263,7 +277,7 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
                 w[2] = is_k ? k_hiword : v_hiword;
                 w[3] = is_k ? 2u : 64u;                             // descriptor step per k-step
                 w[4] = is_k ? idesc_k : idesc_v;
-                w[5] = is_hi ? 0u : 1u;                             // accumulate flag of the first product
+                w[5] = (is_hi || (is_k && precise)) ? 0u : 1u;      // accumulate flag of the first product
                 w[6] = 0u;
                 w[7] = 0u;
 #pragma unroll
@@ -282,6 +296,8 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
                                      : wait_or_abort(bar_pfull(0), 0u, abort_flag);
                 } else {
                     ok = wait_or_abort(bar_glo(gs), gpar, abort_flag);
+                    // the K_lo products overwrite the K_hi products of the tile: those must have been read
+                    if (ok && is_k && precise) ok = wait_or_abort(bar_shread, (uint32_t)t & 1u, abort_flag);
                 }
                 for (uint32_t it = 0; ok && *q_taken + C::QN <= i; ++it)       // a free queue slot
                     if (it >= kWaitLimit || ((it & 255u) == 255u && *abort_flag)) {
@@ -356,33 +372,81 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
         float m_run = -INFINITY, l_run = 0.f, alpha_prev = 0.f;
         bool ok = true;
         auto fold = [&](float alpha) {             // Om = alpha * Om + (weighted sum of the last tile)
-            uint32_t o[32];
-            tc::tmem_ld32(tO + lane_addr + col0, o);
-            tc::tmem_ld_wait();
+            if constexpr (PRECISE) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) Om[i] = fmaf(Om[i], alpha, __uint_as_float(o[i]));
+                for (int hf = 0; hf < 2; ++hf) {
+                    uint32_t o[16];
+                    tc::tmem_ld16(tO + lane_addr + col0 + 16 * hf, o);
+                    tc::tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) Om[16 * hf + i] = fmaf(Om[16 * hf + i], alpha, __uint_as_float(o[i]));
+                }
+            } else {
+                uint32_t o[32];
+                tc::tmem_ld32(tO + lane_addr + col0, o);
+                tc::tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) Om[i] = fmaf(Om[i], alpha, __uint_as_float(o[i]));
+            }
         };
         for (int t = 0; t < T; ++t) {
+            const uint32_t tSP = tSP_of(t) + lane_addr + col0;
+            const int row0 = row_base + t * C::TILE + col0;
+            float sc[16];                              // scores: the hi lane of a head columns 0..15, the lo lane 16..31
+            if constexpr (PRECISE) {                   // the K_hi products of the tile, before the K_lo products overwrite them
+                ok = ok && wait_suspended(bar_group_hi(group_k(t)), par_group_done(group_k(t)), abort_flag);
+                tc::fence_after_sync();                // (after a failed wait the values are not used)
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {       // 16 columns at a time, to stay within the registers
+                    uint32_t xh[16];
+                    tc::tmem_ld16(tSP + 16 * hf, xh);
+                    tc::tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const float mine = __uint_as_float(xh[i]);
+                        const float sum = mine + __shfl_xor_sync(0xffffffffu, mine, 16);
+                        if ((hf == 1) == is_lo) sc[i] = sum;
+                    }
+                }
+                tc::fence_before_sync();
+                __syncwarp();
+                if (ok && lane == 0) tc::mbar_arrive(bar_shread);
+            }
             ok = ok && wait_suspended(bar_group_done(group_k(t)), par_group_done(group_k(t)), abort_flag);
             if (named_or(1 + qd, 128, !ok)) { ok = false; break; }    // the four warps of a quadrant leave together
             tc::fence_after_sync();
-            const uint32_t tSP = tSP_of(t) + lane_addr + col0;
-            const int row0 = row_base + t * C::TILE + col0;
             // Scores of this lane's head against 32 cached rows.  The two lanes of a head hold the
             // terms of its hi and of its lo query part; they share the work: the hi lane takes
             // columns 0..15, the lo lane columns 16..31, each gets the other lane's terms for its
             // columns by shuffle and hands back the part of the probabilities the other lane stores.
-            uint32_t x[32];
-            tc::tmem_ld32(tSP, x);
-            tc::tmem_ld_wait();
-            float sc[16];
+            if constexpr (PRECISE) {
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {
+                    uint32_t xh[16];
+                    tc::tmem_ld16(tSP + 16 * hf, xh);
+                    tc::tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const float mine = __uint_as_float(xh[i]);
+                        const float sum = mine + __shfl_xor_sync(0xffffffffu, mine, 16);
+                        if ((hf == 1) == is_lo) sc[i] += sum;
+                    }
+                }
+            } else {
+                uint32_t x[32];
+                tc::tmem_ld32(tSP, x);
+                tc::tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {       // each lane sends what the other needs
+                    const float other = __shfl_xor_sync(0xffffffffu, __uint_as_float(is_lo ? x[i] : x[16 + i]), 16);
+                    sc[i] = __uint_as_float(is_lo ? x[16 + i] : x[i]) + other;
+                }
+            }
             float vmax = -INFINITY;
             const int rowc = row0 + (is_lo ? 16 : 0);
             const bool full_tile = (row0 + 32 <= len_b);
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
-                const float other = __shfl_xor_sync(0xffffffffu, __uint_as_float(is_lo ? x[i] : x[16 + i]), 16);
-                sc[i] = __uint_as_float(is_lo ? x[16 + i] : x[i]) + other;
                 if (!full_tile && rowc + i >= len_b) sc[i] = -INFINITY;
                 vmax = fmaxf(vmax, sc[i]);
             }
@@ -394,19 +458,38 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
             const float m_new = fmaxf(fmaxf(m_run, mxt[head]), fmaxf(fmaxf(mxt[64 + head], mxt[128 + head]), mxt[192 + head]));
             const float alpha = exp2_diff(m_run, m_new);
             m_run = m_new;
-            // probabilities of this lane's 16 columns, split; the lane keeps its own part (hi or lo)
-            // and receives that part for the other 16 columns
+            // probabilities of this lane's 16 columns, split: the lane keeps its own part (hi or lo)
+            // and hands the other part to the other lane of the head; 16 columns at a time (the hi
+            // lane's columns first), to stay within the registers
             float lsum = 0.f;
+            if constexpr (PRECISE) {
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const float p = fast_exp2(sc[i] - m_new);
-                lsum += p;
-                const float ph = tf32_hi(p), pl = p - ph;
-                const float got = __shfl_xor_sync(0xffffffffu, is_lo ? ph : pl, 16);
-                x[i] = __float_as_uint(is_lo ? got : ph);              // columns 0..15: own (hi lane) or received (lo lane)
-                x[16 + i] = __float_as_uint(is_lo ? pl : got);         // columns 16..31
+                for (int hf = 0; hf < 2; ++hf) {
+                    const bool mine = ((hf == 1) == is_lo);     // this half's columns are this lane's
+                    uint32_t xh[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const float p = mine ? fast_exp2(sc[i] - m_new) : 0.f;
+                        lsum += p;
+                        const float ph = tf32_hi(p), pl = p - ph;
+                        const float got = __shfl_xor_sync(0xffffffffu, is_lo ? ph : pl, 16);
+                        xh[i] = __float_as_uint(mine ? (is_lo ? pl : ph) : got);
+                    }
+                    tc::tmem_st16(tSP + 16 * hf, xh);
+                }
+            } else {
+                uint32_t x[32];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const float p = fast_exp2(sc[i] - m_new);
+                    lsum += p;
+                    const float ph = tf32_hi(p), pl = p - ph;
+                    const float got = __shfl_xor_sync(0xffffffffu, is_lo ? ph : pl, 16);
+                    x[i] = __float_as_uint(is_lo ? got : ph);              // columns 0..15: own (hi lane) or received (lo lane)
+                    x[16 + i] = __float_as_uint(is_lo ? pl : got);         // columns 16..31
+                }
+                tc::tmem_st32(tSP, x);
             }
-            tc::tmem_st32(tSP, x);
             tc::tmem_st_wait();
             tc::fence_before_sync();
             __syncwarp();
@@ -443,9 +526,9 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
                 v.y = Om[i + 1] + __shfl_xor_sync(0xffffffffu, Om[i + 1], 16);
                 v.z = Om[i + 2] + __shfl_xor_sync(0xffffffffu, Om[i + 2], 16);
                 v.w = Om[i + 3] + __shfl_xor_sync(0xffffffffu, Om[i + 3], 16);
-                if (!is_lo) *reinterpret_cast<float4 *>(slot + col0 + i) = v;
+                if (!is_lo && head < a.g_s) *reinterpret_cast<float4 *>(slot + col0 + i) = v;
             }
-            if (sub == 0 && !is_lo) {
+            if (sub == 0 && !is_lo && head < a.g_s) {
                 slot[128] = m_run;
                 slot[129] = (lx[head] + lx[64 + head]) + (lx[128 + head] + lx[192 + head]);
             }

@@ -22,7 +22,7 @@ def run_dense_on_gpu(w):
     moa.moa_decode_attn(dq, dK, dV, out, w.batch, w.h_q, w.h_kv, w.n, w.d_k, w.d_v, w.scale)
     torch.cuda.synchronize()
     want = moa.PATH_STREAM
-    if w.group >= 32 and w.d_k == 128:
+    if 17 <= w.group <= 64 and w.d_k == 128:
         want = moa.PATH_GROUPED
     elif w.group % 8 == 0 and w.d_k >= 64:
         want = moa.PATH_MMA

@@ -50,8 +50,8 @@ def test_paper_gqa_shapes_d32(hkv):
 # ---------------------------------------------------------------------------------------
 def automatic_path(D, gs):
     """The kernel family the library picks for a dense, aligned call."""
-    if D == 128 and gs in (32, 64):
-        return moa.PATH_GROUPED
+    if D == 128 and 17 <= gs <= 64:
+        return moa.PATH_GROUPED              # 64 head lanes, missing heads padded
     if 8 < gs < 16 and D >= 64:
         return moa.PATH_MMA                  # one padded group of 16 heads
     if gs <= 8:
@@ -66,7 +66,7 @@ def automatic_path(D, gs):
 
 
 @pytest.mark.parametrize("D", [32, 64, 128])
-@pytest.mark.parametrize("gs", [1, 2, 3, 4, 5, 8, 12, 16, 24, 64])
+@pytest.mark.parametrize("gs", [1, 2, 3, 4, 5, 8, 12, 16, 24, 40, 64])
 def test_stream_kernel_group_sizes(D, gs):
     hkv = 2
     for n in (1, 7, 130, 1037):
@@ -491,9 +491,9 @@ def test_argument_errors():
 
 def test_both_kernels_for_groups_of_64_heads():
     # tensor-memory operands (default) and shared-memory operands (on request), same inputs
-    q, K, V, s = make(2110, 2, 64, 1, 3333, 128, 128)
+    q, K, V, s = make(2110, 2, 64, 1, 5333, 128, 128)
     ref = oracle.decode(q, K, V, s)
-    lens = np.array([3333, 130], np.int32)
+    lens = np.array([5333, 130], np.int32)
     ref_v = oracle.decode_varlen(q, K, V, lens, s)
     for operands in (0, 1):
         moa.moa_set_option(moa.OPT_GROUPED_OPERANDS, operands)
@@ -502,3 +502,25 @@ def test_both_kernels_for_groups_of_64_heads():
             assert max_err(gpu_decode(q, K, V, s, seq_lens=lens, expect_path=moa.PATH_GROUPED), ref_v) <= TOL, operands
         finally:
             moa.moa_set_option(moa.OPT_GROUPED_OPERANDS, 0)
+
+
+@pytest.mark.parametrize("gs", [17, 24, 32, 33, 48, 63])
+def test_padded_head_groups_on_the_64_lane_kernel(gs):
+    # fewer than 64 heads per K/V head: the missing heads are zero lanes of the operand
+    for (B, hkv, n) in ((2, 2, 700), (1, 1, 4100), (3, 1, 129)):
+        q, K, V, s = make(2200 + gs + n, B, gs * hkv, hkv, n, 128, 128)
+        ref = oracle.decode(q, K, V, s)
+        assert max_err(gpu_decode(q, K, V, s, expect_path=moa.PATH_GROUPED), ref) <= TOL, (gs, B, hkv, n)
+    lens = np.array([700, 3], np.int32)
+    q, K, V, s = make(2300 + gs, 2, gs * 2, 2, 700, 128, 128)
+    assert max_err(gpu_decode(q, K, V, s, seq_lens=lens, expect_path=moa.PATH_GROUPED),
+                   oracle.decode_varlen(q, K, V, lens, s)) <= TOL
+
+
+def test_long_dense_groups_with_larger_scores_on_the_single_chain_kernel():
+    # caches of 4096 rows and more run the 64-lane kernel whose scores are one 32-step chain
+    q, K, V, s = make(2120, 1, 64, 1, 8192, 128, 128, v_dist="uniform")
+    q, K = 2 * q, 2 * K
+    assert max_err(gpu_decode(q, K, V, s, expect_path=moa.PATH_GROUPED), oracle.decode(q, K, V, s)) <= TOL
+    q, K, V, s = make(2121, 2, 48, 1, 4096, 128, 128)
+    assert max_err(gpu_decode(q, K, V, s, expect_path=moa.PATH_GROUPED), oracle.decode(q, K, V, s)) <= TOL
