@@ -275,9 +275,10 @@ const char *moa_strerror(int code);
  *                        0 = automatic).  Larger groups are cut into neighbouring CTAs.
  *   MOA_OPT_DEPENDENT_LAUNCH : 1 (default) = the streaming kernels are launched with
  *                        programmatic stream serialisation, 0 = ordinary launches.
- *   MOA_OPT_GROUPED_OPERANDS : where the tensor-core kernel keeps the query and probability
- *                        operands of groups of 64 heads: 0 (default) = tensor memory,
- *                        1 = shared memory (the arrangement used for groups of 16 and 32).
+ *   MOA_OPT_GROUPED_OPERANDS : 0 (default) = groups of 17..64 heads may use the tensor-core kernel
+ *                        that keeps the query and probability operands in tensor memory
+ *                        (64 head lanes, smaller groups padded); 1 = only the kernel with
+ *                        these operands in shared memory (groups of exactly 16, 32, 64).
  * moa_last_path() reports which kernel family the last successful decode call used.
  */
 #define MOA_OPT_FORCE_PATH 1
@@ -287,7 +288,7 @@ const char *moa_strerror(int code);
 #define MOA_OPT_GROUPED_OPERANDS 5
 #define MOA_PATH_GENERIC   1   /* any d_k, d_v, alignment: one CTA per (batch, query head) */
 #define MOA_PATH_STREAM    2   /* split-sequence streaming kernel on the FMA units, d in {32,64,128} */
-#define MOA_PATH_GROUPED   3   /* tcgen05 tensor-core kernel for large groups (g_s in {16,32,64}, dense) */
+#define MOA_PATH_GROUPED   3   /* tcgen05 tensor-core kernels for groups of 17..64 heads (16 when forced), d = 128, dense layout */
 #define MOA_PATH_MMA       4   /* streaming kernel with warp-level MMA, groups of 8 or 16 heads, d_k, d_v in {64,128} */
 int moa_set_option(int option, int value);
 int moa_last_path(void);
