@@ -21,9 +21,11 @@
 //
 // Tensor memory (512 columns): Q (128), two score/probability regions (128 each; the
 // probabilities of a tile overwrite its scores), O (128).  The tensor core accumulates with
-// truncation, so chains are kept short: the scores of a tile are a chain of 32 steps, and the
-// weighted sum of every tile starts from zero and is folded into fp32 running values held in
-// registers (online softmax, eq. (2) with a running maximum per head).
+// truncation, so chains are kept short: the weighted sum of every tile starts from zero and is
+// folded into fp32 running values held in registers (online softmax, eq. (2) with a running
+// maximum per head).  The scores of a tile are one chain of 32 steps in the variant for long
+// caches and two chains of 16 (K_hi and K_lo products added in fp32 by the softmax group) in
+// the PRECISE variant, see the note at `precise` below.
 //
 // A thread that issues tcgen05.mma cannot look at a barrier without draining the tensor pipe
 // (measured: one shared-memory read between two products costs ~170 cycles of tensor time),
