@@ -483,7 +483,8 @@ static cudaError_t launch_grouped_cfg(const CUtensorMap &mk, const CUtensorMap &
 // the shared-memory-operand kernel, so the combine kernel is shared.
 template <bool PRECISE>
 static cudaError_t launch_grouped64_cfg(const CUtensorMap &mk, const CUtensorMap &mv, const CUtensorMap &mkt,
-                                        const CUtensorMap &mvt, const GroupedArgs &ga, int grid, cudaStream_t st)
+                                        const CUtensorMap &mvt, const GroupedArgs &ga, int grid, cudaStream_t st,
+                                        bool combine = true)
 {
     using C = Grouped64Cfg;
     static bool attr_set[kMaxDevices] = {};
@@ -501,7 +502,7 @@ static cudaError_t launch_grouped64_cfg(const CUtensorMap &mk, const CUtensorMap
     }
     count_launch();
     cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
+    if (e != cudaSuccess || !combine) return e;
     const long long warps = (long long)ga.batch * ga.h_q;
     grouped_combine_kernel<64><<<(int)warps, 128, 0, st>>>(ga);
     count_launch();
@@ -524,9 +525,21 @@ static cudaError_t launch_grouped64(const CUtensorMap &mk, const CUtensorMap &mv
                                     bool fused)
 {
     if (ga.seq_lens == nullptr && !fused && ga.n >= 4096) return launch_grouped64_cfg<false>(mk, mv, mkt, mvt, ga, grid, st);
-    if (ga.g_s == 64) return launch_grouped_cfg<64>(mk, mv, mkt, mvt, ga, grid, st);
-    if (ga.g_s == 32) return launch_grouped_cfg<32>(mk, mv, mkt, mvt, ga, grid, st);
-    return launch_grouped64_cfg<true>(mk, mv, mkt, mvt, ga, grid, st);
+    GroupedArgs rest = ga;
+    if (ga.seq_lens != nullptr && ga.n >= 4096 && ga.g_s == 64) {
+        // A ragged batch of 64-head groups in a long cache: the sequences of 4096 rows and more
+        // go to the single-chain kernel first (the CTAs of the other units leave at once), the
+        // shorter ones to the launch below; slots and splits are the same for both launches
+        // (with padded groups or groups of 32 the second launch has another slot size).
+        GroupedArgs longs = ga;
+        longs.len_lo = 4096;
+        cudaError_t e = launch_grouped64_cfg<false>(mk, mv, mkt, mvt, longs, grid, st, false);
+        if (e != cudaSuccess) return e;
+        rest.len_hi = 4096;
+    }
+    if (ga.g_s == 64) return launch_grouped_cfg<64>(mk, mv, mkt, mvt, rest, grid, st);
+    if (ga.g_s == 32) return launch_grouped_cfg<32>(mk, mv, mkt, mvt, rest, grid, st);
+    return launch_grouped64_cfg<true>(mk, mv, mkt, mvt, rest, grid, st);
 }
 
 static cudaError_t launch_generic(const DecodeArgs &a, cudaStream_t st)
@@ -644,6 +657,7 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
         ga.seq_lens = seq_lens; ga.len_bias = len_bias;
         ga.tailK = nullptr; ga.tailV = nullptr;
         ga.flat = 0;
+        ga.len_lo = 0; ga.len_hi = 0x7fffffff;
         CUtensorMap mkt = mk, mvt = mv;
         if (ragged) {
             // the last, partly filled tile of every unit, zero-padded (and the appended row of

@@ -150,6 +150,7 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
     const int b = sunit / a.h_kv_stored, h = sunit % a.h_kv_stored;
     const int unit = sunit;                                         // tensor-map coordinate
     const int len_b = grouped_len(a, b);           // 0: out-of-range length, the item is skipped
+    if (len_b < a.len_lo || len_b >= a.len_hi) return;   // another launch's unit (uniform for the CTA)
     const int tiles_total = (len_b + C::TILE - 1) / C::TILE;
     const int tiles_per_split = a.seq_lens ? (tiles_total + splits_u - 1) / splits_u : a.tiles_per_split;
     const int tile0 = split * tiles_per_split;

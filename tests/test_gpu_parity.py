@@ -524,3 +524,35 @@ def test_long_dense_groups_with_larger_scores_on_the_single_chain_kernel():
     assert max_err(gpu_decode(q, K, V, s, expect_path=moa.PATH_GROUPED), oracle.decode(q, K, V, s)) <= TOL
     q, K, V, s = make(2121, 2, 48, 1, 4096, 128, 128)
     assert max_err(gpu_decode(q, K, V, s, expect_path=moa.PATH_GROUPED), oracle.decode(q, K, V, s)) <= TOL
+
+
+@pytest.mark.parametrize("hq,hkv", [(64, 1), (128, 2), (48, 1)])
+def test_fused_steps_on_a_ragged_batch_of_long_and_short_sequences(hq, hkv):
+    """Groups on the tcgen05 kernels, capacity above 4096 rows: sequences of 4096 rows and more
+    and shorter ones are served by different kernels within one step."""
+    B, n_max, D, steps = 4, 4400, 128, 3
+    w = mi.Workload("ms", 3100 + hq, B, hq, hkv, n_max, D, D, steps=steps)
+    K, V = w.K(), w.V()
+    lens = np.array([4300, 97, 4095, 4096], np.int32)
+    for b in range(B):
+        K[b, :, lens[b]:] = 0
+        V[b, :, lens[b]:] = 0
+    gK, gV, glens = Guarded(K), Guarded(V), Guarded(lens)
+    gws, nbytes = workspace_for(B, hq, hkv, n_max, D, D)
+    gout = Guarded(shape=(B, hq, D))
+    for t in range(steps):
+        kn, vn, qt = w.k_new(t), w.v_new(t), w.q_step(t)
+        gk, gv, gq = Guarded(kn), Guarded(vn), Guarded(qt)
+        moa.moa_decode_step(gq.ptr, gK.ptr, gV.ptr, gk.ptr, gv.ptr, gout.ptr, glens.ptr, B, hq, hkv, n_max, D, D,
+                            w.scale, gws.ptr, nbytes)
+        torch.cuda.synchronize()
+        assert moa.moa_last_path() == moa.PATH_GROUPED
+        oracle.kv_append(K, V, kn, vn, lens)
+        lens = lens + 1
+        assert max_err(gout.host(), oracle.decode_varlen(qt, K, V, lens, w.scale)) <= TOL, t
+        assert np.array_equal(glens.host(), lens)
+    assert moa.moa_device_status() == 0
+    assert np.array_equal(gK.host().view(np.uint32), K.view(np.uint32))
+    assert np.array_equal(gV.host().view(np.uint32), V.view(np.uint32))
+    for g in (gK, gV, glens, gws, gout):
+        assert g.guards_intact()
