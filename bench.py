@@ -209,6 +209,9 @@ class DenseRun:
 
     def reset(self):
         self.i = 0
+        # every sequence of this workload has n rows after the append: tell the library (it cannot
+        # see the lengths, which live on the device)
+        self.moa.moa_set_option(self.moa.OPT_MIN_ROWS_HINT, self.w.n)
 
     def e2e_step(self):
         w, h = self.w, self.host
@@ -294,6 +297,7 @@ class MultiStepRun:
     def reset(self):
         self.lens.copy_(self.lens0)
         self.t = 0
+        self.moa.moa_set_option(self.moa.OPT_MIN_ROWS_HINT, 0)     # ragged lengths from 512 rows: no promise
 
 
 def time_steps(run, steps, warmup, sampler=None, bracket=False):
@@ -302,6 +306,7 @@ def time_steps(run, steps, warmup, sampler=None, bracket=False):
     the dominant decode kernel (which costs a few microseconds per launch)."""
     import torch
     moa = run.moa
+    run.reset()
     for _ in range(warmup):
         run.step()
     torch.cuda.synchronize()
@@ -600,7 +605,7 @@ def main():
                 "config": {"workload": wname, "batch_per_gpu": w.batch, "h_q": w.h_q, "h_kv": w.h_kv,
                            "n": w.n, "d_k": w.d_k, "d_v": w.d_v, "parallelism": "dp%d (batch-sharded, no collective)" % world,
                            "step": ("moa_decode_step: append + attend over ragged lengths + length advance, one launch" if wname == "multi_step"
-                                    else "moa_append_decode: kv append at row n-1 + decode attention over n rows, %d launch(es) per step"
+                                    else "moa_append_decode: kv append at row n-1 + decode attention over n rows (MOA_OPT_MIN_ROWS_HINT = n), %d launch(es) per step"
                                     % max(1, launches // max(1, args.steps))),
                            "l2": l2_note},
                 "us_per_step": ms * 1e3, "clocks": clocks, "e2e": e2e, "gpu_launches": launches,

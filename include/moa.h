@@ -279,6 +279,14 @@ const char *moa_strerror(int code);
  *                        that keeps the query and probability operands in tensor memory
  *                        (64 head lanes, smaller groups padded); 1 = only the kernel with
  *                        these operands in shared memory (groups of exactly 16, 32, 64).
+ *   MOA_OPT_MIN_ROWS_HINT : the caller's promise that every sequence of the calls that follow
+ *                        has at least this many rows after the call (0 = no promise, the
+ *                        default).  Lengths live on the device, so without the promise a
+ *                        ragged batch of large head groups is served by two launches (one
+ *                        for sequences of 4096 rows and more, one for shorter ones, which
+ *                        need the more accurate kernel); with a promise of >= 4096 by one.
+ *                        A broken promise costs accuracy on the short sequences (errors up
+ *                        to about 1e-5), nothing else.
  * moa_last_path() reports which kernel family the last successful decode call used.
  */
 #define MOA_OPT_FORCE_PATH 1
@@ -286,6 +294,7 @@ const char *moa_strerror(int code);
 #define MOA_OPT_GROUPED_HEADS 3
 #define MOA_OPT_DEPENDENT_LAUNCH 4
 #define MOA_OPT_GROUPED_OPERANDS 5
+#define MOA_OPT_MIN_ROWS_HINT 6
 #define MOA_PATH_GENERIC   1   /* any d_k, d_v, alignment: one CTA per (batch, query head) */
 #define MOA_PATH_STREAM    2   /* split-sequence streaming kernel on the FMA units, d in {32,64,128} */
 #define MOA_PATH_GROUPED   3   /* tcgen05 tensor-core kernels for groups of 17..64 heads (16 when forced), d = 128, dense layout */

@@ -360,6 +360,7 @@ struct GroupedPlan {
 };
 static int g_grouped_heads = 0;   // MOA_OPT_GROUPED_HEADS: 0 = automatic
 static int g_grouped_operands = 0;   // MOA_OPT_GROUPED_OPERANDS
+static int g_min_rows_hint = 0;      // MOA_OPT_MIN_ROWS_HINT
 
 static GroupedPlan plan_grouped(const DeviceState &s, int batch, int h_q, int h_kv, int n, int d_k, int d_v)
 {
@@ -525,6 +526,8 @@ static cudaError_t launch_grouped64(const CUtensorMap &mk, const CUtensorMap &mv
                                     bool fused)
 {
     if (ga.seq_lens == nullptr && !fused && ga.n >= 4096) return launch_grouped64_cfg<false>(mk, mv, mkt, mvt, ga, grid, st);
+    // ragged, but the caller promises that no sequence is short: one launch of the single-chain kernel
+    if (g_min_rows_hint >= 4096 && ga.n >= 4096) return launch_grouped64_cfg<false>(mk, mv, mkt, mvt, ga, grid, st);
     GroupedArgs rest = ga;
     if (ga.seq_lens != nullptr && ga.n >= 4096 && ga.g_s == 64) {
         // A ragged batch of 64-head groups in a long cache: the sequences of 4096 rows and more
@@ -1112,6 +1115,11 @@ int moa_set_option(int option, int value)
     if (option == MOA_OPT_GROUPED_OPERANDS) {
         if (value != 0 && value != 1) return MOA_ERR_INVALID;
         g_grouped_operands = value;
+        return MOA_OK;
+    }
+    if (option == MOA_OPT_MIN_ROWS_HINT) {
+        if (value < 0) return MOA_ERR_INVALID;
+        g_min_rows_hint = value;
         return MOA_OK;
     }
     if (option == MOA_OPT_DEPENDENT_LAUNCH) {

@@ -556,3 +556,22 @@ def test_fused_steps_on_a_ragged_batch_of_long_and_short_sequences(hq, hkv):
     assert np.array_equal(gV.host().view(np.uint32), V.view(np.uint32))
     for g in (gK, gV, glens, gws, gout):
         assert g.guards_intact()
+
+
+def test_minimum_rows_promise_saves_the_second_launch_of_a_ragged_step():
+    B, hq, hkv, n_max, D = 2, 64, 1, 4500, 128
+    q, K, V, s = make(3200, B, hq, hkv, n_max, D, D)
+    lens = np.array([4400, 4100], np.int32)
+    ref = oracle.decode_varlen(q, K, V, lens, s)
+    launches = {}
+    for promise in (0, 4096):
+        moa.moa_set_option(moa.OPT_MIN_ROWS_HINT, promise)
+        try:
+            moa.moa_profile(1)
+            out = gpu_decode(q, K, V, s, seq_lens=lens, expect_path=moa.PATH_GROUPED)
+            launches[promise] = moa.moa_profile_read()[2]
+            moa.moa_profile(0)
+        finally:
+            moa.moa_set_option(moa.OPT_MIN_ROWS_HINT, 0)
+        assert max_err(out, ref) <= TOL, promise
+    assert launches[4096] == launches[0] - 1
