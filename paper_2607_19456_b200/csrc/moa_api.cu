@@ -529,11 +529,12 @@ static cudaError_t launch_grouped64(const CUtensorMap &mk, const CUtensorMap &mv
     // ragged, but the caller promises that no sequence is short: one launch of the single-chain kernel
     if (g_min_rows_hint >= 4096 && ga.n >= 4096) return launch_grouped64_cfg<false>(mk, mv, mkt, mvt, ga, grid, st);
     GroupedArgs rest = ga;
-    if (ga.seq_lens != nullptr && ga.n >= 4096 && ga.g_s == 64) {
-        // A ragged batch of 64-head groups in a long cache: the sequences of 4096 rows and more
-        // go to the single-chain kernel first (the CTAs of the other units leave at once), the
-        // shorter ones to the launch below; slots and splits are the same for both launches
-        // (with padded groups or groups of 32 the second launch has another slot size).
+    const bool two_launches = ga.seq_lens != nullptr && ga.n >= 4096;
+    if (two_launches) {
+        // A ragged batch in a long cache: the sequences of 4096 rows and more go to the
+        // single-chain kernel first (the CTAs of the other units leave at once), the shorter
+        // ones to the launch below; slots and splits are the same for both launches, so the
+        // second one has to use 64 head lanes as well.
         GroupedArgs longs = ga;
         longs.len_lo = 4096;
         cudaError_t e = launch_grouped64_cfg<false>(mk, mv, mkt, mvt, longs, grid, st, false);
@@ -541,7 +542,7 @@ static cudaError_t launch_grouped64(const CUtensorMap &mk, const CUtensorMap &mv
         rest.len_hi = 4096;
     }
     if (ga.g_s == 64) return launch_grouped_cfg<64>(mk, mv, mkt, mvt, rest, grid, st);
-    if (ga.g_s == 32) return launch_grouped_cfg<32>(mk, mv, mkt, mvt, rest, grid, st);
+    if (ga.g_s == 32 && !two_launches) return launch_grouped_cfg<32>(mk, mv, mkt, mvt, rest, grid, st);
     return launch_grouped64_cfg<true>(mk, mv, mkt, mvt, rest, grid, st);
 }
 

@@ -526,7 +526,7 @@ def test_long_dense_groups_with_larger_scores_on_the_single_chain_kernel():
     assert max_err(gpu_decode(q, K, V, s, expect_path=moa.PATH_GROUPED), oracle.decode(q, K, V, s)) <= TOL
 
 
-@pytest.mark.parametrize("hq,hkv", [(64, 1), (128, 2), (48, 1)])
+@pytest.mark.parametrize("hq,hkv", [(64, 1), (128, 2), (48, 1), (32, 1), (34, 2)])
 def test_fused_steps_on_a_ragged_batch_of_long_and_short_sequences(hq, hkv):
     """Groups on the tcgen05 kernels, capacity above 4096 rows: sequences of 4096 rows and more
     and shorter ones are served by different kernels within one step."""
