@@ -92,7 +92,7 @@ def decode_f64(q, K, V, scale):
 
 
 def decode_f32(q, K, V, scale):
-    """Single-precision three-pass variant (timing baseline / sanity band)."""
+    """Algorithm 1 with every intermediate in single precision (timing baseline / sanity band)."""
     q, K, V = _c(q, np.float32), _c(K, np.float32), _c(V, np.float32)
     B, hq, hkv, n, dk, dv = _shapes(q, K, V)
     out = np.empty((B, hq, dv), np.float32)

@@ -146,6 +146,29 @@ int moa_oracle_decode_f64(const double *q, const double *K, const double *V, dou
     return 0;
 }
 
+/* One head in single precision: the same three steps as one_head_f32in, with every
+ * product, sum, exponential and division rounded to fp32 (eqs. (1)-(3) as stated: the
+ * weights are normalised, a[l] = e[l] / Z, before Step III uses them). */
+static void one_head_f32(const float *q, const float *Kg, const float *Vg, float *out,
+                         int rows, int d_k, int d_v, float scale, float *s, float *a)
+{
+    for (int l = 0; l < rows; l++) {                         /* Step I, eq. (1) */
+        float dot = 0.0f;
+        for (int j = 0; j < d_k; j++) dot += q[j] * Kg[(size_t)l * d_k + j];
+        s[l] = scale * dot;
+    }
+    float m = -INFINITY;                                     /* Step II, eq. (2) */
+    for (int l = 0; l < rows; l++) if (s[l] > m) m = s[l];
+    float Z = 0.0f;
+    for (int l = 0; l < rows; l++) { a[l] = expf(s[l] - m); Z += a[l]; }
+    for (int l = 0; l < rows; l++) a[l] = a[l] / Z;
+    for (int d = 0; d < d_v; d++) {                          /* Step III, eq. (3) */
+        float acc = 0.0f;
+        for (int l = 0; l < rows; l++) acc += a[l] * Vg[(size_t)l * d_v + d];
+        out[d] = acc;
+    }
+}
+
 int moa_oracle_decode_f32(const float *q, const float *K, const float *V, float *out,
                           int batch, int h_q, int h_kv, int n, int d_k, int d_v,
                           float scale)
@@ -157,41 +180,22 @@ int moa_oracle_decode_f32(const float *q, const float *K, const float *V, float 
 #pragma omp parallel
     {
         float *s = (float *)malloc(sizeof(float) * (size_t)n);
-        float *e = (float *)malloc(sizeof(float) * (size_t)n);
-        if (!s || !e) {
+        float *a = (float *)malloc(sizeof(float) * (size_t)n);
+        if (!s || !a) {
 #pragma omp atomic write
             failed = 1;
         }
 #pragma omp for schedule(dynamic, 1)
         for (long bg = 0; bg < (long)batch * h_q; bg++) {
-            if (!s || !e) continue;
+            if (!s || !a) continue;
             const int b = (int)(bg / h_q), g = (int)(bg % h_q);
-            const size_t slab = (size_t)b * h_kv + g / group;
-            const float *qq = q + (size_t)bg * d_k;
-            const float *Kg = K + slab * (size_t)n * d_k;
-            const float *Vg = V + slab * (size_t)n * d_v;
-            float *o = out + (size_t)bg * d_v;
-            /* pass 1: scores and their maximum */
-            float m = -INFINITY;
-            for (int l = 0; l < n; l++) {
-                float dot = 0.0f;
-                for (int j = 0; j < d_k; j++) dot += qq[j] * Kg[(size_t)l * d_k + j];
-                s[l] = scale * dot;
-                if (s[l] > m) m = s[l];
-            }
-            /* pass 2: exponentials and the denominator */
-            float Z = 0.0f;
-            for (int l = 0; l < n; l++) { e[l] = expf(s[l] - m); Z += e[l]; }
-            /* pass 3: weighted sum, one cached row at a time */
-            const float inv_Z = 1.0f / Z;
-            for (int d = 0; d < d_v; d++) o[d] = 0.0f;
-            for (int l = 0; l < n; l++) {
-                const float w = e[l] * inv_Z;
-                for (int d = 0; d < d_v; d++) o[d] += w * Vg[(size_t)l * d_v + d];
-            }
+            const size_t slab = (size_t)b * h_kv + g / group;     /* psi-selection */
+            one_head_f32(q + (size_t)bg * d_k, K + slab * (size_t)n * d_k,
+                         V + slab * (size_t)n * d_v, out + (size_t)bg * d_v,
+                         n, d_k, d_v, scale, s, a);
         }
         free(s);
-        free(e);
+        free(a);
     }
     return failed ? -1 : 0;
 }

@@ -46,10 +46,9 @@ int moa_oracle_decode_f64(const double *q, const double *K, const double *V, dou
                           int batch, int h_q, int h_kv, int n, int d_k, int d_v,
                           double scale);
 
-/* The three passes in single precision, sequential over l, in the order the paper's
- * C kernel section describes (scores with a running max, exponentials with a running
- * sum, weights e*(1/Z) accumulated row by row).  A timing baseline and a sanity band;
- * not the parity reference. */
+/* Algorithm 1 (eqs. (1)-(3)) with every intermediate in single precision: what a
+ * straightforward fp32 CPU implementation of the definition gives.  A timing baseline and
+ * a sanity band for the fp32 error; not the parity reference. */
 int moa_oracle_decode_f32(const float *q, const float *K, const float *V, float *out,
                           int batch, int h_q, int h_kv, int n, int d_k, int d_v,
                           float scale);

@@ -222,7 +222,7 @@ def test_matches_torch_sdpa_double(n):
                                          scale=scale).squeeze(2).numpy()
     got = oracle.decode(q, K, V, scale)
     assert np.max(np.abs(got - ref)) < 1e-7
-    # the single-precision three-pass variant sits in the paper's fp32 error band
+    # the single-precision variant sits in the paper's fp32 error band
     got32 = oracle.decode_f32(q, K, V, scale)
     assert np.max(np.abs(got32 - ref)) < 2e-6
 
