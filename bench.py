@@ -10,9 +10,12 @@ Prints ONE JSON line (rank 0).  `value` is the achieved algorithmic HBM bandwidt
 whole job (bytes of the paper's traffic model per step, summed over ranks, divided by
 the step time, max over ranks); `ms_per_step` is the step time.
 
-With N > 1 (launched under torchrun, one rank per GPU) every rank runs its own shard of
-an N-times larger batch: the path has no exchange step, so there is no data-path
-collective and the scaling is weak.
+With N > 1 every rank (one per GPU) runs its own shard of an N-times larger batch: the path
+has no exchange step, so there is no data-path collective and the scaling is weak.  Under
+torchrun the ranks are the launcher's; started plainly with `--gpus N`, this script starts
+the N ranks itself (one child process per GPU, rendezvous on 127.0.0.1).  `--split seq`
+instead cuts the cached rows of one workload over the ranks (one all-gather of the partial
+triples per step; strong scaling).
 
 `--impl reference` times the plain CPU oracle (the only reference there is for this
 paper) on a bounded sample of the same workload, on the host cores.
@@ -39,13 +42,33 @@ FALLBACK_HBM_GBS = 6650.0
 L2_BYTES_ASSUMED = 126 * 1024 * 1024
 
 # DRAM traffic of one launch of the dominant kernel, from an ncu capture
-# (dram__bytes_read.sum + dram__bytes_write.sum), per workload; the summaries these come
-# from are kept as text under profiles/.  None = not captured.
-NCU_TRAFFIC_BYTES = {
-    "gqa": 1074650112 + 3750144,        # profiles/stream_decode_kernel_gqa.md (full-size launch)
-    "mqa_long": 537066496 + 314112,     # profiles/grouped64_decode_kernel_mqa_long.md (full-size launch)
-    "extra_group8_d128": 1075588864 + 4157440,   # profiles/mma_decode_kernel_group8_d128.md (full-size launch)
+# (dram__bytes_read.sum + dram__bytes_write.sum), per workload.  Every entry is stamped with
+# a digest of the kernel sources it was captured with; when those files have changed since,
+# the figure is stale and the line reports null instead.
+NCU_TRAFFIC = {
+    "gqa": {"bytes": 1074650112 + 3750144, "sources": ["moa_stream.cuh", "moa_device.cuh"], "digest": ""},
+    "extra_group8_d128": {"bytes": 1075588864 + 4157440, "sources": ["moa_mma.cuh", "moa_device.cuh"], "digest": ""},
+    "mqa_long": {"bytes": 537066496 + 314112, "sources": ["moa_grouped64.cuh", "moa_grouped.cuh", "moa_tc.cuh"], "digest": ""},
 }
+
+
+def source_digest(files):
+    import hashlib
+    h = hashlib.sha256()
+    for f in files:
+        with open(os.path.join(ROOT, "paper_2607_19456_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic(wname):
+    e = NCU_TRAFFIC.get(wname)
+    if not e:
+        return None
+    try:
+        return e["bytes"] if source_digest(e["sources"]) == e["digest"] else None
+    except OSError:
+        return None
 
 
 def env_int(name, default):
@@ -157,7 +180,9 @@ class DenseRun:
         self.bytes_per_step = moa.moa_min_bytes(B, hq, hkv, n, dk, dv) + 2 * B * hkv * (dk + dv) * 4
         self.decode_bytes = moa.moa_min_bytes(B, hq, hkv, n, dk, dv)
         one = self.decode_bytes
-        self.nsets = 1 if one >= 2 * L2_BYTES_ASSUMED else min(4096, -(-2 * L2_BYTES_ASSUMED // one))
+        # consecutive steps never touch the same buffers: at least two independent sets, and as
+        # many as it takes to exceed twice the L2 size
+        self.nsets = max(2, min(4096, -(-2 * L2_BYTES_ASSUMED // one)))
         S = self.nsets
         ws = mi.small_like(w, seed=w.seed + seed_shift)
         self.host = None
@@ -196,8 +221,7 @@ class DenseRun:
         self.wsbuf = torch.empty(self.ws_bytes, dtype=torch.uint8, device=device)
         self.wsptr = self.wsbuf.data_ptr()
         self.stream = torch.cuda.current_stream().cuda_stream
-        self.l2_note = ("inputs larger than L2 (%.0f MB per step)" % (one / 1e6)) if S == 1 else \
-            ("rotating over %d buffer sets (%.0f MB total, larger than L2)" % (S, S * one / 1e6))
+        self.l2_note = "rotating over %d buffer sets of %.0f MB (%.0f MB in total; L2 is 126 MB)" % (S, one / 1e6, S * one / 1e6)
 
     def step(self):
         w, m = self.w, self.moa
@@ -209,9 +233,12 @@ class DenseRun:
 
     def reset(self):
         self.i = 0
-        # every sequence of this workload has n rows after the append: tell the library (it cannot
-        # see the lengths, which live on the device)
-        self.moa.moa_set_option(self.moa.OPT_MIN_ROWS_HINT, self.w.n)
+
+    def profile(self, mode):
+        self.moa.moa_profile(mode)
+
+    def profile_read(self):
+        return self.moa.moa_profile_read()
 
     def e2e_step(self):
         w, h = self.w, self.host
@@ -297,44 +324,93 @@ class MultiStepRun:
     def reset(self):
         self.lens.copy_(self.lens0)
         self.t = 0
-        self.moa.moa_set_option(self.moa.OPT_MIN_ROWS_HINT, 0)     # ragged lengths from 512 rows: no promise
+
+    def profile(self, mode):
+        self.moa.moa_profile(mode)
+
+    def profile_read(self):
+        return self.moa.moa_profile_read()
 
 
-def time_steps(run, steps, warmup, sampler=None, bracket=False):
-    """-> (ms per step, decode-kernel ms per launch or None, launches in the timed region, clocks).
+class CudaSide:
+    """Where the steps run and how they are timed: one GPU, CUDA events on the current stream."""
+    backend, device = "nccl", "cuda"
+
+    def __init__(self, local):
+        import torch
+        self.torch = torch
+        torch.cuda.set_device(local)
+
+    def sync(self):
+        self.torch.cuda.synchronize()
+
+    def mark(self):
+        e = self.torch.cuda.Event(enable_timing=True)
+        e.record()
+        return e
+
+    @staticmethod
+    def ms_between(e0, e1):
+        return e0.elapsed_time(e1)
+
+
+class HostSide:
+    """The same protocol without a GPU (gloo ranks, wall clock): it exists so that the launch
+    and reduction path of N ranks can be exercised on a CPU-only machine with a stand-in
+    for the kernels; bench.py itself never selects it."""
+    backend, device = "gloo", "cpu"
+
+    def sync(self):
+        pass
+
+    def mark(self):
+        return time.perf_counter()
+
+    @staticmethod
+    def ms_between(e0, e1):
+        return (e1 - e0) * 1e3
+
+
+def time_steps(run, steps, warmup, side, sampler=None, bracket=False, segment=0):
+    """-> (ms per step, decode-kernel ms per launch or None, launches in the timed region, clocks,
+    [ms per step of the first and of the last `segment` steps] or None).
     With bracket=True the library also records a CUDA event pair around every launch of
     the dominant decode kernel (which costs a few microseconds per launch)."""
-    import torch
-    moa = run.moa
     run.reset()
     for _ in range(warmup):
         run.step()
-    torch.cuda.synchronize()
+    side.sync()
     if isinstance(run, MultiStepRun):
         run.reset()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
-    torch.cuda.synchronize()
+    side.sync()
     if sampler:
         sampler.start()
-    moa.moa_profile(2 if bracket else 1)
-    e0.record()
-    for _ in range(steps):
-        run.step()
-    e1.record()
-    torch.cuda.synchronize()
-    kern_ms, kern_n, launches = moa.moa_profile_read()
+    run.profile(2 if bracket else 1)
+    cuts = sorted({0, steps} | ({segment, steps - segment} if 0 < segment and 2 * segment <= steps else set()))
+    marks = {}
+    for i in range(steps + 1):
+        if i in cuts:
+            marks[i] = side.mark()
+        if i < steps:
+            run.step()
+    side.sync()
+    kern_ms, kern_n, launches = run.profile_read()
     LAST_BRACKETED.clear()
     if bracket and kern_n:
-        LAST_BRACKETED.extend(moa.moa_profile_launch_ms(i) * 1e3 for i in range(int(kern_n)))
-    moa.moa_profile(0)
+        LAST_BRACKETED.extend(run.moa.moa_profile_launch_ms(i) * 1e3 for i in range(int(kern_n)))
+    run.profile(0)
     clocks = sampler.stop() if sampler else None
     barrier()
-    ms = e0.elapsed_time(e1) / steps
-    return ms, (kern_ms / kern_n if kern_n else None), launches, clocks
+    ms = side.ms_between(marks[0], marks[steps]) / steps
+    segs = None
+    if len(cuts) == 4:
+        segs = [side.ms_between(marks[0], marks[segment]) / segment,
+                side.ms_between(marks[steps - segment], marks[steps]) / segment]
+    return ms, (kern_ms / kern_n if kern_n else None), launches, clocks, segs
 
 
-_DIST = {"on": False}
+_DIST = {"on": False, "device": "cuda"}
 LAST_BRACKETED = []      # per-launch event times (us) of the last bracketed pass
 
 
@@ -348,7 +424,49 @@ def max_over_ranks(x):
     if not _DIST["on"]:
         return x
     from paper_2607_19456_b200 import shard
-    return shard.reduce_step_time(x, device="cuda")
+    return shard.reduce_step_time(x, device=_DIST["device"])
+
+
+# --------------------------------------------------------------------------------------
+# starting the ranks (plain `python bench.py --gpus N`)
+# --------------------------------------------------------------------------------------
+def free_port():
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        return sk.getsockname()[1]
+
+
+def rank_env(rank, world, port, base=None):
+    """Environment of one child rank: what torchrun would have set, rendezvous on 127.0.0.1."""
+    env = dict(os.environ if base is None else base)
+    env.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world),
+               MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    return env
+
+
+def spawn_ranks(world, argv):
+    """One child process per GPU running this script with the same arguments; rank 0 prints
+    the JSON line.  Returns the first non-zero exit code (children still running are then
+    terminated by their PIDs)."""
+    import subprocess
+    port = free_port()
+    procs = [subprocess.Popen([sys.executable, os.path.abspath(__file__)] + list(argv), env=rank_env(r, world, port))
+             for r in range(world)]
+    rc = 0
+    pending = list(procs)
+    while pending:
+        for p in list(pending):
+            code = p.poll()
+            if code is None:
+                continue
+            pending.remove(p)
+            if code != 0 and rc == 0:
+                rc = code
+                for other in pending:
+                    other.terminate()
+        time.sleep(0.05)
+    return rc
 
 
 # --------------------------------------------------------------------------------------
@@ -418,77 +536,183 @@ def run_reference(args, wname):
 
 
 # --------------------------------------------------------------------------------------
-def main():
+# one sampled parity figure per workload (oracle on one unit of the buffers just timed)
+# --------------------------------------------------------------------------------------
+def sampled_parity(run, w):
+    """Max abs error of the last timed step's output against the oracle on a sample: for the
+    dense workloads the first and the last (batch, kv head) unit of buffer set 0, for the
+    multi-step workload sequence 0 (all heads).  The inputs are read back from the device."""
+    import oracle
+    if isinstance(run, MultiStepRun):
+        if run.t == 0:
+            return None
+        lens = (run.lens0_h[:1] + run.t).astype(np.int32)
+        q = run.q[run.t - 1, :1].cpu().numpy()
+        ref = oracle.decode_varlen(q, run.K[:1].cpu().numpy(), run.V[:1].cpu().numpy(), lens, w.scale)
+        return float(np.max(np.abs(run.out[:1].cpu().numpy().astype(np.float64) - ref)))
+    used = (run.i - 1) % run.nsets if run.i > 0 else 0
+    g, worst = w.group, 0.0
+    for b, h in {(0, 0), (w.batch - 1, w.h_kv - 1)}:
+        q = run.q[used, b:b + 1, h * g:(h + 1) * g].cpu().numpy()
+        K = run.K[used, b:b + 1, h:h + 1].cpu().numpy()
+        V = run.V[used, b:b + 1, h:h + 1].cpu().numpy()
+        got = run.out[used, b:b + 1, h * g:(h + 1) * g].cpu().numpy()
+        worst = max(worst, float(np.max(np.abs(got.astype(np.float64) - oracle.decode(q, K, V, w.scale)))))
+    return worst
+
+
+# --------------------------------------------------------------------------------------
+# sequence split over the ranks (--split seq): one all-gather of partial triples per step
+# --------------------------------------------------------------------------------------
+class SeqSplitRun:
+    """Every rank holds a contiguous range of the cached rows of every (batch, kv head) of one
+    workload; a step is moa_decode_attn_partial over the local rows, one all-gather of
+    batch * h_q * (d_v + 4) floats, and moa_combine_partials (in rank order)."""
+
+    def __init__(self, w, rank, world, device="cuda"):
+        import torch
+        import paper_2607_19456_b200 as moa
+        from paper_2607_19456_b200 import shard
+        self.moa, self.torch, self.w, self.shard = moa, torch, w, shard
+        start, count = shard.shard_rows(w.n, world, rank, align=128)
+        self.n_local = count
+        B, hq, hkv, dk, dv = w.batch, w.h_q, w.h_kv, w.d_k, w.d_v
+        g = torch.Generator(device=device).manual_seed(w.seed + 17 * rank)
+        self.nsets = 2
+        self.q = torch.randn((B, hq, dk), device=device, generator=torch.Generator(device=device).manual_seed(w.seed))
+        self.K = torch.randn((2, B, hkv, max(count, 1), dk), device=device, generator=g)
+        self.V = torch.randn((2, B, hkv, max(count, 1), dv), device=device, generator=g)
+        if w.v_dist == "uniform":
+            self.V.uniform_(-1, 1, generator=g)
+        self.out = torch.zeros((B, hq, dv), device=device)
+        self.decode_bytes = moa.moa_min_bytes(B, hq, hkv, w.n, dk, dv)
+        self.bytes_per_step = self.decode_bytes            # whole job (the rows of all ranks)
+        self.i = 0
+        self.l2_note = "rotating over 2 buffer sets of the local rows"
+
+    def step(self):
+        s = self.i % 2
+        self.i += 1
+        K = self.K[s][:, :, :self.n_local]
+        V = self.V[s][:, :, :self.n_local]
+        self.shard.seq_split_decode(self.q, K, V, self.out, self.w.scale)
+
+    def reset(self):
+        self.i = 0
+
+    def profile(self, mode):
+        self.moa.moa_profile(mode)
+
+    def profile_read(self):
+        return self.moa.moa_profile_read()
+
+
+# --------------------------------------------------------------------------------------
+def parse_args(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=500)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=list(mi.WORKLOADS) + list(EXTRA_WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--split", default="batch", choices=["batch", "seq"],
+                    help="what is cut over the ranks: the batch (no collective) or the cached rows (one all-gather)")
     ap.add_argument("--no-others", action="store_true", help="skip the timing-only lines of the other workloads")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling on a small case)")
     ap.add_argument("--n", type=int, default=0, help="override the workload's cached tokens (profiling on a small case)")
-    args = ap.parse_args()
+    args = ap.parse_args(argv)
     if args.warmup < 3:
         args.warmup = 3
-    wname = args.workload
+    return args
 
+
+def main(argv=None):
+    argv = sys.argv[1:] if argv is None else argv
+    args = parse_args(argv)
     if args.impl == "reference":
-        run_reference(args, wname)
-        return
-
+        run_reference(args, args.workload)
+        return 0
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        return spawn_ranks(args.gpus, argv)               # the children come back here with the rank environment
     import torch
-    import paper_2607_19456_b200 as moa
-
-    rank, world, local = env_int("RANK", 0), env_int("WORLD_SIZE", 1), env_int("LOCAL_RANK", 0)
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: libmoa has no CPU path")
-    torch.cuda.set_device(local)
+    run_rank(args, CudaSide(env_int("LOCAL_RANK", 0)))
+    return 0
+
+
+def run_rank(args, side, make_run=None):
+    """One rank of the benchmark.  `make_run(workload, rank, world)` (tests only) replaces the
+    object whose step() is timed."""
+    import torch
+    rank, world, local = env_int("RANK", 0), env_int("WORLD_SIZE", 1), env_int("LOCAL_RANK", 0)
+    wname = args.workload
+    on_gpu = isinstance(side, CudaSide)
     if world > 1:
         import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-        _DIST["on"] = True
-    moa.lib()                                           # fail loudly if the library is missing
+        if on_gpu:
+            dist.init_process_group(side.backend, device_id=torch.device("cuda", local))
+        else:
+            dist.init_process_group(side.backend)
+        _DIST["on"], _DIST["device"] = True, side.device
+    moa = None
+    if on_gpu:
+        import paper_2607_19456_b200 as moa
+        moa.lib()                                       # fail loudly if the library is missing
 
     w = mi.WORKLOADS[wname] if wname in mi.WORKLOADS else EXTRA_WORKLOADS[wname]
     if args.batch > 0:
         w = mi.small_like(w, batch=args.batch)
     if args.n > 0 and wname != "multi_step":
         w = mi.small_like(w, n=args.n)
-    if wname == "multi_step":
+    seq_split = args.split == "seq" and wname != "multi_step"
+    if make_run is not None:
+        run = make_run(w, rank, world)
+    elif seq_split:
+        run = SeqSplitRun(w, rank, world)
+    elif wname == "multi_step":
         args.steps = min(args.steps, w.steps - args.warmup)
         run = MultiStepRun(w, seed_shift=rank)
     else:
         run = DenseRun(w, seed_shift=rank, host_inputs=True)
 
     l2_note = run.l2_note
-    sampler = ClockSampler(local)
-    ms, _, launches, clocks = time_steps(run, args.steps, args.warmup, sampler)
+    sampler = ClockSampler(local) if on_gpu else None
+    ms, _, launches, clocks, segs = time_steps(run, args.steps, args.warmup, side, sampler, segment=300)
+    per_rank = ms
     ms = max_over_ranks(ms)
+    per_rank_all = None
+    if world > 1:
+        import torch.distributed as dist
+        per_rank_all = [None] * world
+        dist.all_gather_object(per_rank_all, per_rank * 1e3)
     # second pass: the same steps with an event pair around every launch of the dominant kernel
-    bsteps = min(args.steps, 200)
-    _, kern_ms, _, _ = time_steps(run, bsteps, 3, None, bracket=True)
-    if wname == "multi_step":
+    kern_ms = None
+    if on_gpu:
+        _, kern_ms, _, _, _ = time_steps(run, min(args.steps, 200), 3, side, None, bracket=True)
+    if wname == "multi_step" and make_run is None:
         step_bytes = run.bytes_for_steps(0, args.steps) / args.steps
         decode_bytes = step_bytes
     else:
         step_bytes, decode_bytes = run.bytes_per_step, run.decode_bytes
-    value = world * step_bytes / (ms * 1e-3) / 1e9
+    ranks_of_work = 1 if seq_split else world             # seq split: the bytes already are the whole job's
+    value = ranks_of_work * step_bytes / (ms * 1e-3) / 1e9
 
     peak, peak_kind = measured_hbm_peak()
     roof = None
     single_launch = (launches == args.steps)
-    if single_launch or kern_ms:
+    if on_gpu and (single_launch or kern_ms):
         # One launch per step: the kernel's average launch duration over the timed region is
         # the event-timed region divided by its launches (this includes the gap between
         # launches, and no per-launch event overhead).  Otherwise: the bracketed figure.
         k_ms = ms if single_launch else kern_ms
-        ach = decode_bytes / (k_ms * 1e-3) / 1e9
+        kbytes = decode_bytes / (world if seq_split else 1)
+        ach = kbytes / (k_ms * 1e-3) / 1e9
         kname = {moa.PATH_GENERIC: "generic_decode_kernel",
                  moa.PATH_STREAM: "stream_decode_kernel (FMA; scores, online softmax, weighted sum, append, partial merge)",
-                 moa.PATH_GROUPED: "grouped64_decode_kernel / grouped_decode_kernel (tcgen05)",
+                 moa.PATH_GROUPED: "grouped64_decode_kernel (tcgen05; scores, online softmax, weighted sum)",
                  moa.PATH_MMA: "mma_decode_kernel (warp-level TF32 MMA; scores, online softmax, weighted sum, append, "
                                "partial merge)"}.get(moa.moa_last_path(), "?")
         roof = {"bound": "hbm", "kernel": kname, "achieved": ach, "peak": peak,
@@ -500,14 +724,15 @@ def main():
                 "kernel_us_per_launch_event_bracketed": (kern_ms * 1e3 if kern_ms else None),
                 "kernel_us_event_bracketed_min_median_max": (
                     [min(LAST_BRACKETED), statistics.median(LAST_BRACKETED), max(LAST_BRACKETED)] if LAST_BRACKETED else None),
-                "algorithmic_bytes_per_launch": decode_bytes,
-                "traffic": NCU_TRAFFIC_BYTES.get(wname)}
+                "algorithmic_bytes_per_launch": kbytes,
+                "traffic": ncu_traffic(wname)}
 
     # ---- end to end through the host-buffer entry point --------------------------------
     e2e = None
-    if wname != "multi_step" and run.host is not None and args.e2e_steps > 0:
+    dense = isinstance(run, DenseRun)
+    if dense and run.host is not None and args.e2e_steps > 0:
         run.e2e_step()                                   # warm-up: staging buffers are allocated here
-        torch.cuda.synchronize()
+        side.sync()
         barrier()
         t0 = time.perf_counter()
         for _ in range(args.e2e_steps):
@@ -537,7 +762,9 @@ def main():
     # ---- CPU oracle beside it (rank 0, N = 1 only) -------------------------------------
     cpu = None
     parity = None
-    if rank == 0 and world == 1 and not args.no_cpu and wname != "multi_step":
+    if rank == 0 and world == 1 and on_gpu and not args.no_cpu:
+        parity = sampled_parity(run, w)
+    if rank == 0 and world == 1 and dense and not args.no_cpu:
         import oracle
         h = run.host
         Kh, Vh = h["K"].numpy(), h["V"].numpy()
@@ -551,17 +778,26 @@ def main():
             t0 = time.perf_counter(); oracle.decode(qq, KK, VV, w.scale); dt = time.perf_counter() - t0
             spent += dt; passes += 1; best = min(best, dt)
         secs = spent / passes
-        got = run.out[0].cpu().numpy().reshape(w.batch * w.h_kv, w.group, w.d_v)[:units]
-        parity = float(np.max(np.abs(got.astype(np.float64) - ref.astype(np.float64))))
+        used = (run.i - 1) % run.nsets if run.i > 0 else 0
+        got = run.out[used].cpu().numpy().reshape(w.batch * w.h_kv, w.group, w.d_v)[:units]
+        parity = max(parity or 0.0, float(np.max(np.abs(got.astype(np.float64) - ref.astype(np.float64)))))
+        # the single-precision evaluation of the same definition, same sample, same cores
+        f32_passes, f32_spent = 0, 0.0
+        while f32_passes < 3 and f32_spent < 8.0:
+            t0 = time.perf_counter(); oracle.decode_f32(qq, KK, VV, w.scale); f32_spent += time.perf_counter() - t0
+            f32_passes += 1
+        f32_secs = f32_spent / f32_passes
         cpu = {"value": nbytes / secs / 1e9, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
                "sample": "%d of %d (batch, kv-head) groups of the same inputs; mean of %d passes, %.1f s of wall time in total" %
                          (units, w.batch * w.h_kv, passes, spent),
                "us_per_step_extrapolated": secs * 1e6 * (w.batch * w.h_kv) / units,
-               "best_pass_s": best}
+               "best_pass_s": best,
+               "single_precision_variant": {"value": nbytes / f32_secs / 1e9, "unit": UNIT, "passes": f32_passes,
+                                            "us_per_step_extrapolated": f32_secs * 1e6 * (w.batch * w.h_kv) / units}}
 
-    # ---- the other workloads, timing only (device-generated inputs) ---------------------
+    # ---- the other workloads (device-generated inputs): timing and one sampled parity each ----
     others = []
-    if rank == 0 and world == 1 and not args.no_others:
+    if rank == 0 and world == 1 and on_gpu and not args.no_others and make_run is None:
         del run
         torch.cuda.empty_cache()
         for name, ow in list(mi.WORKLOADS.items()) + list(EXTRA_WORKLOADS.items()):
@@ -571,16 +807,18 @@ def main():
                 if name == "multi_step":
                     r = MultiStepRun(ow)
                     k = min(200, ow.steps - 10)
-                    oms, _, _, _ = time_steps(r, k, 10)
-                    _, okern, _, _ = time_steps(r, k, 3, None, bracket=True)
+                    oms, _, _, _, _ = time_steps(r, k, 10, side)
+                    _, okern, _, _, _ = time_steps(r, k, 3, side, None, bracket=True)
                     ob = r.bytes_for_steps(0, k) / k
                     odec = ob
                 else:
                     r = DenseRun(ow, host_inputs=False)
-                    oms, _, _, _ = time_steps(r, 100, 10)
-                    _, okern, _, _ = time_steps(r, 100, 3, None, bracket=True)
+                    k = 600 if name == "mqa_long" else 100
+                    oms, _, _, _, osegs = time_steps(r, k, 10, side, segment=200)
+                    _, okern, _, _, _ = time_steps(r, 100, 3, side, None, bracket=True)
                     ob, odec = r.bytes_per_step, r.decode_bytes
                 others.append({"workload": name, "us_per_step": oms * 1e3, "GBps": ob / (oms * 1e-3) / 1e9,
+                               "frac_of_peak": ob / (oms * 1e-3) / 1e9 / peak,
                                "decode_kernel_us": okern * 1e3 if okern else None,
                                "decode_kernel_GBps": (odec / (okern * 1e-3) / 1e9) if okern else None,
                                "decode_kernel_frac_of_peak": (odec / (okern * 1e-3) / 1e9 / peak) if okern else None,
@@ -588,10 +826,13 @@ def main():
                                "decode_kernel_us_min_median_max": (
                                    [min(LAST_BRACKETED), statistics.median(LAST_BRACKETED), max(LAST_BRACKETED)]
                                    if LAST_BRACKETED else None),
+                               "parity_max_abs_err_vs_oracle": (None if args.no_cpu else sampled_parity(r, ow)),
                                "l2": r.l2_note})
+                if name != "multi_step" and osegs:
+                    others[-1]["us_per_step_first_last_200"] = [osegs[0] * 1e3, osegs[1] * 1e3]
                 if name == "single_head":              # latency-bound: also with its lines resident in L2
                     r.nsets = 1
-                    wms, _, _, _ = time_steps(r, 200, 10)
+                    wms, _, _, _, _ = time_steps(r, 200, 10, side)
                     others[-1]["us_per_step_l2_warm"] = wms * 1e3
                 del r
                 torch.cuda.empty_cache()
@@ -599,16 +840,24 @@ def main():
                 others.append({"workload": name, "error": repr(ex)[:200]})
 
     if rank == 0:
+        if seq_split:
+            step_desc = ("sequence split: moa_decode_attn_partial over %d local rows + all-gather of the partial triples "
+                         "+ moa_combine_partials" % run.n_local)
+            par = "sp%d (cached rows cut over the ranks, one all-gather per step)" % world
+        else:
+            step_desc = ("moa_decode_step: append + attend over ragged lengths + length advance, one launch" if wname == "multi_step"
+                         else "moa_append_decode: kv append at row n-1 + decode attention over n rows, %d launch(es) per step"
+                         % max(1, launches // max(1, args.steps)))
+            par = "dp%d (batch-sharded, no collective)" % world
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-                "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+                "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+                "scaling": "strong" if seq_split else "weak",
                 "vs_baseline": None, "dtype": "f32", "data": "synthetic",
                 "config": {"workload": wname, "batch_per_gpu": w.batch, "h_q": w.h_q, "h_kv": w.h_kv,
-                           "n": w.n, "d_k": w.d_k, "d_v": w.d_v, "parallelism": "dp%d (batch-sharded, no collective)" % world,
-                           "step": ("moa_decode_step: append + attend over ragged lengths + length advance, one launch" if wname == "multi_step"
-                                    else "moa_append_decode: kv append at row n-1 + decode attention over n rows (MOA_OPT_MIN_ROWS_HINT = n), %d launch(es) per step"
-                                    % max(1, launches // max(1, args.steps))),
-                           "l2": l2_note},
-                "us_per_step": ms * 1e3, "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
+                           "n": w.n, "d_k": w.d_k, "d_v": w.d_v, "parallelism": par, "step": step_desc, "l2": l2_note},
+                "us_per_step": ms * 1e3, "us_per_step_per_rank": per_rank_all,
+                "us_per_step_first_last_300": ([segs[0] * 1e3, segs[1] * 1e3] if segs else None),
+                "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
                 "roofline": roof, "cpu_baseline": cpu, "parity_max_abs_err_vs_oracle": parity,
                 "other_workloads": others}
         print(json.dumps(line), flush=True)
@@ -618,4 +867,4 @@ def main():
 
 
 if __name__ == "__main__":
-    main()
+    sys.exit(main())

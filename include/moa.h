@@ -19,6 +19,13 @@
  *  - Arguments are validated on the host before anything is launched; on a non-zero
  *    return nothing has been written.
  *  - Results are deterministic: no floating-point atomics, fixed merge order.
+ *  - Threads: every entry point may be called from any host thread; the library's host
+ *    state is guarded by one internal lock (calls are serialised on the host while they
+ *    enqueue their work; moa_decode_attn_host holds the lock until its copies are done).
+ *    Calls that can overlap on the GPU must not share a workspace: the entry points that
+ *    take no workspace argument share one library-owned buffer per device and therefore
+ *    must be ordered with respect to each other (one stream, or events between streams).
+ *    moa_set_option changes process-wide state and is meant for tests and tuning runs.
  */
 #ifndef MOA_H
 #define MOA_H
@@ -71,8 +78,10 @@ int moa_decode_attn(const float *q, const float *K, const float *V, float *out,
  * A length outside [1, n_max] sets MOA_STATUS_SEQLEN_RANGE and leaves that item's rows
  * of `out` untouched.
  * `workspace`: device memory, 256-byte aligned, at least moa_workspace_bytes(...) bytes,
- * owned by the caller, contents undefined on entry and exit; it must not be shared by
- * calls that can overlap on the GPU.  The call allocates nothing.
+ * owned by the caller, contents undefined on entry and exit (it holds the partial results
+ * of split sequences and the completion counters of the in-kernel merge, which tolerate
+ * arbitrary initial contents); it must not be shared by calls that can overlap on the
+ * GPU.  The call allocates nothing.
  */
 int moa_decode_attn_varlen(const float *q, const float *K, const float *V, float *out,
                            int batch, int h_q, int h_kv, const int32_t *seq_lens,
@@ -232,9 +241,11 @@ int moa_decode_attn_host(const float *q, const float *K, const float *V, float *
  * MOA_NOALLOC_SCRATCH_BYTES bytes that is part of the library image: every GPU that
  * loads the library holds that much memory until the process exits.  The call issues no
  * cudaMalloc, cudaFree or other allocating routine.
- *  - A problem whose scratch need exceeds MOA_NOALLOC_SCRATCH_BYTES (only possible when
- *    MOA_OPT_NUM_CTAS was raised far above the SM count) is rejected with
- *    MOA_ERR_CAPACITY before anything is launched.
+ *  - The array holds the partial slots of the largest plan the library compiles (two slots
+ *    of 16 heads x 132 floats per streaming CTA, one CTA per SM: 2.5 MB on a 148-SM part)
+ *    plus the completion counters.  A problem whose scratch need still exceeds
+ *    MOA_NOALLOC_SCRATCH_BYTES (a part with many more SMs, or MOA_OPT_NUM_CTAS raised far
+ *    above the SM count) is rejected with MOA_ERR_CAPACITY before anything is launched.
  *  - The first call on each device looks up the device address of the array (one
  *    cudaGetSymbolAddress with that device current) and keeps it; make that first call
  *    before starting any stream capture on that device.
@@ -244,7 +255,7 @@ int moa_decode_attn_host(const float *q, const float *K, const float *V, float *
  *    between them) would race on it; order them, or give one of them its own workspace
  *    through moa_decode_attn_varlen.
  */
-#define MOA_NOALLOC_SCRATCH_BYTES (2u << 20)
+#define MOA_NOALLOC_SCRATCH_BYTES (4u << 20)
 int moa_decode_attn_noalloc(const float *q, const float *K, const float *V, float *out,
                             int batch, int h_q, int h_kv, int n, int d_k, int d_v,
                             float scale, void *stream);
@@ -279,14 +290,6 @@ const char *moa_strerror(int code);
  *                        that keeps the query and probability operands in tensor memory
  *                        (64 head lanes, smaller groups padded); 1 = only the kernel with
  *                        these operands in shared memory (groups of exactly 16, 32, 64).
- *   MOA_OPT_MIN_ROWS_HINT : the caller's promise that every sequence of the calls that follow
- *                        has at least this many rows after the call (0 = no promise, the
- *                        default).  Lengths live on the device, so without the promise a
- *                        ragged batch of large head groups is served by two launches (one
- *                        for sequences of 4096 rows and more, one for shorter ones, which
- *                        need the more accurate kernel); with a promise of >= 4096 by one.
- *                        A broken promise costs accuracy on the short sequences (errors up
- *                        to about 1e-5), nothing else.
  * moa_last_path() reports which kernel family the last successful decode call used.
  */
 #define MOA_OPT_FORCE_PATH 1
@@ -294,7 +297,6 @@ const char *moa_strerror(int code);
 #define MOA_OPT_GROUPED_HEADS 3
 #define MOA_OPT_DEPENDENT_LAUNCH 4
 #define MOA_OPT_GROUPED_OPERANDS 5
-#define MOA_OPT_MIN_ROWS_HINT 6
 #define MOA_PATH_GENERIC   1   /* any d_k, d_v, alignment: one CTA per (batch, query head) */
 #define MOA_PATH_STREAM    2   /* split-sequence streaming kernel on the FMA units, d in {32,64,128} */
 #define MOA_PATH_GROUPED   3   /* tcgen05 tensor-core kernels for groups of 17..64 heads (16 when forced), d = 128, dense layout */

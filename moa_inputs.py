@@ -198,3 +198,50 @@ def small_like(w: Workload, **kw) -> Workload:
     """A reduced copy of a workload (same structure, smaller sizes) for quick parity."""
     from dataclasses import replace
     return replace(w, **kw)
+
+
+# ---------------------------------------------------------------------------------------
+# Low-entropy attention: inputs whose softmax mass sits on a few rows, so that no error
+# averages out over the cache.  Pure input shaping (no arithmetic of the method): the query
+# heads of a group share a common direction c, and a cached key is placed at a chosen score
+# level t by making it (t * sqrt(d) / |c|^2) * c plus a little noise.
+# ---------------------------------------------------------------------------------------
+TID_COMMON, TID_QNOISE, TID_KNOISE = 11, 12, 13
+
+
+def _group_common(seed, B, h_kv, d):
+    return normal(seed, TID_COMMON, (B, h_kv, d)).astype(np.float64)
+
+
+def peaked_case(seed, B, h_q, h_kv, n, d, peaks, floor=12.0, v_gap=3.0, q_spread=0.3, d_v=None):
+    """q, K, V (fp32) of a dense cache in which the rows listed in ``peaks`` = [(row, level), ...]
+    score about ``level`` (natural units, after the 1/sqrt(d) scale) for every query head and all
+    other rows about ``-floor`` + N(0, ~1).  The V rows of the peaks alternate between about
+    +v_gap and -v_gap.  Rows may be negative (counted from the end)."""
+    d_v = d if d_v is None else d_v
+    g_s = h_q // h_kv
+    c = _group_common(seed, B, h_kv, d)                                  # [B, h_kv, d]
+    c2 = np.sum(c * c, axis=-1, keepdims=True)
+    unit = c * (np.sqrt(float(d)) / c2)                                  # scores 1.0 against q = c
+    q = np.repeat(c, g_s, axis=1) + q_spread * normal(seed, TID_QNOISE, (B, h_q, d)).astype(np.float64)
+    K = normal(seed, TID_K, (B, h_kv, n, d)).astype(np.float64) - floor * unit[:, :, None, :]
+    V = normal(seed, TID_V, (B, h_kv, n, d_v)).astype(np.float64)
+    kn = normal(seed, TID_KNOISE, (B, h_kv, len(peaks), d)).astype(np.float64)
+    for i, (row, level) in enumerate(peaks):
+        K[:, :, row, :] = level * unit + 0.1 * kn[:, :, i, :]
+        V[:, :, row, :] += v_gap if i % 2 == 0 else -v_gap
+    return q.astype(np.float32), K.astype(np.float32), V.astype(np.float32)
+
+
+def sorted_case(seed, B, h_q, h_kv, n, d, lo=-10.0, hi=10.0, descending=False, q_spread=0.3):
+    """q, K, V (fp32) whose scores run monotonically from ``lo`` to ``hi`` along the cache
+    (or the other way round): every tile raises -- or never raises -- the running maximum."""
+    g_s = h_q // h_kv
+    c = _group_common(seed, B, h_kv, d)
+    c2 = np.sum(c * c, axis=-1, keepdims=True)
+    unit = c * (np.sqrt(float(d)) / c2)
+    q = np.repeat(c, g_s, axis=1) + q_spread * normal(seed, TID_QNOISE, (B, h_q, d)).astype(np.float64)
+    levels = np.linspace(hi, lo, n) if descending else np.linspace(lo, hi, n)
+    K = levels[None, None, :, None] * unit[:, :, None, :] + 0.05 * normal(seed, TID_K, (B, h_kv, n, d)).astype(np.float64)
+    V = normal(seed, TID_V, (B, h_kv, n, d)).astype(np.float64)
+    return q.astype(np.float32), K.astype(np.float32), V.astype(np.float32)

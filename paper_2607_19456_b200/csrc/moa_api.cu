@@ -3,6 +3,8 @@
 #include <cuda_runtime.h>
 #include <math.h>
 #include <stdint.h>
+#include <atomic>
+#include <mutex>
 #include <type_traits>
 #include <utility>
 
@@ -26,10 +28,15 @@ struct DeviceState {
     void *stage[4] = {nullptr, nullptr, nullptr, nullptr};   // host-API staging: q K V out
     size_t stage_bytes[4] = {0, 0, 0, 0};
     cudaStream_t host_stream = nullptr;
-    unsigned *tickets = nullptr;  // device address of g_tickets (resolved once)
-    unsigned ticket_seq = 0;      // launches so far: picks the counter slot round-robin
 };
 static DeviceState g_dev[kMaxDevices];
+// Host state of the library (the table above, the options, the launch accounting) is guarded
+// by one lock, taken by every entry point that reads or changes it; launches are issued
+// under it, so calls from several host threads are serialised on the host side only.
+static std::recursive_mutex g_mu;
+typedef std::lock_guard<std::recursive_mutex> Lock;
+// Tag of the next launch that merges its partials in the kernel (see ticket_arrive).
+static std::atomic<unsigned long long> g_launch_tag{1};
 static int g_force_path = 0;
 static int g_num_ctas = 0;
 static int g_last_path = 0;
@@ -241,9 +248,15 @@ static int stream_grid(const DeviceState &s, const StreamPlan &p, int batch, int
     return (int)(want < cap ? (want < 1 ? 1 : want) : cap);
 }
 
+// Workspace of a streaming launch: two partial slots per CTA, then (256-byte aligned) the
+// completion counters of the in-kernel merge.
+static size_t stream_slot_bytes(const StreamPlan &p, int num_ctas)
+{
+    return ((size_t)num_ctas * 2 * p.G * (p.D + 4) * sizeof(float) + 255) / 256 * 256;
+}
 static size_t stream_ws_bytes(const StreamPlan &p, int num_ctas)
 {
-    return (size_t)num_ctas * 2 * p.G * (p.D + 4) * sizeof(float);
+    return stream_slot_bytes(p, num_ctas) + (num_ctas <= kTicketCtas ? kTicketBytes : 0);
 }
 
 template <class C>
@@ -360,7 +373,6 @@ struct GroupedPlan {
 };
 static int g_grouped_heads = 0;   // MOA_OPT_GROUPED_HEADS: 0 = automatic
 static int g_grouped_operands = 0;   // MOA_OPT_GROUPED_OPERANDS
-static int g_min_rows_hint = 0;      // MOA_OPT_MIN_ROWS_HINT
 
 static GroupedPlan plan_grouped(const DeviceState &s, int batch, int h_q, int h_kv, int n, int d_k, int d_v)
 {
@@ -514,36 +526,13 @@ template <int GH>
 static cudaError_t launch_grouped_cfg(const CUtensorMap &mk, const CUtensorMap &mv, const CUtensorMap &mkt,
                                       const CUtensorMap &mvt, const GroupedArgs &ga, int grid, cudaStream_t st);
 
-// Groups of 17 to 64 heads on 64 head lanes.  Same arguments and partial format as the
-// shared-memory-operand kernel, so the combine kernel is shared.
-//  - Long dense caches: the kernel with Q and P in tensor memory whose scores are one
-//    accumulation chain of 32 steps (the error of an output averages out over the rows).
-//  - Short caches and ragged ones (lengths unknown here): exact groups of 32 or 64 heads run
-//    on the shared-memory-operand kernel (16-step chains, and faster than the next one);
-//    padded groups on the tensor-memory kernel that keeps the two score chains apart.
+// Groups of 17 to 64 heads on 64 head lanes (missing heads are zero lanes): the kernel with Q
+// and P in tensor memory, in the variant that keeps the two score chains apart.  Same arguments
+// and partial format as the shared-memory-operand kernel, so the combine kernel is shared.
 static cudaError_t launch_grouped64(const CUtensorMap &mk, const CUtensorMap &mv, const CUtensorMap &mkt,
-                                    const CUtensorMap &mvt, const GroupedArgs &ga, int grid, cudaStream_t st,
-                                    bool fused)
+                                    const CUtensorMap &mvt, const GroupedArgs &ga, int grid, cudaStream_t st)
 {
-    if (ga.seq_lens == nullptr && !fused && ga.n >= 4096) return launch_grouped64_cfg<false>(mk, mv, mkt, mvt, ga, grid, st);
-    // ragged, but the caller promises that no sequence is short: one launch of the single-chain kernel
-    if (g_min_rows_hint >= 4096 && ga.n >= 4096) return launch_grouped64_cfg<false>(mk, mv, mkt, mvt, ga, grid, st);
-    GroupedArgs rest = ga;
-    const bool two_launches = ga.seq_lens != nullptr && ga.n >= 4096;
-    if (two_launches) {
-        // A ragged batch in a long cache: the sequences of 4096 rows and more go to the
-        // single-chain kernel first (the CTAs of the other units leave at once), the shorter
-        // ones to the launch below; slots and splits are the same for both launches, so the
-        // second one has to use 64 head lanes as well.
-        GroupedArgs longs = ga;
-        longs.len_lo = 4096;
-        cudaError_t e = launch_grouped64_cfg<false>(mk, mv, mkt, mvt, longs, grid, st, false);
-        if (e != cudaSuccess) return e;
-        rest.len_hi = 4096;
-    }
-    if (ga.g_s == 64) return launch_grouped_cfg<64>(mk, mv, mkt, mvt, rest, grid, st);
-    if (ga.g_s == 32 && !two_launches) return launch_grouped_cfg<32>(mk, mv, mkt, mvt, rest, grid, st);
-    return launch_grouped64_cfg<true>(mk, mv, mkt, mvt, rest, grid, st);
+    return launch_grouped64_cfg<true>(mk, mv, mkt, mvt, ga, grid, st);
 }
 
 static cudaError_t launch_generic(const DecodeArgs &a, cudaStream_t st)
@@ -631,7 +620,7 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
     a.v_sb = lay.v.sb; a.v_sh = lay.v.sh; a.v_sr = lay.v.sr;
     a.qscale = scale * kLog2e;
     a.Kw = nullptr; a.Vw = nullptr; a.k_new = nullptr; a.v_new = nullptr; a.lens_rw = nullptr;
-    a.tickets = nullptr;
+    a.tickets = nullptr; a.ticket_tag = 0;
     a.partial_out = partial_out;
     if (fused != nullptr && path == MOA_PATH_GENERIC) return MOA_ERR_UNSUPPORTED;
 
@@ -684,7 +673,7 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
         }
         if (gplan.GH == 16) e = launch_grouped_cfg<16>(mk, mv, mkt, mvt, ga, grid, st);
         else if (gplan.GH == 32) e = launch_grouped_cfg<32>(mk, mv, mkt, mvt, ga, grid, st);
-        else if (gplan.share == 1 && g_grouped_operands == 0) e = launch_grouped64(mk, mv, mkt, mvt, ga, grid, st, fused != nullptr);
+        else if (gplan.share == 1 && g_grouped_operands == 0) e = launch_grouped64(mk, mv, mkt, mvt, ga, grid, st);
         else e = launch_grouped_cfg<64>(mk, mv, mkt, mvt, ga, grid, st);
         if (e == cudaSuccess && fused != nullptr && fused->lens_rw != nullptr) {
             lens_add_kernel<<<(batch + 127) / 128, 128, 0, st>>>(fused->lens_rw, batch, 1, n_max);
@@ -707,12 +696,10 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
         }
         a.ws = static_cast<float *>(ws);
         if (num_ctas <= kTicketCtas) {      // merge partials inside the streaming launch
-            if (dev->tickets == nullptr) {
-                void *p = nullptr;
-                if (cudaGetSymbolAddress(&p, g_tickets) != cudaSuccess || !p) { cudaGetLastError(); return MOA_ERR_CUDA; }
-                dev->tickets = static_cast<unsigned *>(p);
-            }
-            a.tickets = dev->tickets + (size_t)(dev->ticket_seq++ % kTicketSlots) * kTicketStride;
+            a.tickets = reinterpret_cast<unsigned long long *>(static_cast<unsigned char *>(ws) + stream_slot_bytes(plan, num_ctas));
+            unsigned long long tag = g_launch_tag.fetch_add(1) & ((1ull << 44) - 1ull);
+            if (tag == 0) tag = g_launch_tag.fetch_add(1) & ((1ull << 44) - 1ull);
+            a.ticket_tag = (tag << 20) | 1ull;
         }
         if (fused != nullptr) {
             if (a.tickets == nullptr && fused->lens_rw != nullptr) return MOA_ERR_UNSUPPORTED;
@@ -746,6 +733,7 @@ extern "C" {
 int moa_decode_attn(const float *q, const float *K, const float *V, float *out, int batch,
                     int h_q, int h_kv, int n, int d_k, int d_v, float scale, void *stream)
 {
+    Lock lock(g_mu);
     return decode_impl(q, K, V, out, batch, h_q, h_kv, nullptr, 0, n, d_k, d_v, scale, nullptr, 0,
                        true, static_cast<cudaStream_t>(stream));
 }
@@ -753,6 +741,7 @@ int moa_decode_attn(const float *q, const float *K, const float *V, float *out, 
 int moa_decode_attn_noalloc(const float *q, const float *K, const float *V, float *out, int batch,
                             int h_q, int h_kv, int n, int d_k, int d_v, float scale, void *stream)
 {
+    Lock lock(g_mu);
     // Argument errors first, exactly as the allocating entry point reports them.
     if (!q || !K || !V || !out) return MOA_ERR_INVALID;
     int rc = validate_dims(batch, h_q, h_kv, n, d_k, d_v);
@@ -772,18 +761,19 @@ int moa_decode_attn_noalloc(const float *q, const float *K, const float *V, floa
         }
         g_noalloc_scratch_dev[device] = p;
     }
-    // Refuse problems whose partial-result slots would not fit the fixed array.
+    // Refuse problems whose partial-result slots and counters would not fit the fixed array
+    // (the same plan and grid the launch below will use).
     const StreamPlan plan = plan_stream(h_q / h_kv, d_k, d_v);
-    if (plan.ok && stream_ws_bytes(plan, stream_num_ctas(*dev)) > (size_t)MOA_NOALLOC_SCRATCH_BYTES)
+    if (plan.ok && stream_ws_bytes(plan, stream_grid(*dev, plan, batch, h_kv, n)) > (size_t)MOA_NOALLOC_SCRATCH_BYTES)
         return MOA_ERR_CAPACITY;
-    // The launch-accounting hooks create their CUDA events lazily; keep that (an
-    // allocation of driver objects) out of this call if it has not happened yet.
-    const bool prof_saved = g_prof_on;
-    if (g_prof_ev == nullptr) g_prof_on = false;
+    // No CUDA events are created for this call (the launch accounting creates them lazily,
+    // which allocates driver objects); its launches are still counted.
+    const bool events_saved = g_prof_events;
+    if (g_prof_ev == nullptr) g_prof_events = false;
     rc = decode_impl(q, K, V, out, batch, h_q, h_kv, nullptr, 0, n, d_k, d_v, scale,
                      g_noalloc_scratch_dev[device], (size_t)MOA_NOALLOC_SCRATCH_BYTES, false,
                      static_cast<cudaStream_t>(stream), nullptr, false);
-    g_prof_on = prof_saved;
+    g_prof_events = events_saved;
     return rc;
 }
 
@@ -791,6 +781,7 @@ int moa_decode_attn_layers(const float *const *q, const float *const *K, const f
                            int layers, int batch, int h_q, int h_kv, int n, int d_k, int d_v, float scale,
                            void *stream)
 {
+    Lock lock(g_mu);
     if (!q || !K || !V || !out || layers < 1) return MOA_ERR_INVALID;
     for (int l = 0; l < layers; ++l) {
         const int rc = decode_impl(q[l], K[l], V[l], out[l], batch, h_q, h_kv, nullptr, 0, n, d_k, d_v, scale,
@@ -803,6 +794,7 @@ int moa_decode_attn_layers(const float *const *q, const float *const *K, const f
 int moa_decode_attn_partial(const float *q, const float *K, const float *V, float *partial, int batch,
                             int h_q, int h_kv, int n, int d_k, int d_v, float scale, void *stream)
 {
+    Lock lock(g_mu);
     return decode_impl(q, K, V, nullptr, batch, h_q, h_kv, nullptr, 0, n, d_k, d_v, scale, nullptr, 0,
                        true, static_cast<cudaStream_t>(stream), nullptr, true, partial);
 }
@@ -810,6 +802,7 @@ int moa_decode_attn_partial(const float *q, const float *K, const float *V, floa
 int moa_combine_partials(const float *partials, int nparts, float *out, int batch, int h_q, int d_v,
                          void *stream)
 {
+    Lock lock(g_mu);
     if (!partials || !out || nparts < 1 || batch < 1 || h_q < 1 || d_v < 1) return MOA_ERR_INVALID;
     if (d_v > MOA_MAX_DV) return MOA_ERR_UNSUPPORTED;
     if (!aligned(partials, 4) || !aligned(out, 4)) return MOA_ERR_ALIGN;
@@ -828,12 +821,14 @@ int moa_decode_attn_varlen(const float *q, const float *K, const float *V, float
                            int d_v, float scale, void *workspace, size_t workspace_bytes,
                            void *stream)
 {
+    Lock lock(g_mu);
     return decode_impl(q, K, V, out, batch, h_q, h_kv, seq_lens, 0, n_max, d_k, d_v, scale,
                        workspace, workspace_bytes, false, static_cast<cudaStream_t>(stream));
 }
 
 size_t moa_workspace_bytes(int batch, int h_q, int h_kv, int n_max, int d_k, int d_v)
 {
+    Lock lock(g_mu);
     if (validate_dims(batch, h_q, h_kv, n_max, d_k, d_v) != MOA_OK) return 0;
     StreamPlan plan = plan_stream(h_q / h_kv, d_k, d_v);
     if (!plan.ok) return 256;              // generic path: no scratch; keep the result non-zero
@@ -874,6 +869,7 @@ static int kv_append_impl(float *K, float *V, const float *k_new, const float *v
 int moa_kv_append(float *K, float *V, const float *k_new, const float *v_new, const int32_t *pos,
                   int batch, int h_kv, int n_max, int d_k, int d_v, void *stream)
 {
+    Lock lock(g_mu);
     if (batch < 1 || h_kv < 1 || n_max < 1 || d_k < 1 || d_v < 1) return MOA_ERR_INVALID;
     return kv_append_impl(K, V, k_new, v_new, pos, batch, h_kv, n_max, d_k, d_v,
                           dense_layout(h_kv, n_max, d_k, d_v), stream);
@@ -889,6 +885,7 @@ int moa_kv_append_strided(float *K, float *V, const float *k_new, const float *v
                           int batch, int h_kv, int n_max, int d_k, int d_v, const long long *k_strides,
                           const long long *v_strides, void *stream)
 {
+    Lock lock(g_mu);
     if (batch < 1 || h_kv < 1 || n_max < 1 || d_k < 1 || d_v < 1) return MOA_ERR_INVALID;
     Layout lay;
     if (!strided_layout(k_strides, v_strides, h_kv, n_max, d_k, d_v, &lay) || !writable_layout(lay, batch, h_kv))
@@ -898,6 +895,7 @@ int moa_kv_append_strided(float *K, float *V, const float *k_new, const float *v
 
 int moa_lens_add(int32_t *lens, int batch, int delta, void *stream)
 {
+    Lock lock(g_mu);
     if (!lens || batch < 1) return MOA_ERR_INVALID;
     if (!aligned(lens, 4)) return MOA_ERR_ALIGN;
     DeviceState *dev = nullptr;
@@ -963,6 +961,7 @@ int moa_decode_step(const float *q, float *K, float *V, const float *k_new, cons
                     float *out, int32_t *lens, int batch, int h_q, int h_kv, int n_max, int d_k,
                     int d_v, float scale, void *workspace, size_t workspace_bytes, void *stream)
 {
+    Lock lock(g_mu);
     return step_impl(q, K, V, k_new, v_new, out, lens, lens, batch, h_q, h_kv, n_max, d_k, d_v, scale,
                      workspace, workspace_bytes, stream, true);
 }
@@ -971,6 +970,7 @@ int moa_append_decode(const float *q, float *K, float *V, const float *k_new, co
                       float *out, const int32_t *pos, int batch, int h_q, int h_kv, int n_max, int d_k,
                       int d_v, float scale, void *workspace, size_t workspace_bytes, void *stream)
 {
+    Lock lock(g_mu);
     return step_impl(q, K, V, k_new, v_new, out, nullptr, pos, batch, h_q, h_kv, n_max, d_k, d_v, scale,
                      workspace, workspace_bytes, stream, false);
 }
@@ -980,6 +980,7 @@ int moa_decode_attn_strided(const float *q, const float *K, const float *V, floa
                             const long long *k_strides, const long long *v_strides, void *workspace,
                             size_t workspace_bytes, void *stream)
 {
+    Lock lock(g_mu);
     if (validate_dims(batch, h_q, h_kv, n_max, d_k, d_v) == MOA_ERR_INVALID) return MOA_ERR_INVALID;
     Layout lay;
     if (!strided_layout(k_strides, v_strides, h_kv, n_max, d_k, d_v, &lay)) return MOA_ERR_INVALID;
@@ -993,6 +994,7 @@ int moa_decode_step_strided(const float *q, float *K, float *V, const float *k_n
                             const long long *k_strides, const long long *v_strides, void *workspace,
                             size_t workspace_bytes, void *stream)
 {
+    Lock lock(g_mu);
     if (validate_dims(batch, h_q, h_kv, n_max, d_k, d_v) == MOA_ERR_INVALID) return MOA_ERR_INVALID;
     Layout lay;
     if (!strided_layout(k_strides, v_strides, h_kv, n_max, d_k, d_v, &lay) || !writable_layout(lay, batch, h_kv))
@@ -1004,6 +1006,7 @@ int moa_decode_step_strided(const float *q, float *K, float *V, const float *k_n
 int moa_decode_attn_host(const float *q, const float *K, const float *V, float *out, int batch,
                          int h_q, int h_kv, int n, int d_k, int d_v, float scale)
 {
+    Lock lock(g_mu);
     if (!q || !K || !V || !out) return MOA_ERR_INVALID;
     int rc = validate_dims(batch, h_q, h_kv, n, d_k, d_v);
     if (rc != MOA_OK) return rc;
@@ -1048,6 +1051,7 @@ int moa_decode_attn_host(const float *q, const float *K, const float *V, float *
 
 int moa_device_status(void *stream, int *status_out)
 {
+    Lock lock(g_mu);
     if (!status_out) return MOA_ERR_INVALID;
     DeviceState *dev = nullptr;
     int rc = current_device(&dev);
@@ -1073,6 +1077,7 @@ long long moa_min_bytes(int batch, int h_q, int h_kv, long long n, int d_k, int 
 
 int moa_release(void)
 {
+    Lock lock(g_mu);
     DeviceState *dev = nullptr;
     int rc = current_device(&dev);
     if (rc != MOA_OK) return rc;
@@ -1103,6 +1108,7 @@ const char *moa_strerror(int code)
 
 int moa_set_option(int option, int value)
 {
+    Lock lock(g_mu);
     if (option == MOA_OPT_FORCE_PATH) {
         if (value < 0 || value > MOA_PATH_MMA) return MOA_ERR_INVALID;
         g_force_path = value;
@@ -1118,11 +1124,6 @@ int moa_set_option(int option, int value)
         g_grouped_operands = value;
         return MOA_OK;
     }
-    if (option == MOA_OPT_MIN_ROWS_HINT) {
-        if (value < 0) return MOA_ERR_INVALID;
-        g_min_rows_hint = value;
-        return MOA_OK;
-    }
     if (option == MOA_OPT_DEPENDENT_LAUNCH) {
         if (value != 0 && value != 1) return MOA_ERR_INVALID;
         g_dependent_launch = value;
@@ -1136,10 +1137,11 @@ int moa_set_option(int option, int value)
     return MOA_ERR_INVALID;
 }
 
-int moa_last_path(void) { return g_last_path; }
+int moa_last_path(void) { Lock lock(g_mu); return g_last_path; }
 
 int moa_profile(int enable)
 {
+    Lock lock(g_mu);
     g_prof_on = enable != 0;
     g_prof_events = enable == 2;
     if (g_prof_on) { g_prof_all = 0; g_prof_timed = 0; }
@@ -1149,6 +1151,7 @@ int moa_profile(int enable)
 int moa_profile_read(double *decode_kernel_ms, long long *decode_kernel_launches,
                      long long *all_kernel_launches)
 {
+    Lock lock(g_mu);
     if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return MOA_ERR_CUDA; }
     double ms = 0.0;
     long long timed = 0;
@@ -1170,6 +1173,7 @@ int moa_profile_read(double *decode_kernel_ms, long long *decode_kernel_launches
 
 int moa_profile_launch_ms(long long index, double *ms)
 {
+    Lock lock(g_mu);
     if (!ms || index < 0 || index >= g_prof_timed) return MOA_ERR_INVALID;
     if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return MOA_ERR_CUDA; }
     float t = 0.f;

@@ -138,8 +138,9 @@ struct DecodeArgs {
     const float *k_new;       // [batch, stored kv heads, d_k] row appended at index seq_lens[b]
     const float *v_new;       // [batch, stored kv heads, d_v]
     int32_t *lens_rw;         // lengths advanced by one when the whole grid is done, or nullptr
-    unsigned *tickets;        // completion counters (kTicketStride words, all zero between
-                              // launches), or nullptr: partials are merged by a second kernel
+    unsigned long long *tickets;   // completion counters (kTicketStride words at the end of the
+                                   // workspace), or nullptr: partials are merged by a second kernel
+    unsigned long long ticket_tag; // what one arrival adds to a counter word: (launch tag << 20) + 1
     float *partial_out;       // nullptr, or [batch, h_q, d_v + 4]: emit the unnormalised triple
                               // (o[d_v], m, l, 2 pad) instead of the normalised output row
 };
@@ -163,11 +164,37 @@ __device__ __forceinline__ void emit_columns(const DecodeArgs &a, size_t bh, int
 
 // Completion counters of one launch: word c counts the CTAs that have delivered their
 // partial for the split unit whose first segment lies in CTA c; the last word counts CTAs
-// that have finished altogether.  Whoever brings a counter to its final value resets it.
+// that have finished altogether.  The counters live at the end of the workspace the call
+// was given, so calls with workspaces of their own never share one.  A workspace's contents
+// are undefined on entry, so a counter proves that it belongs to the launch: every arrival
+// adds `inc` = (tag << 20) + 1, where tag is a process-wide launch number (44 bits, never
+// zero); a word is a live counter of this launch after j arrivals exactly when it equals
+// j * inc.  Zero is the state before the first arrival; anything else is a leftover and is
+// replaced.  Whoever brings a counter to its final value resets the word to zero, which keeps
+// a captured launch (whose tag is frozen) replayable.  The ordinary path is one atomicAdd per
+// arrival; the compare-and-swap only runs on a leftover, i.e. once per word of a workspace
+// that was handed over uninitialised.
 constexpr int kTicketCtas = 1024;
 constexpr int kTicketStride = kTicketCtas + 1;
-constexpr int kTicketSlots = 32;
-__device__ unsigned g_tickets[kTicketSlots * kTicketStride];
+constexpr size_t kTicketBytes = (size_t)kTicketStride * sizeof(unsigned long long);
+constexpr unsigned long long kTicketCountMask = (1ull << 20) - 1ull;
+
+// Count one arrival on `word`; returns the number of arrivals of this launch before this one.
+__device__ __forceinline__ unsigned ticket_arrive(unsigned long long *word, unsigned long long inc)
+{
+    unsigned long long old = atomicAdd(word, inc);
+    for (;;) {
+        const unsigned long long j = old & kTicketCountMask;
+        if (old == j * inc) return (unsigned)j;
+        // A leftover (to which the increment above was added in vain): claim the word as the
+        // first arrival, or count again if another CTA has claimed it meanwhile.
+        const unsigned long long seen = *reinterpret_cast<volatile unsigned long long *>(word);
+        const unsigned long long js = seen & kTicketCountMask;
+        if (seen == js * inc) { old = atomicAdd(word, inc); continue; }
+        if (atomicCAS(word, seen, inc) == seen) return 0u;
+        old = ~0ull;                            // lost the race: look again
+    }
+}
 
 // Length of sequence b as the kernels see it; 0 for an out-of-range length (the item is
 // then skipped by construction: it owns no row blocks).

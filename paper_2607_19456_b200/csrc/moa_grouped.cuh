@@ -207,6 +207,12 @@ __device__ __forceinline__ float from_ordered_bits(uint32_t u)
     return __uint_as_float((u & 0x80000000u) ? (u & 0x7FFFFFFFu) : ~u);
 }
 __device__ __forceinline__ float tf32_hi(float x) { return __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
+// Nearest TF32 value (10 mantissa bits kept, the rest rounded away).  Operands this library
+// writes itself are split as hi = tf32_rn(x), lo = tf32_rn(x - hi): nothing is left for the
+// tensor core to cut off, and the rounding errors (at most 2^-23 of x) have no preferred sign.
+// A streamed operand is multiplied as loaded, i.e. with hi = tf32_hi(x) (what the tensor core
+// keeps of an fp32 word), and its remainder x - tf32_hi(x) is left to the tensor core's cut.
+__device__ __forceinline__ float tf32_rn(float x) { return __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xFFFFE000u); }
 
 __device__ __forceinline__ void named_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
 __device__ __forceinline__ bool named_or(int id, int n, bool pred)
@@ -339,10 +345,10 @@ grouped_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_co
         for (int i = tid; i < GH * 128; i += C::THREADS) {
             const int g = i >> 7, k = i & 127;
             const float x = qb[i] * a.qscale;
-            const float hi = tf32_hi(x);
+            const float hi = tf32_rn(x);
             const uint32_t chunk = (uint32_t)(k >> 5) * C::OPCH, col = (uint32_t)(k & 31) * 4;
             *reinterpret_cast<float *>(smem + C::OFF_Q + chunk + tc::swz128(g, col)) = hi;
-            *reinterpret_cast<float *>(smem + C::OFF_Q + chunk + tc::swz128(GH + g, col)) = x - hi;
+            *reinterpret_cast<float *>(smem + C::OFF_Q + chunk + tc::swz128(GH + g, col)) = tf32_rn(x - hi);
         }
         if (tid < GH) mref[tid] = -INFINITY;
     }
@@ -628,9 +634,9 @@ grouped_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_co
             // probabilities, split into hi|lo, as the K-major B operand of this row quarter
 #pragma unroll
             for (int g = 0; g < HH; ++g) {
-                const float ph = tf32_hi(p[g]);
+                const float ph = tf32_rn(p[g]);
                 *reinterpret_cast<float *>(pch + tc::swz128(h0 + g, lane * 4)) = ph;
-                *reinterpret_cast<float *>(pch + tc::swz128(GH + h0 + g, lane * 4)) = p[g] - ph;
+                *reinterpret_cast<float *>(pch + tc::swz128(GH + h0 + g, lane * 4)) = tf32_rn(p[g] - ph);
             }
             tc::fence_before_sync();
             tc::fence_async_smem();

@@ -213,8 +213,8 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
             const float xs[4] = {x4.x * a.qscale, x4.y * a.qscale, x4.z * a.qscale, x4.w * a.qscale};
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                const float hi = tf32_hi(xs[k]);
-                v[i + k] = __float_as_uint(is_lo ? xs[k] - hi : hi);
+                const float hi = tf32_rn(xs[k]);
+                v[i + k] = __float_as_uint(is_lo ? tf32_rn(xs[k] - hi) : hi);
             }
         }
         tc::tmem_st32(tQ + lane_addr + col0, v);

@@ -90,7 +90,9 @@ __device__ __forceinline__ void mma_tf32_16x8x8(float (&c)[4], uint32_t a0, uint
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// x = hi + lo with hi exactly representable in TF32 (10 mantissa bits kept).
+// x = hi + lo (+ at most 2^-23 of x): hi the nearest TF32 value (10 mantissa bits kept), lo the
+// remainder rounded to TF32 as well, so that the tensor core, which ignores the low 13 bits of
+// an operand, has nothing left to cut off and the rounding errors have no preferred sign.
 struct Split4 {
     uint32_t h[4], l[4];
 };
@@ -100,9 +102,9 @@ __device__ __forceinline__ Split4 split4(const float4 &v)
     const float x[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        const uint32_t hb = __float_as_uint(x[i]) & 0xFFFFE000u;
+        const uint32_t hb = (__float_as_uint(x[i]) + 0x1000u) & 0xFFFFE000u;
         s.h[i] = hb;
-        s.l[i] = __float_as_uint(x[i] - __uint_as_float(hb));
+        s.l[i] = (__float_as_uint(x[i] - __uint_as_float(hb)) + 0x1000u) & 0xFFFFE000u;
     }
     return s;
 }
@@ -290,9 +292,9 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
             const long long c_first = cc.first / bpc, c_last = (unit_end - 1) / bpc;
             if (tid == 0) {
                 __threadfence();               // this CTA's partial is visible before it is counted
-                const unsigned arrived = atomicAdd(&a.tickets[c_first], 1u);
+                const unsigned arrived = ticket_arrive(&a.tickets[c_first], a.ticket_tag);
                 const int last = (arrived == (unsigned)(c_last - c_first));
-                if (last) a.tickets[c_first] = 0u;
+                if (last) a.tickets[c_first] = 0ull;
                 s_last = last;
             }
             __syncthreads();
@@ -391,17 +393,21 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
     };
     auto score_tile = [&](ScoreState<NJ, NT> &st, const float *sK, int nr, int k, auto full_tag) -> bool {
         constexpr bool FULL = decltype(full_tag)::value;
-        // 2*NJ k-steps; six independent accumulator chains in flight (three products x two chains
-        // for one head tile, three products x two head tiles otherwise); a K fragment is loaded
-        // and split once and used for all head tiles
-        constexpr int NCH = (NT == 1) ? 2 : 1;
-        float sh[NT][NCH][4], sl[NT][NCH][4], sm[NT][NCH][4];
+        // 2*NJ k-steps.  The warp-level MMA accumulates with truncation, and what a truncation
+        // costs is set by the size of the accumulator, so the large hi*hi products of a score are
+        // spread over NCH short chains (four k-steps each at d = 128 with one head tile) that are
+        // added in fp32 afterwards; the two small cross terms share one chain each.  A K fragment
+        // is loaded and split once and used for all head tiles.
+        constexpr int NCH = (NT == 1) ? 4 : 2;
+        float sh[NT][NCH][4], sl[NT][4], sm[NT][4];
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-            for (int c = 0; c < NCH; ++c)
+            for (int i = 0; i < 4; ++i) {
+                sl[nt][i] = 0.f; sm[nt][i] = 0.f;
 #pragma unroll
-                for (int i = 0; i < 4; ++i) { sh[nt][c][i] = 0.f; sl[nt][c][i] = 0.f; sm[nt][c][i] = 0.f; }
+                for (int c = 0; c < NCH; ++c) sh[nt][c][i] = 0.f;
+            }
 #pragma unroll
         for (int j = 0; j < NJ; ++j) {
             const Split4 ka = split4(*reinterpret_cast<const float4 *>(sK + chunk_at(rowA, t + 4 * j)));
@@ -412,7 +418,7 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
                 const uint32_t al[4] = {ka.l[2 * e], kb.l[2 * e], ka.l[2 * e + 1], kb.l[2 * e + 1]};
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt)
-                    mma3(sh[nt][e % NCH], sl[nt][e % NCH], sm[nt][e % NCH], ah, al, st.qh[nt][j][2 * e],
+                    mma3(sh[nt][(2 * j + e) % NCH], sl[nt], sm[nt], ah, al, st.qh[nt][j][2 * e],
                          st.qh[nt][j][2 * e + 1], st.ql[nt][j][2 * e], st.ql[nt][j][2 * e + 1]);
             }
         }
@@ -423,10 +429,10 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
             float s[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                if constexpr (NCH == 2)
-                    s[i] = (sh[nt][0][i] + sh[nt][1][i]) + ((sl[nt][0][i] + sl[nt][1][i]) + (sm[nt][0][i] + sm[nt][1][i]));
+                if constexpr (NCH == 4)
+                    s[i] = ((sh[nt][0][i] + sh[nt][1][i]) + (sh[nt][2][i] + sh[nt][3][i])) + (sl[nt][i] + sm[nt][i]);
                 else
-                    s[i] = sh[nt][0][i] + (sl[nt][0][i] + sm[nt][0][i]);
+                    s[i] = (sh[nt][0][i] + sh[nt][1][i]) + (sl[nt][i] + sm[nt][i]);
             }
             if (!FULL) {
                 if (rowA >= nr) { s[0] = -INFINITY; s[1] = -INFINITY; }
@@ -570,9 +576,9 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
         __syncthreads();
         if (tid == 0) {
             __threadfence();
-            const unsigned done = atomicAdd(&a.tickets[kTicketCtas], 1u);
+            const unsigned done = ticket_arrive(&a.tickets[kTicketCtas], a.ticket_tag);
             const int last = (done == gridDim.x - 1);
-            if (last) a.tickets[kTicketCtas] = 0u;
+            if (last) a.tickets[kTicketCtas] = 0ull;
             s_last = last;
         }
         __syncthreads();

@@ -240,9 +240,9 @@ __global__ void __launch_bounds__(C::THREADS, 1) stream_decode_kernel(const Deco
             const long long c_first = cc.first / bpc, c_last = (unit_end - 1) / bpc;
             if (tid == 0) {
                 __threadfence();               // this CTA's partial is visible before it is counted
-                const unsigned arrived = atomicAdd(&a.tickets[c_first], 1u);
+                const unsigned arrived = ticket_arrive(&a.tickets[c_first], a.ticket_tag);
                 const int last = (arrived == (unsigned)(c_last - c_first));
-                if (last) a.tickets[c_first] = 0u;
+                if (last) a.tickets[c_first] = 0ull;
                 s_last = last;
             }
             __syncthreads();
@@ -345,9 +345,9 @@ __global__ void __launch_bounds__(C::THREADS, 1) stream_decode_kernel(const Deco
         __syncthreads();
         if (tid == 0) {
             __threadfence();
-            const unsigned done = atomicAdd(&a.tickets[kTicketCtas], 1u);
+            const unsigned done = ticket_arrive(&a.tickets[kTicketCtas], a.ticket_tag);
             const int last = (done == gridDim.x - 1);
-            if (last) a.tickets[kTicketCtas] = 0u;
+            if (last) a.tickets[kTicketCtas] = 0ull;
             s_last = last;
         }
         __syncthreads();

@@ -517,8 +517,8 @@ def test_padded_head_groups_on_the_64_lane_kernel(gs):
                    oracle.decode_varlen(q, K, V, lens, s)) <= TOL
 
 
-def test_long_dense_groups_with_larger_scores_on_the_single_chain_kernel():
-    # caches of 4096 rows and more run the 64-lane kernel whose scores are one 32-step chain
+def test_long_dense_groups_with_larger_scores():
+    # long dense caches on the 64-lane kernel
     q, K, V, s = make(2120, 1, 64, 1, 8192, 128, 128, v_dist="uniform")
     q, K = 2 * q, 2 * K
     assert max_err(gpu_decode(q, K, V, s, expect_path=moa.PATH_GROUPED), oracle.decode(q, K, V, s)) <= TOL
@@ -528,8 +528,7 @@ def test_long_dense_groups_with_larger_scores_on_the_single_chain_kernel():
 
 @pytest.mark.parametrize("hq,hkv", [(64, 1), (128, 2), (48, 1), (32, 1), (34, 2)])
 def test_fused_steps_on_a_ragged_batch_of_long_and_short_sequences(hq, hkv):
-    """Groups on the tcgen05 kernels, capacity above 4096 rows: sequences of 4096 rows and more
-    and shorter ones are served by different kernels within one step."""
+    """Groups on the tcgen05 kernels: long and very short sequences within one step."""
     B, n_max, D, steps = 4, 4400, 128, 3
     w = mi.Workload("ms", 3100 + hq, B, hq, hkv, n_max, D, D, steps=steps)
     K, V = w.K(), w.V()
@@ -558,20 +557,34 @@ def test_fused_steps_on_a_ragged_batch_of_long_and_short_sequences(hq, hkv):
         assert g.guards_intact()
 
 
-def test_minimum_rows_promise_saves_the_second_launch_of_a_ragged_step():
-    B, hq, hkv, n_max, D = 2, 64, 1, 4500, 128
-    q, K, V, s = make(3200, B, hq, hkv, n_max, D, D)
-    lens = np.array([4400, 4100], np.int32)
-    ref = oracle.decode_varlen(q, K, V, lens, s)
-    launches = {}
-    for promise in (0, 4096):
-        moa.moa_set_option(moa.OPT_MIN_ROWS_HINT, promise)
-        try:
-            moa.moa_profile(1)
-            out = gpu_decode(q, K, V, s, seq_lens=lens, expect_path=moa.PATH_GROUPED)
-            launches[promise] = moa.moa_profile_read()[2]
-            moa.moa_profile(0)
-        finally:
-            moa.moa_set_option(moa.OPT_MIN_ROWS_HINT, 0)
-        assert max_err(out, ref) <= TOL, promise
-    assert launches[4096] == launches[0] - 1
+def test_calls_on_two_streams_with_their_own_workspaces_do_not_disturb_each_other():
+    """The completion counters of the in-kernel merge live in each call's workspace: a long
+    launch on one stream and many short ones on another may overlap freely."""
+    big = mi.Workload("ov1", 3300, 4, 32, 8, 8192, 128, 128)
+    small = mi.Workload("ov2", 3301, 1, 8, 2, 700, 128, 128)
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    dev = {}
+    for name, w in (("big", big), ("small", small)):
+        q, K, V = (torch.from_numpy(x).cuda() for x in (w.q(), w.K(), w.V()))
+        nbytes = moa.moa_workspace_bytes(w.batch, w.h_q, w.h_kv, w.n, w.d_k, w.d_v)
+        # a workspace full of garbage: its contents are undefined on entry
+        ws = torch.randint(-2**31, 2**31 - 1, (nbytes // 4 + 1,), dtype=torch.int32, device="cuda")
+        out = torch.full((w.batch, w.h_q, w.d_v), float("nan"), device="cuda")
+        dev[name] = (w, q, K, V, ws, nbytes, out)
+    torch.cuda.synchronize()
+    outs_small = []
+    for rep in range(3):
+        w, q, K, V, ws, nb, out = dev["big"]
+        moa.moa_decode_attn_varlen(q, K, V, out, w.batch, w.h_q, w.h_kv, None, w.n, w.d_k, w.d_v, w.scale, ws, nb,
+                                   stream=s1.cuda_stream)
+        w, q, K, V, ws, nb, out = dev["small"]
+        for _ in range(40):                      # more launches than any fixed pool of counter slots
+            moa.moa_decode_attn_varlen(q, K, V, out, w.batch, w.h_q, w.h_kv, None, w.n, w.d_k, w.d_v, w.scale, ws, nb,
+                                       stream=s2.cuda_stream)
+        torch.cuda.synchronize()
+        outs_small.append(out.cpu().numpy().copy())
+    assert moa.moa_device_status() == 0
+    for name in ("big", "small"):
+        w, q, K, V, ws, nb, out = dev[name]
+        assert max_err(out.cpu().numpy(), oracle.decode(w.q(), w.K(), w.V(), w.scale)) <= TOL, name
+    assert all(np.array_equal(o, outs_small[0]) for o in outs_small)

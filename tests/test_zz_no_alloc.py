@@ -9,6 +9,7 @@ import numpy as np
 import pytest
 
 import moa_inputs as mi
+import oracle
 import paper_2607_19456_b200 as moa
 
 pytestmark = pytest.mark.gpu
@@ -23,12 +24,15 @@ def both_entry_points(w):
     ref = torch.full((w.batch, w.h_q, w.d_v), float("nan"), device="cuda")
     got = torch.full((w.batch, w.h_q, w.d_v), float("nan"), device="cuda")
     moa.moa_decode_attn(q, K, V, ref, *args)
-    assert moa.moa_last_path() in (moa.PATH_STREAM, moa.PATH_MMA)    # the kernels that use scratch
     moa.moa_decode_attn_noalloc(q, K, V, got, *args)
-    assert moa.moa_last_path() in (moa.PATH_STREAM, moa.PATH_MMA)
+    assert moa.moa_last_path() in (moa.PATH_STREAM, moa.PATH_MMA)    # the kernels that use scratch
     torch.cuda.synchronize()
     assert moa.moa_device_status() == 0
-    return ref.cpu().numpy(), got.cpu().numpy()
+    return ref.cpu().numpy(), got.cpu().numpy(), oracle.decode(w.q(), w.K(), w.V(), w.scale)
+
+
+def err(a, b):
+    return float(np.max(np.abs(a.astype(np.float64) - b.astype(np.float64))))
 
 
 def test_noalloc_matches_the_allocating_entry_point_twice_in_a_row():
@@ -37,16 +41,28 @@ def test_noalloc_matches_the_allocating_entry_point_twice_in_a_row():
     first = mi.Workload("na1", 4101, 3, 32, 8, 6000, 128, 128)
     second = mi.Workload("na2", 4102, 2, 16, 1, 1777, 64, 64)
     for w in (first, second):
-        ref, got = both_entry_points(w)
+        ref, got, want = both_entry_points(w)
         assert np.all(np.isfinite(got))
-        assert float(np.max(np.abs(got.astype(np.float64) - ref.astype(np.float64)))) <= TOL
+        assert err(got, ref) <= TOL          # the two entry points agree ...
+        assert err(got, want) <= TOL         # ... and both with the CPU oracle
+        assert err(ref, want) <= TOL
+
+
+@pytest.mark.parametrize("hq,hkv,d", [(64, 1, 128), (32, 2, 128), (12, 1, 128), (128, 2, 64)])
+def test_noalloc_serves_the_largest_plans(hq, hkv, d):
+    # tiles of 16 heads at d = 128 need the most scratch per CTA (2.5 MB on 148 SMs): MQA with
+    # 64 heads, groups of 16 and of 9..15, and the same at d = 64; twice in a row each
+    w = mi.Workload("na4", 4110 + hq + d, 2, hq, hkv, 3000, d, d)
+    for _ in range(2):
+        ref, got, want = both_entry_points(w)
+        assert err(got, want) <= TOL and err(got, ref) <= TOL
 
 
 def test_noalloc_rejects_a_scratch_need_beyond_the_fixed_array():
     w = mi.Workload("na3", 4103, 1, 8, 1, 64, 128, 128)
     q, K, V = (torch.from_numpy(x).cuda() for x in (w.q(), w.K(), w.V()))
     out = torch.full((w.batch, w.h_q, w.d_v), -7.0, device="cuda")
-    moa.moa_set_option(moa.OPT_NUM_CTAS, 4000)              # 4000 CTAs * 2 slots * 8 heads > 2 MiB
+    moa.moa_set_option(moa.OPT_NUM_CTAS, 4000)              # 4000 CTAs * 2 slots * 8 heads * 132 floats > 4 MiB
     try:
         with pytest.raises(moa.MoaError) as e:
             moa.moa_decode_attn_noalloc(q, K, V, out, w.batch, w.h_q, w.h_kv, w.n, w.d_k, w.d_v, w.scale)
