@@ -113,6 +113,25 @@ __device__ __forceinline__ float exp2_diff(float a, float b)
     return (a == -INFINITY) ? 0.0f : fast_exp2(a - b);
 }
 
+// ---- compensated accumulation for the merges -------------------------------------------
+// A merge adds up to a thousand partial triples.  When the softmax mass sits on a few rows,
+// one partial is of order 1 and the rest are tiny, and every plain addition would round at
+// the size of the large one: the error grows like the square root of the number of
+// partials.  The merges therefore keep a running compensation (Kahan): s += x * f with the
+// rounding error of each addition carried into the next.
+__device__ __forceinline__ void comp_fma(float &s, float &c, float x, float f)
+{
+    const float y = fmaf(x, f, -c);
+    const float t = s + y;
+    c = (t - s) - y;
+    s = t;
+}
+__device__ __forceinline__ void comp_fma4(float4 &s, float4 &c, const float4 &x, float f)
+{
+    comp_fma(s.x, c.x, x.x, f); comp_fma(s.y, c.y, x.y, f);
+    comp_fma(s.z, c.z, x.z, f); comp_fma(s.w, c.w, x.w, f);
+}
+
 // ---- problem description passed to the decode kernels ----------------------------------
 struct DecodeArgs {
     const float *q;           // [batch, h_q, d_k]
@@ -349,10 +368,13 @@ __device__ __forceinline__ void merge_unit_partials(const DecodeArgs &a, float *
     };
     // thread -> (head, float4 column); with fewer threads than G * LPR a thread takes several
     constexpr int kMaxItems = 4;
-    float M[kMaxItems], L[kMaxItems];
-    float4 acc[kMaxItems];
+    float M[kMaxItems], L[kMaxItems], Lc[kMaxItems];
+    float4 acc[kMaxItems], accc[kMaxItems];
 #pragma unroll
-    for (int it = 0; it < kMaxItems; ++it) { M[it] = -INFINITY; L[it] = 0.f; acc[it] = make_float4(0.f, 0.f, 0.f, 0.f); }
+    for (int it = 0; it < kMaxItems; ++it) {
+        M[it] = -INFINITY; L[it] = 0.f; Lc[it] = 0.f;
+        acc[it] = make_float4(0.f, 0.f, 0.f, 0.f); accc[it] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
     for (int base = 0; base < ns; base += per_round) {
         const int cnt = (ns - base < per_round) ? ns - base : per_round;
         for (int i = tid; i < cnt * G; i += nthreads) {
@@ -370,15 +392,15 @@ __device__ __forceinline__ void merge_unit_partials(const DecodeArgs &a, float *
                 for (int i = 0; i < cnt; ++i) Mn = fmaxf(Mn, stage[(i * G + hg) * 2]);
                 const float keep = exp2_diff(M[it], Mn);
                 acc[it].x *= keep; acc[it].y *= keep; acc[it].z *= keep; acc[it].w *= keep;
-                L[it] *= keep;
+                accc[it].x *= keep; accc[it].y *= keep; accc[it].z *= keep; accc[it].w *= keep;
+                L[it] *= keep; Lc[it] *= keep;
                 M[it] = Mn;
 #pragma unroll 8
                 for (int i = 0; i < cnt; ++i) {      // partials in CTA order; the loads are independent
                     const float f = exp2_diff(stage[(i * G + hg) * 2], Mn);
-                    L[it] = fmaf(stage[(i * G + hg) * 2 + 1], f, L[it]);
+                    comp_fma(L[it], Lc[it], stage[(i * G + hg) * 2 + 1], f);
                     const float4 x = __ldcg(reinterpret_cast<const float4 *>(slot_of(c_first + base + i, hg) + d4 * 4));
-                    acc[it].x = fmaf(x.x, f, acc[it].x); acc[it].y = fmaf(x.y, f, acc[it].y);
-                    acc[it].z = fmaf(x.z, f, acc[it].z); acc[it].w = fmaf(x.w, f, acc[it].w);
+                    comp_fma4(acc[it], accc[it], x, f);
                 }
             }
         }

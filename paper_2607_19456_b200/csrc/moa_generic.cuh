@@ -95,13 +95,13 @@ __global__ void __launch_bounds__(128) combine_partials_kernel(const float *part
     const float *base = parts + (size_t)r * ps;
     float M = -INFINITY;
     for (int i = 0; i < nparts; ++i) M = fmaxf(M, base[(size_t)i * part_stride + d_v]);
-    float L = 0.f;
+    float L = 0.f, Lc = 0.f;
     for (int i = 0; i < nparts; ++i)
-        L = fmaf(base[(size_t)i * part_stride + d_v + 1], exp2_diff(base[(size_t)i * part_stride + d_v], M), L);
+        comp_fma(L, Lc, base[(size_t)i * part_stride + d_v + 1], exp2_diff(base[(size_t)i * part_stride + d_v], M));
     for (int d = threadIdx.x; d < d_v; d += blockDim.x) {
-        float acc = 0.f;
+        float acc = 0.f, accc = 0.f;
         for (int i = 0; i < nparts; ++i)
-            acc = fmaf(base[(size_t)i * part_stride + d], exp2_diff(base[(size_t)i * part_stride + d_v], M), acc);
+            comp_fma(acc, accc, base[(size_t)i * part_stride + d], exp2_diff(base[(size_t)i * part_stride + d_v], M));
         out[(size_t)r * d_v + d] = acc / L;
     }
 }

@@ -729,8 +729,8 @@ template <int GH>
 __global__ void __launch_bounds__(128) grouped_combine_kernel(const GroupedArgs a)
 {
     constexpr int PS = 132;
-    __shared__ float4 s_acc[4][32];
-    __shared__ float s_l[4];
+    __shared__ float4 s_acc[4][32], s_accc[4][32];
+    __shared__ float s_l[4], s_lc[4];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const long long wid = blockIdx.x;
     const int b = (int)(wid / a.h_q), gq = (int)(wid % a.h_q);
@@ -760,28 +760,29 @@ __global__ void __launch_bounds__(128) grouped_combine_kernel(const GroupedArgs 
         for (int off = 16; off >= 1; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
         M = fmaxf(M, m);
     }
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    float L = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f), accc = acc;
+    float L = 0.f, Lc = 0.f;
 #pragma unroll 4
     for (int sp = warp; sp < used; sp += 4) {
         const float *row = base + (size_t)sp * stride;
         const float f = exp2_diff(row[128], M);
-        L = fmaf(row[129], f, L);
+        comp_fma(L, Lc, row[129], f);
         const float4 t = *reinterpret_cast<const float4 *>(row + lane * 4);
-        acc.x = fmaf(t.x, f, acc.x); acc.y = fmaf(t.y, f, acc.y);
-        acc.z = fmaf(t.z, f, acc.z); acc.w = fmaf(t.w, f, acc.w);
+        comp_fma4(acc, accc, t, f);
     }
-    s_acc[warp][lane] = acc;
-    if (lane == 0) s_l[warp] = L;
+    // (sum, compensation) of the four warps, added in warp order with the same care
+    s_acc[warp][lane] = acc; s_accc[warp][lane] = accc;
+    if (lane == 0) { s_l[warp] = L; s_lc[warp] = Lc; }
     __syncthreads();
     if (warp != 0) return;
-    acc = s_acc[0][lane];
-    L = s_l[0];
+    acc = s_acc[0][lane]; accc = s_accc[0][lane];
+    L = s_l[0]; Lc = s_lc[0];
 #pragma unroll
     for (int w = 1; w < 4; ++w) {
-        const float4 t = s_acc[w][lane];
-        acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
-        L += s_l[w];
+        comp_fma4(acc, accc, s_acc[w][lane], 1.0f);
+        comp_fma4(acc, accc, s_accc[w][lane], -1.0f);
+        comp_fma(L, Lc, s_l[w], 1.0f);
+        comp_fma(L, Lc, s_lc[w], -1.0f);
     }
     if (a.partial_out != nullptr) {
         float *dst = a.partial_out + ((size_t)b * a.h_q + gq) * 132;

@@ -267,15 +267,14 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
                 float M = -INFINITY;
 #pragma unroll
                 for (int v = 0; v < P; ++v) M = fmaxf(M, merge_ml[(v * 8 + h8) * 2]);
-                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                float L = 0.f;
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f), accc = acc;
+                float L = 0.f, Lc = 0.f;
 #pragma unroll
                 for (int v = 0; v < P; ++v) {
                     const float f = exp2_diff(merge_ml[(v * 8 + h8) * 2], M);
                     const float4 x = *reinterpret_cast<const float4 *>(merge_o + ((size_t)(v * 8 + h8)) * D + d4 * 4);
-                    acc.x = fmaf(x.x, f, acc.x); acc.y = fmaf(x.y, f, acc.y);
-                    acc.z = fmaf(x.z, f, acc.z); acc.w = fmaf(x.w, f, acc.w);
-                    L = fmaf(merge_ml[(v * 8 + h8) * 2 + 1], f, L);
+                    comp_fma4(acc, accc, x, f);
+                    comp_fma(L, Lc, merge_ml[(v * 8 + h8) * 2 + 1], f);
                 }
                 if (complete) {
                     if (hg < a.g_s) emit_columns(a, (size_t)cc.b * a.h_q + (size_t)cc.h * a.g_s + hg, D, d4, acc, M, L);

@@ -216,15 +216,14 @@ __global__ void __launch_bounds__(C::THREADS, 1) stream_decode_kernel(const Deco
             float M = -INFINITY;
 #pragma unroll 4
             for (int v = 0; v < VW; ++v) M = fmaxf(M, merge_ml[(v * G + g) * 2]);
-            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-            float L = 0.f;
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f), accc = acc;
+            float L = 0.f, Lc = 0.f;
 #pragma unroll 4
             for (int v = 0; v < VW; ++v) {
                 const float f = exp2_diff(merge_ml[(v * G + g) * 2], M);
                 const float4 t = *reinterpret_cast<const float4 *>(merge_o + ((size_t)(v * G + g)) * D + d4 * 4);
-                acc.x = fmaf(t.x, f, acc.x); acc.y = fmaf(t.y, f, acc.y);
-                acc.z = fmaf(t.z, f, acc.z); acc.w = fmaf(t.w, f, acc.w);
-                L = fmaf(merge_ml[(v * G + g) * 2 + 1], f, L);
+                comp_fma4(acc, accc, t, f);
+                comp_fma(L, Lc, merge_ml[(v * G + g) * 2 + 1], f);
             }
             if (complete) {
                 if (g < a.g_s) emit_columns(a, (size_t)cc.b * a.h_q + (size_t)cc.h * a.g_s + g, D, d4, acc, M, L);
@@ -409,16 +408,15 @@ __global__ void __launch_bounds__(128) stream_combine_kernel(const DecodeArgs a,
     };
     float M = -INFINITY;
     for (long long c = c_first; c <= c_last; ++c) M = fmaxf(M, slot_ptr(c)[D]);
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    float L = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f), accc = acc;
+    float L = 0.f, Lc = 0.f;
     for (long long c = c_first; c <= c_last; ++c) {
         const float *p = slot_ptr(c);
         const float f = exp2_diff(p[D], M);
-        L = fmaf(p[D + 1], f, L);
+        comp_fma(L, Lc, p[D + 1], f);
         if (lane < LPR) {
             const float4 t = *reinterpret_cast<const float4 *>(p + lane * 4);
-            acc.x = fmaf(t.x, f, acc.x); acc.y = fmaf(t.y, f, acc.y);
-            acc.z = fmaf(t.z, f, acc.z); acc.w = fmaf(t.w, f, acc.w);
+            comp_fma4(acc, accc, t, f);
         }
     }
     if (lane < LPR) emit_columns(a, (size_t)b * a.h_q + gq, D, lane, acc, M, L);
