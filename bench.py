@@ -387,7 +387,8 @@ def time_steps(run, steps, warmup, side, sampler=None, bracket=False, segment=0)
     if sampler:
         sampler.start()
     run.profile(2 if bracket else 1)
-    cuts = sorted({0, steps} | ({segment, steps - segment} if 0 < segment and 2 * segment <= steps else set()))
+    have_segs = 0 < segment and 2 * segment <= steps
+    cuts = sorted({0, steps} | ({segment, steps - segment} if have_segs else set()))
     marks = {}
     for i in range(steps + 1):
         if i in cuts:
@@ -404,7 +405,7 @@ def time_steps(run, steps, warmup, side, sampler=None, bracket=False, segment=0)
     barrier()
     ms = side.ms_between(marks[0], marks[steps]) / steps
     segs = None
-    if len(cuts) == 4:
+    if have_segs:
         segs = [side.ms_between(marks[0], marks[segment]) / segment,
                 side.ms_between(marks[steps - segment], marks[steps]) / segment]
     return ms, (kern_ms / kern_n if kern_n else None), launches, clocks, segs

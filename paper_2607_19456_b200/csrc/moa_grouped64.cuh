@@ -35,9 +35,11 @@
 // softmax group does is on the tensor core's critical path: while it works on tile t the
 // tensor core multiplies tile t+1's K chunks and tile t-1's V chunks.
 //
-// Roles (736 threads): warp 0 TMA producer, warp 1 MMA issuer (and owner of the tensor
+// Roles (768 threads): warp 0 TMA producer, warp 3 MMA issuer (and owner of the tensor
 // memory allocation), warp 22 batch scheduler, warps 4-19 softmax (warp w: lane quadrant w % 4, columns 32 * ((w-4)/4)
-// .. +31 of a 128-column region), warps 2, 3, 20, 21 turn chunks into their lo parts.  Every
+// .. +31 of a 128-column region), warps 1, 2, 20, 21 turn chunks into their lo parts, warp 23
+// idles.  After the set-up the softmax warpgroups take registers from the others
+// (setmaxnreg): they hold the running weighted sum and a tile's scores at once.  Every
 // hand-off is an mbarrier; every wait is bounded.
 #pragma once
 
@@ -76,7 +78,7 @@ struct Grouped64Cfg {
     static constexpr int NBUF = 13;                // 16 KB chunk buffers
     static constexpr int NG = 4;                   // groups of four chunks with barriers of their own (> NBUF / 4)
     static constexpr int CHUNK = 16384;
-    static constexpr int THREADS = 736;            // 23 warps
+    static constexpr int THREADS = 768;            // 24 warps = 6 warpgroups (register reallocation works on whole warpgroups)
     static constexpr int QN = 4;                   // batch descriptors queued between scheduler and issuer
     static constexpr int CONV_WARPS = 4;
     static constexpr int SOFT_WARPS = 16;
@@ -223,6 +225,10 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
     tc::fence_before_sync();
     __syncthreads();
     tc::fence_after_sync();
+    // 24 warps x 80 registers at launch; the two warpgroups without softmax work (warps 0-3 and
+    // 20-23) hand 32 registers per thread back to the pool of the CTA, from which the four softmax warpgroups
+    // take 16 each (only registers that were handed back can be taken).
+    if (!is_soft) asm volatile("setmaxnreg.dec.sync.aligned.u32 48;");
 
     if (warp == 0) {
         // ================= TMA producer =================
@@ -369,73 +375,62 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
         }
     } else if (is_soft) {
         // ================= softmax group: thread = (lane of the stacked operand, 32 columns) ==========
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 96;");
         float Om[32];                              // running weighted sum: this lane's part, features col0..col0+31
 #pragma unroll
         for (int i = 0; i < 32; ++i) Om[i] = 0.f;
         float m_run = -INFINITY, l_run = 0.f, alpha_prev = 0.f;
         bool ok = true;
         auto fold = [&](float alpha) {             // Om = alpha * Om + (weighted sum of the last tile)
-            if constexpr (PRECISE) {
 #pragma unroll
-                for (int hf = 0; hf < 2; ++hf) {
-                    uint32_t o[16];
-                    tc::tmem_ld16(tO + lane_addr + col0 + 16 * hf, o);
-                    tc::tmem_ld_wait();
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) Om[16 * hf + i] = fmaf(Om[16 * hf + i], alpha, __uint_as_float(o[i]));
-                }
-            } else {
-                uint32_t o[32];
-                tc::tmem_ld32(tO + lane_addr + col0, o);
+            for (int hf = 0; hf < 2; ++hf) {
+                uint32_t o[16];
+                tc::tmem_ld16(tO + lane_addr + col0 + 16 * hf, o);
                 tc::tmem_ld_wait();
 #pragma unroll
-                for (int i = 0; i < 32; ++i) Om[i] = fmaf(Om[i], alpha, __uint_as_float(o[i]));
+                for (int i = 0; i < 16; ++i) Om[16 * hf + i] = fmaf(Om[16 * hf + i], alpha, __uint_as_float(o[i]));
             }
         };
         for (int t = 0; t < T; ++t) {
             const uint32_t tSP = tSP_of(t) + lane_addr + col0;
             const int row0 = row_base + t * C::TILE + col0;
             float sc[16];                              // scores: the hi lane of a head columns 0..15, the lo lane 16..31
-            if constexpr (PRECISE) {                   // the K_hi products of the tile, before the K_lo products overwrite them
-                ok = ok && wait_suspended(bar_group_hi(group_k(t)), par_group_done(group_k(t)), abort_flag);
-                tc::fence_after_sync();                // (after a failed wait the values are not used)
-#pragma unroll
-                for (int hf = 0; hf < 2; ++hf) {       // 16 columns at a time, to stay within the registers
-                    uint32_t xh[16];
-                    tc::tmem_ld16(tSP + 16 * hf, xh);
-                    tc::tmem_ld_wait();
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const float mine = __uint_as_float(xh[i]);
-                        const float sum = mine + __shfl_xor_sync(0xffffffffu, mine, 16);
-                        if ((hf == 1) == is_lo) sc[i] = sum;
-                    }
-                }
-                tc::fence_before_sync();
-                __syncwarp();
-                if (ok && lane == 0) tc::mbar_arrive(bar_shread);
-            }
-            ok = ok && wait_suspended(bar_group_done(group_k(t)), par_group_done(group_k(t)), abort_flag);
-            if (named_or(1 + qd, 128, !ok)) { ok = false; break; }    // the four warps of a quadrant leave together
-            tc::fence_after_sync();
             // Scores of this lane's head against 32 cached rows.  The two lanes of a head hold the
             // terms of its hi and of its lo query part; they share the work: the hi lane takes
             // columns 0..15, the lo lane columns 16..31, each gets the other lane's terms for its
             // columns by shuffle and hands back the part of the probabilities the other lane stores.
             if constexpr (PRECISE) {
+                // the K_hi products of the tile are read out before the K_lo products start the
+                // region afresh; the two are added here in fp32
+                uint32_t xa[32];
+                ok = ok && wait_suspended(bar_group_hi(group_k(t)), par_group_done(group_k(t)), abort_flag);
+                tc::fence_after_sync();                // (after a failed wait the values are not used)
+                tc::tmem_ld32(tSP, xa);
+                tc::tmem_ld_wait();
+                tc::fence_before_sync();
+                __syncwarp();
+                if (ok && lane == 0) tc::mbar_arrive(bar_shread);
+                ok = ok && wait_suspended(bar_group_done(group_k(t)), par_group_done(group_k(t)), abort_flag);
+                if (named_or(1 + qd, 128, !ok)) { ok = false; break; }    // the four warps of a quadrant leave together
+                tc::fence_after_sync();
 #pragma unroll
-                for (int hf = 0; hf < 2; ++hf) {
-                    uint32_t xh[16];
-                    tc::tmem_ld16(tSP + 16 * hf, xh);
+                for (int hf = 0; hf < 2; ++hf) {       // 16 columns at a time, to stay within the registers
+                    uint32_t xb[16];
+                    tc::tmem_ld16(tSP + 16 * hf, xb);
                     tc::tmem_ld_wait();
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const float mine = __uint_as_float(xh[i]);
-                        const float sum = mine + __shfl_xor_sync(0xffffffffu, mine, 16);
-                        if ((hf == 1) == is_lo) sc[i] += sum;
-                    }
+                    for (int i = 0; i < 16; ++i)
+                        xa[16 * hf + i] = __float_as_uint(__uint_as_float(xa[16 * hf + i]) + __uint_as_float(xb[i]));
+                }
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {       // each lane sends what the other needs
+                    const float other = __shfl_xor_sync(0xffffffffu, __uint_as_float(is_lo ? xa[i] : xa[16 + i]), 16);
+                    sc[i] = __uint_as_float(is_lo ? xa[16 + i] : xa[i]) + other;
                 }
             } else {
+                ok = ok && wait_suspended(bar_group_done(group_k(t)), par_group_done(group_k(t)), abort_flag);
+                if (named_or(1 + qd, 128, !ok)) { ok = false; break; }    // the four warps of a quadrant leave together
+                tc::fence_after_sync();
                 uint32_t x[32];
                 tc::tmem_ld32(tSP, x);
                 tc::tmem_ld_wait();
@@ -465,22 +460,7 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
             // and hands the other part to the other lane of the head; 16 columns at a time (the hi
             // lane's columns first), to stay within the registers
             float lsum = 0.f;
-            if constexpr (PRECISE) {
-#pragma unroll
-                for (int hf = 0; hf < 2; ++hf) {
-                    const bool mine = ((hf == 1) == is_lo);     // this half's columns are this lane's
-                    uint32_t xh[16];
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const float p = mine ? fast_exp2(sc[i] - m_new) : 0.f;
-                        lsum += p;
-                        const float ph = tf32_hi(p), pl = p - ph;
-                        const float got = __shfl_xor_sync(0xffffffffu, is_lo ? ph : pl, 16);
-                        xh[i] = __float_as_uint(mine ? (is_lo ? pl : ph) : got);
-                    }
-                    tc::tmem_st16(tSP + 16 * hf, xh);
-                }
-            } else {
+            {
                 uint32_t x[32];
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
@@ -536,7 +516,7 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
                 slot[129] = (lx[head] + lx[64 + head]) + (lx[128 + head] + lx[192 + head]);
             }
         }
-    } else {
+    } else if (warp != 23) {
         // ================= converters: chunk -> its lo part, in place =================
         // Each of the four converter warps takes every fourth chunk, so that four conversions are in flight: a
         // conversion is a chain of barrier wait, 16 KB of loads, 16 KB of stores and barrier
