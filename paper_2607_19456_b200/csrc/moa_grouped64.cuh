@@ -192,6 +192,25 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
     tc::fence_before_sync();
     __syncthreads();
     tc::fence_after_sync();
+    // The first ring-full of chunks needs nothing but the barriers: the producer starts those
+    // loads now, so that they travel while the query operand is being built.
+    ChunkSeq pseq(T);                              // the producer's position (warp 0, lane 0)
+    auto issue_load = [&](const ChunkSeq &s) {
+        const int buf = s.seq % NBUF;
+        const uint32_t dst = sRing + (uint32_t)buf * C::CHUNK;
+        const uint32_t fb = bar_gfull((s.seq >> 2) % NG);
+        mbar_expect_tx(fb, C::CHUNK);
+        const bool tail = (s.t == tail_t);
+        const int row = tail ? 0 : row_base + s.t * C::TILE;
+        if (s.is_k) {
+            tc::tma_load_3d(dst, tail ? &tmapKt : &tmapK, 32 * s.c, row, unit, fb);
+        } else {
+            for (int dg = 0; dg < 4; ++dg)
+                tc::tma_load_3d(dst + dg * 4096, tail ? &tmapVt : &tmapV, 32 * dg, row + 32 * s.c, unit, fb);
+        }
+    };
+    if (warp == 0 && lane == 0)
+        for (; !pseq.done && pseq.seq < NBUF; pseq.next()) issue_load(pseq);
     const uint32_t tmem = *tmem_slot;
     const uint32_t tQ = tmem, tO = tmem + 384u;
     auto tSP_of = [tmem](int t) -> uint32_t { return tmem + 128u + (uint32_t)(t & 1) * 128u; };
@@ -233,20 +252,10 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
     if (warp == 0) {
         // ================= TMA producer =================
         if (lane == 0) {
-            for (ChunkSeq s(T); !s.done; s.next()) {
-                const int buf = s.seq % NBUF, use = s.seq / NBUF;
+            for (; !pseq.done; pseq.next()) {
+                const int buf = pseq.seq % NBUF, use = pseq.seq / NBUF;
                 if (use > 0 && !wait_suspended(bar_empty(buf), (uint32_t)(use - 1) & 1u, abort_flag)) break;
-                const uint32_t dst = sRing + (uint32_t)buf * C::CHUNK;
-                const uint32_t fb = bar_gfull((s.seq >> 2) % NG);
-                mbar_expect_tx(fb, C::CHUNK);
-                const bool tail = (s.t == tail_t);
-                const int row = tail ? 0 : row_base + s.t * C::TILE;
-                if (s.is_k) {
-                    tc::tma_load_3d(dst, tail ? &tmapKt : &tmapK, 32 * s.c, row, unit, fb);
-                } else {
-                    for (int dg = 0; dg < 4; ++dg)
-                        tc::tma_load_3d(dst + dg * 4096, tail ? &tmapVt : &tmapV, 32 * dg, row + 32 * s.c, unit, fb);
-                }
+                issue_load(pseq);
             }
         }
     } else if (warp == 22) {
