@@ -290,6 +290,13 @@ const char *moa_strerror(int code);
  *                        that keeps the query and probability operands in tensor memory
  *                        (64 head lanes, smaller groups padded); 1 = only the kernel with
  *                        these operands in shared memory (groups of exactly 16, 32, 64).
+ *   MOA_OPT_WAIT_LIMIT : number of polls after which the FMA streaming kernel gives up waiting
+ *                        for a tile it has requested (0 = the built-in limit of 2^22 polls).
+ *                        When a wait runs out the kernel sets MOA_STATUS_WAIT_TIMEOUT, stops
+ *                        consuming and returns; the results of that call are invalid.
+ *   MOA_OPT_TEST_SKIP_COPY : test hook for exactly that path: the copies of the row block with
+ *                        this flat index are announced but never issued (nothing is in flight,
+ *                        nothing out of bounds), so the wait for them runs out (-1 = off).
  * moa_last_path() reports which kernel family the last successful decode call used.
  */
 #define MOA_OPT_FORCE_PATH 1
@@ -297,6 +304,8 @@ const char *moa_strerror(int code);
 #define MOA_OPT_GROUPED_HEADS 3
 #define MOA_OPT_DEPENDENT_LAUNCH 4
 #define MOA_OPT_GROUPED_OPERANDS 5
+#define MOA_OPT_WAIT_LIMIT 7
+#define MOA_OPT_TEST_SKIP_COPY 8
 #define MOA_PATH_GENERIC   1   /* any d_k, d_v, alignment: one CTA per (batch, query head) */
 #define MOA_PATH_STREAM    2   /* split-sequence streaming kernel on the FMA units, d in {32,64,128} */
 #define MOA_PATH_GROUPED   3   /* tcgen05 tensor-core kernels for groups of 17..64 heads (16 when forced), d = 128, dense layout */

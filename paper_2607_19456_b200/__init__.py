@@ -18,6 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libmoa.so")
 OK, ERR_INVALID, ERR_UNSUPPORTED, ERR_ALIGN, ERR_CAPACITY, ERR_WORKSPACE, ERR_CUDA = range(7)
 STATUS_APPEND_RANGE, STATUS_SEQLEN_RANGE, STATUS_WAIT_TIMEOUT = 1, 2, 4
 OPT_FORCE_PATH, OPT_NUM_CTAS, OPT_GROUPED_HEADS, OPT_DEPENDENT_LAUNCH, OPT_GROUPED_OPERANDS = 1, 2, 3, 4, 5
+OPT_WAIT_LIMIT, OPT_TEST_SKIP_COPY = 7, 8
 NOALLOC_SCRATCH_BYTES = 4 << 20
 PATH_AUTO, PATH_GENERIC, PATH_STREAM, PATH_GROUPED, PATH_MMA = 0, 1, 2, 3, 4
 

@@ -72,6 +72,8 @@ struct TimedLaunch {                      // RAII: event before / after the domi
 static inline void count_launch(int n = 1) { if (g_prof_on) g_prof_all += n; }
 
 static int g_dependent_launch = 1;   // MOA_OPT_DEPENDENT_LAUNCH
+static int g_wait_limit = 0;         // MOA_OPT_WAIT_LIMIT: 0 = the built-in limit
+static long long g_skip_copy_block = -1;   // MOA_OPT_TEST_SKIP_COPY
 
 // Launch with programmatic stream serialisation: the kernel may start while its predecessor
 // in the stream is still running and synchronises with it on the device (griddepcontrol.wait).
@@ -621,6 +623,8 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
     a.qscale = scale * kLog2e;
     a.Kw = nullptr; a.Vw = nullptr; a.k_new = nullptr; a.v_new = nullptr; a.lens_rw = nullptr;
     a.tickets = nullptr; a.ticket_tag = 0;
+    a.wait_limit = g_wait_limit > 0 ? (uint32_t)g_wait_limit : kWaitLimit;
+    a.skip_copy_block = g_skip_copy_block;
     a.partial_out = partial_out;
     if (fused != nullptr && path == MOA_PATH_GENERIC) return MOA_ERR_UNSUPPORTED;
 
@@ -1127,6 +1131,16 @@ int moa_set_option(int option, int value)
     if (option == MOA_OPT_DEPENDENT_LAUNCH) {
         if (value != 0 && value != 1) return MOA_ERR_INVALID;
         g_dependent_launch = value;
+        return MOA_OK;
+    }
+    if (option == MOA_OPT_WAIT_LIMIT) {
+        if (value < 0) return MOA_ERR_INVALID;
+        g_wait_limit = value;
+        return MOA_OK;
+    }
+    if (option == MOA_OPT_TEST_SKIP_COPY) {
+        if (value < -1) return MOA_ERR_INVALID;
+        g_skip_copy_block = value;
         return MOA_OK;
     }
     if (option == MOA_OPT_NUM_CTAS) {

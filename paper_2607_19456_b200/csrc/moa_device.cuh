@@ -80,9 +80,9 @@ __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepco
 // gives up, raises MOA_STATUS_WAIT_TIMEOUT and leaves without touching the data.
 constexpr uint32_t kWaitLimit = 1u << 22;
 
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t limit = kWaitLimit)
 {
-    for (uint32_t it = 0; it < kWaitLimit; ++it)
+    for (uint32_t it = 0; it < limit; ++it)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
@@ -162,6 +162,9 @@ struct DecodeArgs {
     unsigned long long ticket_tag; // what one arrival adds to a counter word: (launch tag << 20) + 1
     float *partial_out;       // nullptr, or [batch, h_q, d_v + 4]: emit the unnormalised triple
                               // (o[d_v], m, l, 2 pad) instead of the normalised output row
+    uint32_t wait_limit;      // polls after which a wait on a tile's arrival gives up (FMA streaming kernel)
+    long long skip_copy_block;// test hook: the copies of this row block are announced but never
+                              // issued, so the wait for them runs out (-1: off)
 };
 
 // Final emission of one float4 column group of a (batch, query head) row: the normalised

@@ -151,11 +151,12 @@ __global__ void __launch_bounds__(C::THREADS, 1) stream_decode_kernel(const Deco
             const uint32_t dst = smem_u32(my_ring + (size_t)stage * C::STAGE_FLOATS);
             const uint32_t bytes = (uint32_t)nr_cache * D * 4u;
             mbar_expect_tx(bar, 2u * (uint32_t)nr * D * 4u);
-            if (nr_cache > 0) {
+            const bool skip = (jl == a.skip_copy_block);     // test hook: nothing is copied, the wait expires
+            if (nr_cache > 0 && !skip) {
                 bulk_g2s(dst, Ksrc, bytes, bar);
                 bulk_g2s(dst + R * D * 4u, Vsrc, bytes, bar);
             }
-            if (has_new) {
+            if (has_new && !skip) {
                 bulk_g2s(dst + bytes, a.k_new + slab * D, D * 4u, bar);
                 bulk_g2s(dst + R * D * 4u + bytes, a.v_new + slab * D, D * 4u, bar);
             }
@@ -317,7 +318,7 @@ __global__ void __launch_bounds__(C::THREADS, 1) stream_decode_kernel(const Deco
             begin_unit();
         }
         const int stage = k % S;
-        if (!failed && !mbar_wait_bounded(my_bar0 + 8u * stage, (uint32_t)(k / S) & 1u)) {
+        if (!failed && !mbar_wait_bounded(my_bar0 + 8u * stage, (uint32_t)(k / S) & 1u, a.wait_limit)) {
             failed = true;
             if (lane == 0) raise_status(MOA_STATUS_WAIT_TIMEOUT);
         }
