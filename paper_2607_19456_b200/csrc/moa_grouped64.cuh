@@ -75,11 +75,10 @@ struct Grouped64Cfg {
     static constexpr int GH = 64;
     static constexpr int D = 128;
     static constexpr int TILE = 128;
-    static constexpr int NBUF = 13;                // 16 KB chunk buffers
+    static constexpr int NBUF = 12;                // 16 KB chunk buffers: three groups of four, so that a group always sits in the same buffers
     static constexpr int NG = 4;                   // groups of four chunks with barriers of their own (> NBUF / 4)
     static constexpr int CHUNK = 16384;
     static constexpr int THREADS = 768;            // 24 warps = 6 warpgroups (register reallocation works on whole warpgroups)
-    static constexpr int QN = 4;                   // batch descriptors queued between scheduler and issuer
     static constexpr int CONV_WARPS = 4;
     static constexpr int SOFT_WARPS = 16;
     static constexpr int PS = D + 4;
@@ -92,9 +91,52 @@ struct Grouped64Cfg {
     static constexpr uint32_t OFF_ABORT = OFF_TMEM + 4;
     static constexpr uint32_t OFF_SHARE = OFF_ABORT + 4;            // flat mode: unit, first CTA, CTA count
     static constexpr uint32_t OFF_QCNT = OFF_SHARE + 16;            // batches published / batches taken
-    static constexpr uint32_t OFF_QUEUE = (OFF_QCNT + 8 + 15) / 16 * 16;   // [QN][16] words
-    static constexpr size_t SMEM_BYTES = OFF_QUEUE + QN * 64;
+    static constexpr size_t SMEM_BYTES = OFF_QCNT + 16;
 };
+
+// Batch number -> what it multiplies: operand kind, hi or lo pass, tile, chunk group (ring order).
+struct Batch64 {
+    bool is_k, is_hi;
+    int t, g;
+    __device__ __forceinline__ Batch64(int i, int T)
+    {
+        if (i < 2) { is_k = true; t = 0; is_hi = (i == 0); }
+        else {
+            const int jj = i - 2, r = jj & 3;
+            t = jj >> 2;
+            if (t >= T - 1) { is_k = false; t = T - 1; is_hi = (r == 0); }
+            else { is_k = (r == 0 || r == 2); is_hi = (r < 2); if (is_k) t += 1; }
+        }
+        g = is_k ? (t == 0 ? 0 : 2 * t - 1) : (t < T - 1 ? 2 * t + 2 : 2 * T - 1);
+    }
+};
+
+// The sixteen products of one batch: group slot SLOT of the ring (buffers 4*SLOT .. 4*SLOT+3), K
+// chunks (K-major B operand) or V chunks (MN-major).  `ring_lo` is the ring's shared-memory
+// address >> 4; all other descriptor fields are constants.  Issued by one thread.
+template <bool IS_K, int SLOT>
+__device__ __forceinline__ void issue_batch64(uint32_t d, uint32_t a0, uint32_t ring_lo, uint32_t acc0,
+                                              uint32_t bar_first, uint32_t bar_mid, uint32_t bar_end)
+{
+    // descriptor words: [addr>>4 | lbo>>4 << 16] and [sbo>>4 | version << 14 | layout << 29]
+    constexpr uint32_t hiword = IS_K ? (64u | (1u << 14) | (2u << 29)) : (32u | (1u << 14) | (1u << 29));
+    constexpr uint32_t lbo = IS_K ? (1u << 16) : (256u << 16);
+    constexpr uint32_t step = IS_K ? 2u : 64u;                       // descriptor step per k-step
+    constexpr uint32_t idesc = tc::idesc_tf32(128, 128, false, !IS_K);
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+#pragma unroll
+        for (uint32_t ks = 0; ks < 4; ++ks) {
+            const uint32_t lo = ring_lo + (lbo + (uint32_t)(4 * SLOT + c) * (Grouped64Cfg::CHUNK >> 4) + ks * step);
+            tc::mma_tf32_ts(d, a0 + (32u * c + 8u * ks), tc::pack64(lo, hiword), idesc, (c == 0 && ks == 0) ? acc0 : 1u);
+        }
+        // hi batch: one commit per pair of chunks (bar_first = 0: none after chunks 0 and 2);
+        // lo batch: one per chunk, so that the producer can refill buffer by buffer
+        if (bar_first != 0u) tc::mma_commit(bar_first + 8u * (uint32_t)c);
+        else if (c == 1) tc::mma_commit(bar_mid);
+    }
+    if (bar_first == 0u) tc::mma_commit(bar_end);
+}
 
 template <bool PRECISE>
 __global__ void __launch_bounds__(Grouped64Cfg::THREADS, 1)
@@ -113,8 +155,6 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + C::OFF_ABORT);
     int *s_share = reinterpret_cast<int *>(smem + C::OFF_SHARE);
     volatile int *q_ready = reinterpret_cast<volatile int *>(smem + C::OFF_QCNT);
-    volatile int *q_taken = q_ready + 1;
-    const uint32_t queue = smem_u32(smem) + C::OFF_QUEUE;       // 64 bytes per batch
 
     const uint32_t sRing = smem_u32(smem) + C::OFF_RING;
     // Per ring buffer (every role sees every use of every buffer, so one parity bit per use):
@@ -183,7 +223,7 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
         mbar_init(bar_ofree, C::SOFT_WARPS); mbar_init(bar_shread, C::SOFT_WARPS);
         mbar_fence_init();
         *abort_flag = 0;
-        *q_ready = 0; *q_taken = 0;
+        *q_ready = 0;
         tc::prefetch_tmap(&tmapK);
         tc::prefetch_tmap(&tmapV);
         if (a.tailK != nullptr) { tc::prefetch_tmap(&tmapKt); tc::prefetch_tmap(&tmapVt); }
@@ -260,125 +300,73 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
         }
     } else if (warp == 22) {
         // ================= batch scheduler (one thread) =================
-        // The thread that issues tcgen05.mma has about 64 cycles between two products before the
-        // tensor pipe runs dry, so everything else the issue needs is done here: the order of the
-        // batches, their descriptors and barrier addresses, and the waiting.  Batches of 16
-        // products, in the order
+        // The thread that issues tcgen05.mma cannot look at a barrier between two products without
+        // draining the tensor pipe, so the waiting is done here.  Batches of 16 products, in the order
         //     K_hi(0) K_lo(0)  [K_hi(t+1) V_hi(t) K_lo(t+1) V_lo(t)] for t = 0..T-2  V_hi(T-1) V_lo(T-1):
         // between the hi and the lo batch of a group runs a batch of the other operand, which is
-        // the time the converters have.  A batch is published (16 words) once its barriers are
-        // complete; the queue holds QN of them.
+        // the time the converters have.  Batch i is released (q_ready = i + 1) once everything
+        // it reads is complete; the issuer derives the rest from i.
         if (lane == 0) {
-            const uint32_t idesc_k = tc::idesc_tf32(128, 128, false, false);   // B = K chunk, K-major
-            const uint32_t idesc_v = tc::idesc_tf32(128, 128, false, true);    // B = V chunk, MN-major
-            // descriptor words: [addr>>4 | lbo>>4 << 16] and [sbo>>4 | version << 14 | layout << 29]
-            const uint32_t k_hiword = 64u | (1u << 14) | (2u << 29), v_hiword = 32u | (1u << 14) | (1u << 29);
-            const uint32_t k_base = (sRing >> 4) | (1u << 16), v_base = (sRing >> 4) | (256u << 16);
             const int nbatch = 4 * T;
             bool ok = true;
             for (int i = 0; ok && i < nbatch; ++i) {
-                bool is_k, is_hi;
-                int t;
-                if (i < 2) { is_k = true; t = 0; is_hi = (i == 0); }
-                else {
-                    const int jj = i - 2, r = jj & 3;
-                    t = jj >> 2;
-                    if (t >= T - 1) { is_k = false; t = T - 1; is_hi = (r == 0); }
-                    else { is_k = (r == 0 || r == 2); is_hi = (r < 2); if (is_k) t += 1; }
-                }
-                const int g = is_k ? (t == 0 ? 0 : 2 * t - 1) : (t < T - 1 ? 2 * t + 2 : 2 * T - 1);
-                const int gs = g % NG;
-                const uint32_t gpar = (uint32_t)(g / NG) & 1u;
-                uint32_t w[16];
-                w[0] = is_k ? tSP_of(t) : tO;                       // D
-                w[1] = is_k ? tQ : tSP_of(t);                       // A
-                w[2] = is_k ? k_hiword : v_hiword;
-                w[3] = is_k ? 2u : 64u;                             // descriptor step per k-step
-                w[4] = is_k ? idesc_k : idesc_v;
-                w[5] = (is_hi || (is_k && precise)) ? 0u : 1u;      // accumulate flag of the first product
-                w[6] = 0u;
-                w[7] = 0u;
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const int buf = (4 * g + c) % NBUF;
-                    w[8 + c] = (is_k ? k_base : v_base) + (uint32_t)buf * (C::CHUNK >> 4);
-                    w[12 + c] = is_hi ? bar_hi(buf) : bar_empty(buf);
-                }
-                // what the batch needs: hi products the four chunks (a weighted sum also the tile's
-                // probabilities and the fold of the previous tile's weighted sum, which the softmax
-                // group does after storing the probabilities); lo products the four conversions
-                if (is_hi) {
+                const Batch64 bt(i, T);
+                const int gs = bt.g % NG;
+                const uint32_t gpar = (uint32_t)(bt.g / NG) & 1u;
+                // hi products need the four chunks (a weighted sum also the tile's probabilities and
+                // the fold of the previous tile's weighted sum, which the softmax group does after
+                // storing the probabilities); lo products the four conversions
+                if (bt.is_hi) {
                     ok = wait_or_abort(bar_gfull(gs), gpar, abort_flag);
-                    if (ok && !is_k)
-                        ok = (t > 0) ? wait_or_abort(bar_ofree, (uint32_t)(t - 1) & 1u, abort_flag)
-                                     : wait_or_abort(bar_pfull(0), 0u, abort_flag);
+                    if (ok && !bt.is_k)
+                        ok = (bt.t > 0) ? wait_or_abort(bar_ofree, (uint32_t)(bt.t - 1) & 1u, abort_flag)
+                                        : wait_or_abort(bar_pfull(0), 0u, abort_flag);
                 } else {
                     ok = wait_or_abort(bar_glo(gs), gpar, abort_flag);
                     // the K_lo products overwrite the K_hi products of the tile: those must have been read
-                    if (ok && is_k && precise) ok = wait_or_abort(bar_shread, (uint32_t)t & 1u, abort_flag);
+                    if (ok && bt.is_k && precise) ok = wait_or_abort(bar_shread, (uint32_t)bt.t & 1u, abort_flag);
                 }
-                for (uint32_t it = 0; ok && *q_taken + C::QN <= i; ++it)       // a free queue slot
-                    if (it >= kWaitLimit || ((it & 255u) == 255u && *abort_flag)) {
-                        if (it >= kWaitLimit) { *abort_flag = 1; raise_status(MOA_STATUS_WAIT_TIMEOUT); }
-                        ok = false;
-                    }
                 if (!ok) break;
-                const uint32_t slot = queue + (uint32_t)(i % C::QN) * 64u;
-                sts_volatile_v4(slot, w[0], w[1], w[2], w[3]);
-                sts_volatile_v4(slot + 16u, w[4], w[5], w[6], w[7]);
-                sts_volatile_v4(slot + 32u, w[8], w[9], w[10], w[11]);
-                sts_volatile_v4(slot + 48u, w[12], w[13], w[14], w[15]);
                 __threadfence_block();
                 *q_ready = i + 1;
             }
         }
     } else if (warp == 3) {
         // ================= MMA issuer (one thread) =================
+        // Everything a batch needs is a function of its number: operand (K or V), tile, group and
+        // with it the ring buffers (a group always occupies the same four), so the sixteen
+        // descriptors of a batch are one run-time base plus compile-time offsets.  Commits: a hi
+        // batch signals after its second and its fourth chunk (the converters of a pair of chunks
+        // wait for the pair), a lo batch after every chunk (the producer refills buffer by buffer:
+        // a group-wise refill starts the loads too late to cover their latency).
         if (lane == 0) {
             const int nbatch = 4 * T;
-            int have = 0;
+            const uint32_t ring_lo = sRing >> 4;
             bool ok = true;
-            uint4 n0, n1, n2, n3;                  // the next batch, fetched ahead
-            bool fetched = false;
             for (int i = 0; ok && i < nbatch; ++i) {
-                if (!fetched) {
-                    for (uint32_t it = 0; have <= i; ++it) {
-                        have = *q_ready;
-                        if (it >= kWaitLimit || ((it & 255u) == 255u && *abort_flag)) {
-                            if (it >= kWaitLimit) { *abort_flag = 1; raise_status(MOA_STATUS_WAIT_TIMEOUT); }
-                            ok = false;
-                            break;
-                        }
+                const Batch64 bt(i, T);
+                const uint32_t d = bt.is_k ? tSP_of(bt.t) : tO;
+                const uint32_t a0 = bt.is_k ? tQ : tSP_of(bt.t);
+                const uint32_t acc0 = (bt.is_hi || (bt.is_k && precise)) ? 0u : 1u;
+                const int slot = bt.g % 3, buf0 = 4 * slot;
+                const uint32_t bar_first = bt.is_hi ? 0u : bar_empty(buf0);     // lo batch: barriers of the four buffers (8 bytes apart)
+                const uint32_t bar_mid = bar_hi(buf0 + 1), bar_end = bar_hi(buf0 + 3);
+                for (uint32_t it = 0; *q_ready <= i; ++it)             // the operands of this batch are complete
+                    if (it >= kWaitLimit || ((it & 255u) == 255u && *abort_flag)) {
+                        if (it >= kWaitLimit) { *abort_flag = 1; raise_status(MOA_STATUS_WAIT_TIMEOUT); }
+                        ok = false;
+                        break;
                     }
-                    if (!ok) break;
-                    __threadfence_block();
-                    const uint32_t slot = queue + (uint32_t)(i % C::QN) * 64u;
-                    n0 = lds_volatile_v4(slot); n1 = lds_volatile_v4(slot + 16u);
-                    n2 = lds_volatile_v4(slot + 32u); n3 = lds_volatile_v4(slot + 48u);
-                    *q_taken = i + 1;
-                }
-                const uint32_t d = n0.x, a0 = n0.y, hiword = n0.z, step = n0.w, idesc = n1.x, acc0 = n1.y;
-                const uint32_t bdesc[4] = {n2.x, n2.y, n2.z, n2.w}, done[4] = {n3.x, n3.y, n3.z, n3.w};
-                fetched = false;
+                if (!ok) break;
+                __threadfence_block();
                 tc::fence_after_sync();
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    if (c == 3 && i + 1 < nbatch) {    // fetch the next batch while this chunk is multiplied
-                        have = *q_ready;
-                        if (have > i + 1) {
-                            __threadfence_block();
-                            const uint32_t slot = queue + (uint32_t)((i + 1) % C::QN) * 64u;
-                            n0 = lds_volatile_v4(slot); n1 = lds_volatile_v4(slot + 16u);
-                            n2 = lds_volatile_v4(slot + 32u); n3 = lds_volatile_v4(slot + 48u);
-                            *q_taken = i + 2;
-                            fetched = true;
-                        }
-                    }
-#pragma unroll
-                    for (uint32_t ks = 0; ks < 4; ++ks)
-                        tc::mma_tf32_ts(d, a0 + 32u * c + 8u * ks, tc::pack64(bdesc[c] + ks * step, hiword), idesc,
-                                        (c == 0 && ks == 0) ? acc0 : 1u);
-                    tc::mma_commit(done[c]);
+                switch ((bt.is_k ? 0 : 3) + slot) {
+                case 0: issue_batch64<true, 0>(d, a0, ring_lo, acc0, bar_first, bar_mid, bar_end); break;
+                case 1: issue_batch64<true, 1>(d, a0, ring_lo, acc0, bar_first, bar_mid, bar_end); break;
+                case 2: issue_batch64<true, 2>(d, a0, ring_lo, acc0, bar_first, bar_mid, bar_end); break;
+                case 3: issue_batch64<false, 0>(d, a0, ring_lo, acc0, bar_first, bar_mid, bar_end); break;
+                case 4: issue_batch64<false, 1>(d, a0, ring_lo, acc0, bar_first, bar_mid, bar_end); break;
+                default: issue_batch64<false, 2>(d, a0, ring_lo, acc0, bar_first, bar_mid, bar_end); break;
                 }
             }
         }
@@ -539,7 +527,7 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
         for (ChunkSeq s(T); ok && !s.done; s.next()) {
             if ((s.seq & 3) != team) continue;
             const int buf = s.seq % NBUF, use = s.seq / NBUF;
-            ok = wait_suspended(bar_hi(buf), (uint32_t)use & 1u, abort_flag);
+            ok = wait_suspended(bar_hi(buf | 1), (uint32_t)use & 1u, abort_flag);    // one commit per pair of chunks
             if (!ok) break;
             float4 *p = reinterpret_cast<float4 *>(smem + C::OFF_RING + (uint32_t)buf * C::CHUNK);
 #pragma unroll
