@@ -46,9 +46,10 @@ L2_BYTES_ASSUMED = 126 * 1024 * 1024
 # a digest of the kernel sources it was captured with; when those files have changed since,
 # the figure is stale and the line reports null instead.
 NCU_TRAFFIC = {
-    "gqa": {"bytes": 1074650112 + 3750144, "sources": ["moa_stream.cuh", "moa_device.cuh"], "digest": ""},
-    "extra_group8_d128": {"bytes": 1075588864 + 4157440, "sources": ["moa_mma.cuh", "moa_device.cuh"], "digest": ""},
-    "mqa_long": {"bytes": 537066496 + 314112, "sources": ["moa_grouped64.cuh", "moa_grouped.cuh", "moa_tc.cuh"], "digest": ""},
+    "gqa": {"bytes": 1074633984 + 427008, "sources": ["moa_stream.cuh", "moa_device.cuh"], "digest": "c2d07a9d9c5d5733"},
+    "extra_group8_d128": {"bytes": 1075583744 + 736768, "sources": ["moa_mma.cuh", "moa_device.cuh"], "digest": "64e296a5cd5f0df2"},
+    "multi_step": {"bytes": 351774720 + 679680, "sources": ["moa_stream.cuh", "moa_device.cuh"], "digest": "c2d07a9d9c5d5733"},
+    "mqa_long": {"bytes": 537104896 + 371200, "sources": ["moa_grouped64.cuh", "moa_grouped.cuh", "moa_tc.cuh"], "digest": "3a2f58bdc1f62840"},
 }
 
 
