@@ -682,7 +682,7 @@ def run_rank(args, side, make_run=None):
 
     l2_note = run.l2_note
     sampler = ClockSampler(local) if on_gpu else None
-    ms, _, launches, clocks, segs = time_steps(run, args.steps, args.warmup, side, sampler, segment=300)
+    ms, _, launches, clocks, segs = time_steps(run, args.steps, args.warmup, side, sampler, segment=min(300, args.steps // 2))
     per_rank = ms
     ms = max_over_ranks(ms)
     per_rank_all = None
@@ -858,7 +858,7 @@ def run_rank(args, side, make_run=None):
                 "config": {"workload": wname, "batch_per_gpu": w.batch, "h_q": w.h_q, "h_kv": w.h_kv,
                            "n": w.n, "d_k": w.d_k, "d_v": w.d_v, "parallelism": par, "step": step_desc, "l2": l2_note},
                 "us_per_step": ms * 1e3, "us_per_step_per_rank": per_rank_all,
-                "us_per_step_first_last_300": ([segs[0] * 1e3, segs[1] * 1e3] if segs else None),
+                "us_per_step_first_last_segment": ({"steps": min(300, args.steps // 2), "first": segs[0] * 1e3, "last": segs[1] * 1e3} if segs else None),
                 "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
                 "roofline": roof, "cpu_baseline": cpu, "parity_max_abs_err_vs_oracle": parity,
                 "other_workloads": others}
