@@ -512,14 +512,16 @@ static cudaError_t launch_grouped64_cfg(const CUtensorMap &mk, const CUtensorMap
         attr_set[dev] = true;
     }
     {
+        // programmatic stream serialisation: the kernel's set-up overlaps the tail-copy kernel
+        // before it, the combine kernel's launch overlaps this kernel's end
         TimedLaunch t(st);
-        grouped64_decode_kernel<PRECISE><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(mk, mv, mkt, mvt, ga);
+        launch_dependent(grouped64_decode_kernel<PRECISE>, grid, C::THREADS, C::SMEM_BYTES, st, mk, mv, mkt, mvt, ga);
     }
     count_launch();
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess || !combine) return e;
     const long long warps = (long long)ga.batch * ga.h_q;
-    grouped_combine_kernel<64><<<(int)warps, 128, 0, st>>>(ga);
+    launch_dependent(grouped_combine_kernel<64>, (int)warps, 128, 0, st, ga);
     count_launch();
     return cudaGetLastError();
 }

@@ -151,6 +151,9 @@ __device__ __forceinline__ FlatShare flat_share(const GroupedArgs &a, int grid, 
 __global__ void __launch_bounds__(256) grouped_tail_kernel(const GroupedArgs a, const float *K, const float *V, float *Kw,
                                                            float *Vw, const float *k_new, const float *v_new)
 {
+    // The main kernel that follows may be scheduled while this one runs (programmatic dependent
+    // launch): it only waits for this grid before it fetches the tiles copied here.
+    launch_dependents();
     const int unit = blockIdx.x >> 3, part = blockIdx.x & 7, b = unit / a.h_kv_stored;
     const int len = grouped_len(a, b);
     if (len == 0) {
@@ -731,6 +734,7 @@ __global__ void __launch_bounds__(128) grouped_combine_kernel(const GroupedArgs 
     constexpr int PS = 132;
     __shared__ float4 s_acc[4][32], s_accc[4][32];
     __shared__ float s_l[4], s_lc[4];
+    grid_dependency_wait();                        // the partials of the main kernel (a no-op for an ordinary launch)
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const long long wid = blockIdx.x;
     const int b = (int)(wid / a.h_q), gq = (int)(wid % a.h_q);

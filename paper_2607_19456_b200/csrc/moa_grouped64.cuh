@@ -235,6 +235,7 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
     // The first ring-full of chunks needs nothing but the barriers: the producer starts those
     // loads now, so that they travel while the query operand is being built.
     ChunkSeq pseq(T);                              // the producer's position (warp 0, lane 0)
+    bool tail_ready = false;                       // the grid that wrote the tail copies is complete
     auto issue_load = [&](const ChunkSeq &s) {
         const int buf = s.seq % NBUF;
         const uint32_t dst = sRing + (uint32_t)buf * C::CHUNK;
@@ -242,6 +243,9 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
         mbar_expect_tx(fb, C::CHUNK);
         const bool tail = (s.t == tail_t);
         const int row = tail ? 0 : row_base + s.t * C::TILE;
+        // Launched with programmatic stream serialisation, this kernel may have started while the
+        // tail-copy kernel before it was still running; nothing else it reads comes from there.
+        if (tail && !tail_ready) { grid_dependency_wait(); tail_ready = true; }
         if (s.is_k) {
             tc::tma_load_3d(dst, tail ? &tmapKt : &tmapK, 32 * s.c, row, unit, fb);
         } else {
@@ -550,6 +554,7 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
 
     tc::fence_before_sync();
     __syncthreads();
+    launch_dependents();                           // the combine kernel may be scheduled; it waits for this grid itself
     if (warp == 3) tc::tmem_dealloc(tmem, 512);
 }
 
