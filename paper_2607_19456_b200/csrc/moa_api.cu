@@ -496,7 +496,6 @@ static cudaError_t launch_grouped_cfg(const CUtensorMap &mk, const CUtensorMap &
 
 // Groups of 64 heads with Q and P in tensor memory; same arguments and partial format as
 // the shared-memory-operand kernel, so the combine kernel is shared.
-template <bool PRECISE>
 static cudaError_t launch_grouped64_cfg(const CUtensorMap &mk, const CUtensorMap &mv, const CUtensorMap &mkt,
                                         const CUtensorMap &mvt, const GroupedArgs &ga, int grid, cudaStream_t st,
                                         bool combine = true)
@@ -506,7 +505,7 @@ static cudaError_t launch_grouped64_cfg(const CUtensorMap &mk, const CUtensorMap
     int dev = 0;
     cudaGetDevice(&dev);
     if (!attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(grouped64_decode_kernel<PRECISE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(grouped64_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)C::SMEM_BYTES);
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
@@ -515,7 +514,7 @@ static cudaError_t launch_grouped64_cfg(const CUtensorMap &mk, const CUtensorMap
         // programmatic stream serialisation: the kernel's set-up overlaps the tail-copy kernel
         // before it, the combine kernel's launch overlaps this kernel's end
         TimedLaunch t(st);
-        launch_dependent(grouped64_decode_kernel<PRECISE>, grid, C::THREADS, C::SMEM_BYTES, st, mk, mv, mkt, mvt, ga);
+        launch_dependent(grouped64_decode_kernel, grid, C::THREADS, C::SMEM_BYTES, st, mk, mv, mkt, mvt, ga);
     }
     count_launch();
     cudaError_t e = cudaGetLastError();
@@ -536,7 +535,7 @@ static cudaError_t launch_grouped_cfg(const CUtensorMap &mk, const CUtensorMap &
 static cudaError_t launch_grouped64(const CUtensorMap &mk, const CUtensorMap &mv, const CUtensorMap &mkt,
                                     const CUtensorMap &mvt, const GroupedArgs &ga, int grid, cudaStream_t st)
 {
-    return launch_grouped64_cfg<true>(mk, mv, mkt, mvt, ga, grid, st);
+    return launch_grouped64_cfg(mk, mv, mkt, mvt, ga, grid, st);
 }
 
 static cudaError_t launch_generic(const DecodeArgs &a, cudaStream_t st)

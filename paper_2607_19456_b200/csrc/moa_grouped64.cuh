@@ -1,5 +1,5 @@
-// moa_grouped64.cuh -- tensor-core decode kernel for groups of 64 query heads per K/V head
-// (MQA), with the small operands (Q, P) resident in tensor memory.
+// moa_grouped64.cuh -- tensor-core decode kernel for groups of up to 64 query heads per K/V head
+// (MQA and large GQA groups), with the small operands (Q, P) resident in tensor memory.
 //
 // Steps I and III of Algorithm 1 (eqs. (1),(3)) per tile of 128 cached rows, heads on the
 // M axis:
@@ -20,27 +20,28 @@
 // lane, so the two parts of a head meet by one shuffle inside a warp.
 //
 // Tensor memory (512 columns): Q (128), two score/probability regions (128 each; the
-// probabilities of a tile overwrite its scores), O (128).  The tensor core accumulates with
-// truncation, so chains are kept short: the weighted sum of every tile starts from zero and is
-// folded into fp32 running values held in registers (online softmax, eq. (2) with a running
-// maximum per head).  The scores of a tile are one chain of 32 steps in the variant for long
-// caches and two chains of 16 (K_hi and K_lo products added in fp32 by the softmax group) in
-// the PRECISE variant, see the note at `precise` below.
+// probabilities of a tile overwrite its scores), O (128).
 //
-// A thread that issues tcgen05.mma cannot look at a barrier without draining the tensor pipe
-// (measured: one shared-memory read between two products costs ~170 cycles of tensor time),
-// so the issuer asks once per batch, on barriers that collect a whole batch: all four chunks
-// of a group landed -> 16 hi products; the first two conversions done -> 8 lo products; the
-// other two -> 8 more.  Nothing the
-// softmax group does is on the tensor core's critical path: while it works on tile t the
-// tensor core multiplies tile t+1's K chunks and tile t-1's V chunks.
+// Accuracy: the tensor core accumulates with truncation, and what a truncation costs is set by
+// the size of the accumulator, so small terms are never added on top of large ones.  The K_hi
+// products of a tile are read out of its region by the softmax group before the K_lo products
+// start the region afresh, and the two are added in fp32 (two chains of 16 steps per score); the
+// weighted sum of every tile starts from zero and is folded into fp32 running values held in
+// registers (online softmax, eq. (2) with a running maximum per head).
+//
+// A thread that issues tcgen05.mma cannot look at a barrier without draining the tensor pipe,
+// so a scheduler thread does the waiting and releases batches of 16 products by number (all four
+// chunks of a group landed -> hi products; their four conversions done -> lo products); the
+// issuing thread derives everything else from that number: a chunk group always occupies the
+// same four ring buffers, so the descriptors are a run-time base plus compile-time offsets.
 //
 // Roles (768 threads): warp 0 TMA producer, warp 3 MMA issuer (and owner of the tensor
-// memory allocation), warp 22 batch scheduler, warps 4-19 softmax (warp w: lane quadrant w % 4, columns 32 * ((w-4)/4)
-// .. +31 of a 128-column region), warps 1, 2, 20, 21 turn chunks into their lo parts, warp 23
-// idles.  After the set-up the softmax warpgroups take registers from the others
-// (setmaxnreg): they hold the running weighted sum and a tile's scores at once.  Every
-// hand-off is an mbarrier; every wait is bounded.
+// memory allocation), warp 22 batch scheduler, warps 4-19 softmax (warp w: lane quadrant w % 4,
+// columns 32 * ((w-4)/4) .. +31 of a 128-column region), warps 1, 2, 20, 21 turn chunks into
+// their lo parts (none of them on the issuer's scheduler quarter), warp 23 idles.  After the
+// set-up the softmax warpgroups take registers from the others (setmaxnreg): they hold the
+// running weighted sum and a tile's K_hi products at once.  Every hand-off is an mbarrier;
+// every wait is bounded.
 #pragma once
 
 #include "moa_grouped.cuh"
@@ -138,7 +139,6 @@ __device__ __forceinline__ void issue_batch64(uint32_t d, uint32_t a0, uint32_t 
     if (bar_first == 0u) tc::mma_commit(bar_end);
 }
 
-template <bool PRECISE>
 __global__ void __launch_bounds__(Grouped64Cfg::THREADS, 1)
 grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_constant__ CUtensorMap tmapV,
                         const __grid_constant__ CUtensorMap tmapKt, const __grid_constant__ CUtensorMap tmapVt,
@@ -201,17 +201,6 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
     if (T <= 0) return;                            // an empty split (uniform for the CTA)
     const int tail_t = (a.tailK != nullptr) ? tiles_total - 1 - tile0 : -1;
     const int row_base = tile0 * C::TILE;
-    // The tensor core accumulates with truncation, and an error of one unit in the last place of
-    // a score costs the same whatever the size of the term that was added.  With the K_lo
-    // products on top of the K_hi products a score is a chain of 32 steps instead of 16, which
-    // doubles its error: measured against the fp64 oracle 5.1e-6 (max) at 128 rows, 2.2e-6 at
-    // 1000, 1.1e-6 at 4000, 2.7e-7 at 16000 -- the error of an output averages out over the rows.
-    // The PRECISE variant therefore keeps the two chains apart (the softmax group reads the K_hi
-    // products out before the K_lo products start the region afresh: 2.9e-6 at 128 rows), at
-    // the price of one more hand-over per tile; the host uses it for caches of fewer than 4096
-    // rows and for ragged caches, whose lengths it does not know.
-    constexpr bool precise = PRECISE;
-
     // ---- set-up --------------------------------------------------------------------------
     if (tid == 0) {
         for (int i = 0; i < NBUF; ++i) { mbar_init(bar_hi(i), 1); mbar_init(bar_empty(i), 1); }
@@ -328,7 +317,7 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
                 } else {
                     ok = wait_or_abort(bar_glo(gs), gpar, abort_flag);
                     // the K_lo products overwrite the K_hi products of the tile: those must have been read
-                    if (ok && bt.is_k && precise) ok = wait_or_abort(bar_shread, (uint32_t)bt.t & 1u, abort_flag);
+                    if (ok && bt.is_k) ok = wait_or_abort(bar_shread, (uint32_t)bt.t & 1u, abort_flag);
                 }
                 if (!ok) break;
                 __threadfence_block();
@@ -351,7 +340,7 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
                 const Batch64 bt(i, T);
                 const uint32_t d = bt.is_k ? tSP_of(bt.t) : tO;
                 const uint32_t a0 = bt.is_k ? tQ : tSP_of(bt.t);
-                const uint32_t acc0 = (bt.is_hi || (bt.is_k && precise)) ? 0u : 1u;
+                const uint32_t acc0 = (bt.is_hi || bt.is_k) ? 0u : 1u;    // only the V_lo products continue an accumulation
                 const int slot = bt.g % 3, buf0 = 4 * slot;
                 const uint32_t bar_first = bt.is_hi ? 0u : bar_empty(buf0);     // lo batch: barriers of the four buffers (8 bytes apart)
                 const uint32_t bar_mid = bar_hi(buf0 + 1), bar_end = bar_hi(buf0 + 3);
@@ -400,7 +389,7 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
             // terms of its hi and of its lo query part; they share the work: the hi lane takes
             // columns 0..15, the lo lane columns 16..31, each gets the other lane's terms for its
             // columns by shuffle and hands back the part of the probabilities the other lane stores.
-            if constexpr (PRECISE) {
+            {
                 // the K_hi products of the tile are read out before the K_lo products start the
                 // region afresh; the two are added here in fp32
                 uint32_t xa[32];
@@ -427,18 +416,6 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
                 for (int i = 0; i < 16; ++i) {       // each lane sends what the other needs
                     const float other = __shfl_xor_sync(0xffffffffu, __uint_as_float(is_lo ? xa[i] : xa[16 + i]), 16);
                     sc[i] = __uint_as_float(is_lo ? xa[16 + i] : xa[i]) + other;
-                }
-            } else {
-                ok = ok && wait_suspended(bar_group_done(group_k(t)), par_group_done(group_k(t)), abort_flag);
-                if (named_or(1 + qd, 128, !ok)) { ok = false; break; }    // the four warps of a quadrant leave together
-                tc::fence_after_sync();
-                uint32_t x[32];
-                tc::tmem_ld32(tSP, x);
-                tc::tmem_ld_wait();
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {       // each lane sends what the other needs
-                    const float other = __shfl_xor_sync(0xffffffffu, __uint_as_float(is_lo ? x[i] : x[16 + i]), 16);
-                    sc[i] = __uint_as_float(is_lo ? x[16 + i] : x[i]) + other;
                 }
             }
             float vmax = -INFINITY;
