@@ -167,7 +167,13 @@ EXTRA_WORKLOADS = {
     "extra_group8_d64": mi.Workload("extra_group8_d64", 1102, 16, 64, 8, 16384, 64, 64),
     "extra_group16_d128": mi.Workload("extra_group16_d128", 1103, 16, 128, 8, 8192, 128, 128),
     "extra_mha_d32": mi.Workload("extra_mha_d32", 1104, 64, 32, 32, 4096, 32, 32),
+    # 32 query heads on one K/V head at d = 64 (the shape of the paper's GQA/MQA traffic table), long cache
+    "extra_mqa_d64": mi.Workload("extra_mqa_d64", 1105, 8, 32, 1, 131072, 64, 64),
 }
+# Workloads whose step is issued as two calls, moa_kv_append + moa_decode_attn: the tensor-core
+# path for rows of 64 features needs a dense cache of known length, which the fused call (lengths
+# on the device) cannot promise.
+TWO_CALL_STEP = {"extra_mqa_d64"}
 
 
 class DenseRun:
@@ -222,6 +228,7 @@ class DenseRun:
         self.wsbuf = torch.empty(self.ws_bytes, dtype=torch.uint8, device=device)
         self.wsptr = self.wsbuf.data_ptr()
         self.stream = torch.cuda.current_stream().cuda_stream
+        self.two_call = w.name in TWO_CALL_STEP
         self.l2_note = "rotating over %d buffer sets of %.0f MB (%.0f MB in total; L2 is 126 MB)" % (S, one / 1e6, S * one / 1e6)
 
     def step(self):
@@ -229,6 +236,10 @@ class DenseRun:
         q, K, V, out = self.ptrs[self.i % self.nsets]
         kn, vn, pos = self.aux
         self.i += 1
+        if self.two_call:
+            m.moa_kv_append(K, V, kn, vn, pos, w.batch, w.h_kv, w.n, w.d_k, w.d_v, self.stream)
+            m.moa_decode_attn(q, K, V, out, w.batch, w.h_q, w.h_kv, w.n, w.d_k, w.d_v, w.scale, self.stream)
+            return
         m.moa_append_decode(q, K, V, kn, vn, out, pos, w.batch, w.h_q, w.h_kv, w.n, w.d_k, w.d_v, w.scale,
                             self.wsptr, self.ws_bytes, self.stream)
 

@@ -555,6 +555,80 @@ static cudaError_t launch_generic(const DecodeArgs &a, cudaStream_t st)
     return cudaGetLastError();
 }
 
+// Groups of 17..32 or of exactly 64 heads at d = 64 on a dense cache with an even number of rows:
+// the 64-lane tensor-core kernel in pair mode.  Two consecutive cached rows of 64 features are
+// read as one row of 128; every head takes two pseudo-heads whose query is zero in one half, so
+// one of them sees the even and the other the odd cached rows; a combine kernel of its own puts
+// the halves together.  64 heads run as two virtual kv heads of 32 (the K/V tiles are read twice,
+// the second time from L2).
+struct PairPlan {
+    bool ok = false;
+    int share = 1, gs = 0, splits = 1, tiles_per_split = 1;
+    size_t ws_bytes = 0;
+};
+static PairPlan plan_grouped_pair(const DeviceState &s, int batch, int h_q, int h_kv, int n, int d_k, int d_v)
+{
+    PairPlan p;
+    const int g_s = h_q / h_kv;
+    if (d_k != 64 || d_v != 64 || (n & 1) || n < 2) return p;
+    if (!((g_s > 16 && g_s <= 32) || g_s == 64)) return p;
+    if (g_grouped_operands != 0 || (g_force_path != 0 && g_force_path != MOA_PATH_GROUPED)) return p;
+    p.share = g_s == 64 ? 2 : 1;
+    p.gs = g_s == 64 ? 32 : g_s;
+    const long long vunits = (long long)batch * h_kv * p.share;
+    if (vunits > 0x7fffffffLL / 256) return p;
+    const int tiles = (n / 2 + 127) / 128;
+    long long splits = vunits >= s.sm_count ? 1 : s.sm_count / vunits;
+    if (splits > tiles) splits = tiles;
+    p.splits = (int)splits;
+    p.tiles_per_split = (tiles + p.splits - 1) / p.splits;
+    p.ws_bytes = (size_t)vunits * p.splits * 64 * 132 * sizeof(float);
+    p.ok = true;
+    return p;
+}
+
+static cudaError_t launch_grouped_pair(const PairPlan &pp, const float *q, const float *K, const float *V, float *out,
+                                       float *ws, int batch, int h_q, int h_kv, int n, float scale, cudaStream_t st)
+{
+    const long long units = (long long)batch * h_kv;
+    CUtensorMap mk, mv;
+    if (!make_cache_map(&mk, K, units, n / 2, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_cache_map(&mv, V, units, n / 2, 32, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B))
+        return cudaErrorInvalidValue;
+    GroupedArgs ga;
+    ga.q = q; ga.out = out; ga.ws = ws;
+    ga.batch = batch; ga.h_q = h_q; ga.h_kv = h_kv * pp.share; ga.n = n / 2;
+    ga.g_s = pp.gs; ga.h_kv_stored = h_kv; ga.share = pp.share;
+    ga.splits = pp.splits; ga.tiles_per_split = pp.tiles_per_split;
+    ga.qscale = scale * kLog2e;
+    ga.partial_out = nullptr; ga.seq_lens = nullptr; ga.len_bias = 0;
+    ga.tailK = nullptr; ga.tailV = nullptr; ga.flat = 0;
+    ga.len_lo = 0; ga.len_hi = 0x7fffffff;
+    ga.pair = 1;
+    using C = Grouped64Cfg;
+    static bool attr_set[kMaxDevices] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (!attr_set[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(grouped64_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)C::SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        attr_set[dev] = true;
+    }
+    {
+        TimedLaunch t(st);
+        launch_dependent(grouped64_decode_kernel, (int)(units * pp.share * pp.splits), C::THREADS, C::SMEM_BYTES, st,
+                         mk, mv, mk, mv, ga);
+    }
+    count_launch();
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const long long rows = (long long)batch * h_q;
+    launch_dependent(grouped_pair_combine_kernel, (int)((rows + 3) / 4), 128, 0, st, ga);
+    count_launch();
+    return cudaGetLastError();
+}
+
 // Shared implementation of the decode entry points.  `ws` may be null when the chosen
 // path needs none.
 struct FusedStep {                 // extra work folded into the streaming launch
@@ -592,6 +666,23 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
         if (!make_rows_map(&probe, K, plan.Dk, n_max, h_kv, batch, lay.k) ||
             !make_rows_map(&probe, V, plan.D, n_max, h_kv, batch, lay.v))
             fast_ok = false;
+    }
+    if (fast_ok && allow_grouped && lay.dense && seq_lens == nullptr && fused == nullptr && partial_out == nullptr) {
+        const PairPlan pp = plan_grouped_pair(*dev, batch, h_q, h_kv, n_max, d_k, d_v);
+        if (pp.ok && (library_ws || (ws && ws_bytes >= pp.ws_bytes))) {
+            if (library_ws) {
+                if (dev->ws_bytes < pp.ws_bytes) {
+                    if (dev->ws) { cudaDeviceSynchronize(); cudaFree(dev->ws); dev->ws = nullptr; dev->ws_bytes = 0; }
+                    if (cudaMalloc(&dev->ws, pp.ws_bytes) != cudaSuccess) { cudaGetLastError(); return MOA_ERR_CUDA; }
+                    dev->ws_bytes = pp.ws_bytes;
+                }
+                ws = dev->ws;
+            } else if (!aligned(ws, 256)) return MOA_ERR_ALIGN;
+            if (launch_grouped_pair(pp, q, K, V, out, static_cast<float *>(ws), batch, h_q, h_kv, n_max, scale, st) != cudaSuccess)
+                return MOA_ERR_CUDA;
+            g_last_path = MOA_PATH_GROUPED;
+            return MOA_OK;
+        }
     }
     int path = fast_ok ? (plan.mma ? MOA_PATH_MMA : MOA_PATH_STREAM) : MOA_PATH_GENERIC;
     // Large head groups go to the tcgen05 kernel; ragged caches and the fused step need scratch
@@ -656,6 +747,7 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
         ga.tailK = nullptr; ga.tailV = nullptr;
         ga.flat = 0;
         ga.len_lo = 0; ga.len_hi = 0x7fffffff;
+        ga.pair = 0;
         CUtensorMap mkt = mk, mvt = mv;
         if (ragged) {
             // the last, partly filled tile of every unit, zero-padded (and the appended row of
@@ -846,6 +938,8 @@ size_t moa_workspace_bytes(int batch, int h_q, int h_kv, int n_max, int d_k, int
     if (dev != nullptr || current_device(&dev) == MOA_OK) {
         const GroupedPlan gp = plan_grouped(*dev, batch, h_q, h_kv, n_max, d_k, d_v);
         if (gp.ok && gp.ws_ragged() > need) need = gp.ws_ragged();
+        const PairPlan pp = plan_grouped_pair(*dev, batch, h_q, h_kv, n_max, d_k, d_v);
+        if (pp.ok && pp.ws_bytes > need) need = pp.ws_bytes;
     }
     return (need + 255) / 256 * 256;
 }

@@ -87,6 +87,8 @@ struct GroupedArgs {
                                // to their lengths (see flat_share)
     int len_lo, len_hi;        // this launch handles the units with len_lo <= length < len_hi (a ragged batch may be
                                // served by two launches of different kernels; slots and splits are the same for both)
+    int pair;                  // 64-lane kernel on rows of 64 features: two consecutive cached rows form one row of
+                               // 128 (n counts such pairs), a head takes two pseudo-heads (even rows, odd rows); dense only
 };
 
 // Rows of sequence b as this kernel family sees them; 0 for an out-of-range length.
@@ -797,6 +799,42 @@ __global__ void __launch_bounds__(128) grouped_combine_kernel(const GroupedArgs 
     const float inv = 1.0f / L;
     *reinterpret_cast<float4 *>(a.out + ((size_t)b * a.h_q + gq) * 128 + lane * 4) =
         make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+}
+
+// Merge for the 64-lane kernel in pair mode (rows of 64 features): a head's result is spread over
+// two pseudo-heads, 2j (even cached rows: features 0..63 of its 128-wide partial are meaningful)
+// and 2j+1 (odd rows: features 64..127), each with a maximum and a sum of its own, times the
+// splits of the unit.  One warp per (batch, query head), partials in (split, parity) order,
+// compensated sums.
+__global__ void __launch_bounds__(128) grouped_pair_combine_kernel(const GroupedArgs a)
+{
+    constexpr int PS = 132, GH = 64;
+    grid_dependency_wait();
+    const int lane = threadIdx.x & 31;
+    const long long wid = (long long)blockIdx.x * 4 + (threadIdx.x >> 5);
+    if (wid >= (long long)a.batch * a.h_q) return;
+    const int b = (int)(wid / a.h_q), gq = (int)(wid % a.h_q);
+    const int vh = gq / a.g_s, j = gq % a.g_s;     // virtual kv head (a.h_kv of them per batch item), head inside it
+    const int tiles_total = (a.n + 127) / 128;
+    const int used = (tiles_total + a.tiles_per_split - 1) / a.tiles_per_split;     // non-empty splits
+    const float *base = a.ws + ((((size_t)b * a.h_kv + vh) * a.splits) * GH + 2 * j) * PS;
+    const size_t stride = (size_t)GH * PS;
+    float M = -INFINITY;
+    for (int i = lane; i < 2 * used; i += 32) M = fmaxf(M, base[(size_t)(i >> 1) * stride + (size_t)(i & 1) * PS + 128]);
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
+    float2 acc = make_float2(0.f, 0.f), accc = acc;
+    float L = 0.f, Lc = 0.f;
+    for (int i = 0; i < 2 * used; ++i) {
+        const float *row = base + (size_t)(i >> 1) * stride + (size_t)(i & 1) * PS;
+        const float f = exp2_diff(row[128], M);
+        comp_fma(L, Lc, row[129], f);
+        const float2 t = *reinterpret_cast<const float2 *>(row + 64 * (i & 1) + 2 * lane);
+        comp_fma(acc.x, accc.x, t.x, f);
+        comp_fma(acc.y, accc.y, t.y, f);
+    }
+    const float inv = 1.0f / L;
+    *reinterpret_cast<float2 *>(a.out + ((size_t)b * a.h_q + gq) * 64 + 2 * lane) = make_float2(acc.x * inv, acc.y * inv);
 }
 
 }  // namespace moa

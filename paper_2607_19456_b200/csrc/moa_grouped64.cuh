@@ -189,8 +189,10 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
         if (s_share[0] < 0) return;
         sunit = s_share[0]; split = (int)blockIdx.x - s_share[1]; splits_u = s_share[2];
     }
-    const int b = sunit / a.h_kv_stored, h = sunit % a.h_kv_stored;
-    const int unit = sunit;                                         // tensor-map coordinate
+    // pair mode: `sunit` counts virtual kv heads (a.share per stored one, 32 query heads each)
+    const int unit = a.pair ? sunit / a.share : sunit;              // tensor-map coordinate: stored (batch, kv head)
+    const int b = a.pair ? sunit / a.h_kv : sunit / a.h_kv_stored;
+    const int h = a.pair ? sunit % a.h_kv : sunit % a.h_kv_stored;  // (virtual) kv head inside the batch item
     const int len_b = grouped_len(a, b);           // 0: out-of-range length, the item is skipped
     if (len_b < a.len_lo || len_b >= a.len_hi) return;   // another launch's unit (uniform for the CTA)
     const int tiles_total = (len_b + C::TILE - 1) / C::TILE;
@@ -259,11 +261,17 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
     if (is_soft) {
         // Q operand: this lane's part (hi or lo) of (scale * log2 e) * q[head], columns = features
         // (a group of fewer than 64 heads is padded: the lanes of the missing heads hold zeros)
-        const float *qb = a.q + ((size_t)b * a.h_q + (size_t)h * a.g_s + head) * 128 + col0;
+        // Pair mode (rows of 64 features, two cached rows per 128-wide row): pseudo-head 2j holds
+        // q of head j in features 0..63 and zeros in 64..127 (it sees the even cached rows),
+        // pseudo-head 2j+1 the other way round.
+        const int qhead = a.pair ? head >> 1 : head;
+        const bool has_q = qhead < a.g_s && (!a.pair || (sub >> 1) == (head & 1));
+        const float *qb = a.pair ? a.q + ((size_t)b * a.h_q + (size_t)h * a.g_s + qhead) * 64 + 32 * (sub & 1)
+                                 : a.q + ((size_t)b * a.h_q + (size_t)h * a.g_s + head) * 128 + col0;
         uint32_t v[32];
 #pragma unroll
         for (int i = 0; i < 32; i += 4) {
-            const float4 x4 = head < a.g_s ? *reinterpret_cast<const float4 *>(qb + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+            const float4 x4 = has_q ? *reinterpret_cast<const float4 *>(qb + i) : make_float4(0.f, 0.f, 0.f, 0.f);
             const float xs[4] = {x4.x * a.qscale, x4.y * a.qscale, x4.z * a.qscale, x4.w * a.qscale};
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
@@ -478,6 +486,7 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
             const float l_pair = l_run + __shfl_xor_sync(0xffffffffu, l_run, 16);   // each lane summed 16 of the 32 columns
             if (!is_lo) lx[sub * 64 + head] = l_pair;
             named_sync(1 + qd, 128);
+            const bool qhead_ok = (a.pair ? head >> 1 : head) < a.g_s;
             float *slot = (a.flat ? a.ws + ((size_t)blockIdx.x * GH) * PS
                                   : a.ws + ((((size_t)b * a.h_kv + h) * a.splits + split) * GH) * PS) + (size_t)head * PS;
 #pragma unroll
@@ -487,9 +496,9 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
                 v.y = Om[i + 1] + __shfl_xor_sync(0xffffffffu, Om[i + 1], 16);
                 v.z = Om[i + 2] + __shfl_xor_sync(0xffffffffu, Om[i + 2], 16);
                 v.w = Om[i + 3] + __shfl_xor_sync(0xffffffffu, Om[i + 3], 16);
-                if (!is_lo && head < a.g_s) *reinterpret_cast<float4 *>(slot + col0 + i) = v;
+                if (!is_lo && qhead_ok) *reinterpret_cast<float4 *>(slot + col0 + i) = v;
             }
-            if (sub == 0 && !is_lo && head < a.g_s) {
+            if (sub == 0 && !is_lo && qhead_ok) {
                 slot[128] = m_run;
                 slot[129] = (lx[head] + lx[64 + head]) + (lx[128 + head] + lx[192 + head]);
             }

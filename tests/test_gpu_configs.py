@@ -24,6 +24,8 @@ def run_dense_on_gpu(w):
     want = moa.PATH_STREAM
     if 17 <= w.group <= 64 and w.d_k == 128:
         want = moa.PATH_GROUPED
+    elif (17 <= w.group <= 32 or w.group == 64) and w.d_k == 64 and w.n % 2 == 0:
+        want = moa.PATH_GROUPED              # rows of 64 features, taken in pairs
     elif w.group % 8 == 0 and w.d_k >= 64:
         want = moa.PATH_MMA
     assert moa.moa_last_path() == want
@@ -67,7 +69,7 @@ def test_dense_configs_full_size_sampled(name, count):
 
 
 @pytest.mark.parametrize("name,count", [("extra_group8_d128", 6), ("extra_group8_d64", 6), ("extra_group16_d128", 6),
-                                        ("extra_mha_d32", 12)])
+                                        ("extra_mha_d32", 12), ("extra_mqa_d64", 2)])
 def test_extra_bench_shapes_full_size_sampled(name, count):
     # the timing-only shapes of bench.py (warp-MMA kernel at 8 and 16 heads per row, d = 32)
     import bench

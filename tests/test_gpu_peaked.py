@@ -32,6 +32,8 @@ FAMILIES = {
     "mma_g16_d128": (32, 2, 128, moa.PATH_AUTO, 0, moa.PATH_MMA, False),
     "tcgen05_tmem_g64": (64, 1, 128, moa.PATH_AUTO, 0, moa.PATH_GROUPED, True),
     "tcgen05_tmem_g48": (48, 1, 128, moa.PATH_AUTO, 0, moa.PATH_GROUPED, True),
+    "tcgen05_pair_g32_d64": (32, 1, 64, moa.PATH_AUTO, 0, moa.PATH_GROUPED, True),
+    "tcgen05_pair_g64_d64": (64, 1, 64, moa.PATH_AUTO, 0, moa.PATH_GROUPED, True),
     "tcgen05_smem_g64": (64, 1, 128, moa.PATH_GROUPED, 1, moa.PATH_GROUPED, True),
     "tcgen05_smem_g32": (32, 1, 128, moa.PATH_GROUPED, 1, moa.PATH_GROUPED, True),
 }
