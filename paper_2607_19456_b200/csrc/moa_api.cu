@@ -603,7 +603,6 @@ static cudaError_t launch_grouped_pair(const PairPlan &pp, const float *q, const
     ga.qscale = scale * kLog2e;
     ga.partial_out = nullptr; ga.seq_lens = nullptr; ga.len_bias = 0;
     ga.tailK = nullptr; ga.tailV = nullptr; ga.flat = 0;
-    ga.len_lo = 0; ga.len_hi = 0x7fffffff;
     ga.pair = 1;
     using C = Grouped64Cfg;
     static bool attr_set[kMaxDevices] = {};
@@ -746,8 +745,7 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
         ga.seq_lens = seq_lens; ga.len_bias = len_bias;
         ga.tailK = nullptr; ga.tailV = nullptr;
         ga.flat = 0;
-        ga.len_lo = 0; ga.len_hi = 0x7fffffff;
-        ga.pair = 0;
+            ga.pair = 0;
         CUtensorMap mkt = mk, mvt = mv;
         if (ragged) {
             // the last, partly filled tile of every unit, zero-padded (and the appended row of

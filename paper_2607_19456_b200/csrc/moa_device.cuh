@@ -113,6 +113,39 @@ __device__ __forceinline__ float exp2_diff(float a, float b)
     return (a == -INFINITY) ? 0.0f : fast_exp2(a - b);
 }
 
+// ---- packed single precision (two fp32 values per instruction, sm_100) --------------------
+// The role warps of the tensor-core kernel are bound by instruction issue; additions,
+// subtractions and fused multiply-adds on pairs of floats halve those instructions.  Same
+// rounding (to nearest) as the scalar instructions, so results do not change.
+__device__ __forceinline__ uint64_t pack2(uint32_t lo, uint32_t hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, uint32_t &lo, uint32_t &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b)
+{
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b)
+{
+    uint64_t r;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+
 // ---- compensated accumulation for the merges -------------------------------------------
 // A merge adds up to a thousand partial triples.  When the softmax mass sits on a few rows,
 // one partial is of order 1 and the rest are tiny, and every plain addition would round at

@@ -85,8 +85,6 @@ struct GroupedArgs {
     float *tailK, *tailV;      // [stored units][128][128]: zero-padded copy of every unit's last tile, or nullptr
     int flat;                  // 0, or the grid size: ragged caches, CTAs are dealt to the units in proportion
                                // to their lengths (see flat_share)
-    int len_lo, len_hi;        // this launch handles the units with len_lo <= length < len_hi (a ragged batch may be
-                               // served by two launches of different kernels; slots and splits are the same for both)
     int pair;                  // 64-lane kernel on rows of 64 features: two consecutive cached rows form one row of
                                // 128 (n counts such pairs), a head takes two pseudo-heads (even rows, odd rows); dense only
 };
@@ -313,7 +311,6 @@ grouped_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_co
     const int b = sunit / a.h_kv_stored, h = (sunit % a.h_kv_stored) * a.share + sub;   // virtual head
     const int unit = sunit;                                         // tensor-map coordinate
     const int len_b = grouped_len(a, b);           // 0: out-of-range length, the item is skipped
-    if (len_b < a.len_lo || len_b >= a.len_hi) return;   // another launch's unit (uniform for the CTA)
     const int tiles_total = (len_b + C::TILE - 1) / C::TILE;
     const int tiles_per_split = a.seq_lens ? (tiles_total + splits_u - 1) / splits_u : a.tiles_per_split;
     const int tile0 = split * tiles_per_split;

@@ -194,7 +194,6 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
     const int b = a.pair ? sunit / a.h_kv : sunit / a.h_kv_stored;
     const int h = a.pair ? sunit % a.h_kv : sunit % a.h_kv_stored;  // (virtual) kv head inside the batch item
     const int len_b = grouped_len(a, b);           // 0: out-of-range length, the item is skipped
-    if (len_b < a.len_lo || len_b >= a.len_hi) return;   // another launch's unit (uniform for the CTA)
     const int tiles_total = (len_b + C::TILE - 1) / C::TILE;
     const int tiles_per_split = a.seq_lens ? (tiles_total + splits_u - 1) / splits_u : a.tiles_per_split;
     const int tile0 = split * tiles_per_split;
@@ -374,9 +373,9 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
     } else if (is_soft) {
         // ================= softmax group: thread = (lane of the stacked operand, 32 columns) ==========
         asm volatile("setmaxnreg.inc.sync.aligned.u32 96;");
-        float Om[32];                              // running weighted sum: this lane's part, features col0..col0+31
+        uint64_t Om[16];                           // running weighted sum: this lane's part, features col0..col0+31, in pairs
 #pragma unroll
-        for (int i = 0; i < 32; ++i) Om[i] = 0.f;
+        for (int i = 0; i < 16; ++i) Om[i] = 0ull;
         float m_run = -INFINITY, l_run = 0.f, alpha_prev = 0.f;
         bool ok = true;
         auto fold = [&](float alpha) {             // Om = alpha * Om + (weighted sum of the last tile)
@@ -385,8 +384,9 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
                 uint32_t o[16];
                 tc::tmem_ld16(tO + lane_addr + col0 + 16 * hf, o);
                 tc::tmem_ld_wait();
+                const uint64_t al2 = pack2(__float_as_uint(alpha), __float_as_uint(alpha));
 #pragma unroll
-                for (int i = 0; i < 16; ++i) Om[16 * hf + i] = fmaf(Om[16 * hf + i], alpha, __uint_as_float(o[i]));
+                for (int i = 0; i < 8; ++i) Om[8 * hf + i] = fma2(Om[8 * hf + i], al2, pack2(o[2 * i], o[2 * i + 1]));
             }
         };
         for (int t = 0; t < T; ++t) {
@@ -417,13 +417,18 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
                     tc::tmem_ld16(tSP + 16 * hf, xb);
                     tc::tmem_ld_wait();
 #pragma unroll
-                    for (int i = 0; i < 16; ++i)
-                        xa[16 * hf + i] = __float_as_uint(__uint_as_float(xa[16 * hf + i]) + __uint_as_float(xb[i]));
+                    for (int i = 0; i < 8; ++i)
+                        unpack2(add2(pack2(xa[16 * hf + 2 * i], xa[16 * hf + 2 * i + 1]), pack2(xb[2 * i], xb[2 * i + 1])),
+                                xa[16 * hf + 2 * i], xa[16 * hf + 2 * i + 1]);
                 }
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {       // each lane sends what the other needs
-                    const float other = __shfl_xor_sync(0xffffffffu, __uint_as_float(is_lo ? xa[i] : xa[16 + i]), 16);
-                    sc[i] = __uint_as_float(is_lo ? xa[16 + i] : xa[i]) + other;
+                for (int i = 0; i < 16; i += 2) {    // each lane sends what the other needs; sums two at a time
+                    const uint32_t o0 = __shfl_xor_sync(0xffffffffu, is_lo ? xa[i] : xa[16 + i], 16);
+                    const uint32_t o1 = __shfl_xor_sync(0xffffffffu, is_lo ? xa[i + 1] : xa[17 + i], 16);
+                    uint32_t s0, s1;
+                    unpack2(add2(pack2(is_lo ? xa[16 + i] : xa[i], is_lo ? xa[17 + i] : xa[i + 1]), pack2(o0, o1)), s0, s1);
+                    sc[i] = __uint_as_float(s0);
+                    sc[i + 1] = __uint_as_float(s1);
                 }
             }
             float vmax = -INFINITY;
@@ -445,18 +450,32 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
             // probabilities of this lane's 16 columns, split: the lane keeps its own part (hi or lo)
             // and hands the other part to the other lane of the head; 16 columns at a time (the hi
             // lane's columns first), to stay within the registers
-            float lsum = 0.f;
+            float lsum;
             {
                 uint32_t x[32];
+                const uint64_t m2 = pack2(__float_as_uint(m_new), __float_as_uint(m_new));
+                uint64_t ls2 = 0ull;
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const float p = fast_exp2(sc[i] - m_new);
-                    lsum += p;
-                    const float ph = tf32_hi(p), pl = p - ph;
-                    const float got = __shfl_xor_sync(0xffffffffu, is_lo ? ph : pl, 16);
-                    x[i] = __float_as_uint(is_lo ? got : ph);              // columns 0..15: own (hi lane) or received (lo lane)
-                    x[16 + i] = __float_as_uint(is_lo ? pl : got);         // columns 16..31
+                for (int i = 0; i < 16; i += 2) {       // two columns at a time (packed subtractions and additions)
+                    uint32_t d0, d1;
+                    unpack2(sub2(pack2(__float_as_uint(sc[i]), __float_as_uint(sc[i + 1])), m2), d0, d1);
+                    const float p0 = fast_exp2(__uint_as_float(d0)), p1 = fast_exp2(__uint_as_float(d1));
+                    const uint64_t p2 = pack2(__float_as_uint(p0), __float_as_uint(p1));
+                    ls2 = add2(ls2, p2);
+                    const uint64_t ph2 = p2 & 0xFFFFE000FFFFE000ull;          // hi parts (what the tensor core keeps)
+                    uint32_t ph0, ph1, pl0, pl1;
+                    unpack2(ph2, ph0, ph1);
+                    unpack2(sub2(p2, ph2), pl0, pl1);
+                    const uint32_t g0 = __shfl_xor_sync(0xffffffffu, is_lo ? ph0 : pl0, 16);
+                    const uint32_t g1 = __shfl_xor_sync(0xffffffffu, is_lo ? ph1 : pl1, 16);
+                    x[i] = is_lo ? g0 : ph0;                                   // columns 0..15: own (hi lane) or received (lo lane)
+                    x[i + 1] = is_lo ? g1 : ph1;
+                    x[16 + i] = is_lo ? pl0 : g0;                              // columns 16..31
+                    x[16 + i + 1] = is_lo ? pl1 : g1;
                 }
+                uint32_t l0, l1;
+                unpack2(ls2, l0, l1);
+                lsum = __uint_as_float(l0) + __uint_as_float(l1);
                 tc::tmem_st32(tSP, x);
             }
             tc::tmem_st_wait();
@@ -491,11 +510,14 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
                                   : a.ws + ((((size_t)b * a.h_kv + h) * a.splits + split) * GH) * PS) + (size_t)head * PS;
 #pragma unroll
             for (int i = 0; i < 32; i += 4) {
+                uint32_t w[4];
+                unpack2(Om[i / 2], w[0], w[1]);
+                unpack2(Om[i / 2 + 1], w[2], w[3]);
                 float4 v;
-                v.x = Om[i] + __shfl_xor_sync(0xffffffffu, Om[i], 16);
-                v.y = Om[i + 1] + __shfl_xor_sync(0xffffffffu, Om[i + 1], 16);
-                v.z = Om[i + 2] + __shfl_xor_sync(0xffffffffu, Om[i + 2], 16);
-                v.w = Om[i + 3] + __shfl_xor_sync(0xffffffffu, Om[i + 3], 16);
+                v.x = __uint_as_float(w[0]) + __shfl_xor_sync(0xffffffffu, __uint_as_float(w[0]), 16);
+                v.y = __uint_as_float(w[1]) + __shfl_xor_sync(0xffffffffu, __uint_as_float(w[1]), 16);
+                v.z = __uint_as_float(w[2]) + __shfl_xor_sync(0xffffffffu, __uint_as_float(w[2]), 16);
+                v.w = __uint_as_float(w[3]) + __shfl_xor_sync(0xffffffffu, __uint_as_float(w[3]), 16);
                 if (!is_lo && qhead_ok) *reinterpret_cast<float4 *>(slot + col0 + i) = v;
             }
             if (sub == 0 && !is_lo && qhead_ok) {
@@ -526,10 +548,14 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
 #pragma unroll
                 for (int i = 0; i < PER / 4; ++i) v[i] = p[ct + (part * (PER / 4) + i) * TT];
 #pragma unroll
-                for (int i = 0; i < PER / 4; ++i) {
-                    v[i].x -= tf32_hi(v[i].x); v[i].y -= tf32_hi(v[i].y);
-                    v[i].z -= tf32_hi(v[i].z); v[i].w -= tf32_hi(v[i].w);
-                    p[ct + (part * (PER / 4) + i) * TT] = v[i];
+                for (int i = 0; i < PER / 4; ++i) {       // lo = x - hi(x), two floats per instruction
+                    const uint64_t a01 = pack2(__float_as_uint(v[i].x), __float_as_uint(v[i].y));
+                    const uint64_t a23 = pack2(__float_as_uint(v[i].z), __float_as_uint(v[i].w));
+                    uint32_t w[4];
+                    unpack2(sub2(a01, a01 & 0xFFFFE000FFFFE000ull), w[0], w[1]);
+                    unpack2(sub2(a23, a23 & 0xFFFFE000FFFFE000ull), w[2], w[3]);
+                    p[ct + (part * (PER / 4) + i) * TT] = make_float4(__uint_as_float(w[0]), __uint_as_float(w[1]),
+                                                                      __uint_as_float(w[2]), __uint_as_float(w[3]));
                 }
             }
             tc::fence_async_smem();
