@@ -409,7 +409,8 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
                 __syncwarp();
                 if (ok && lane == 0) tc::mbar_arrive(bar_shread);
                 ok = ok && wait_suspended(bar_group_done(group_k(t)), par_group_done(group_k(t)), abort_flag);
-                if (named_or(1 + qd, 128, !ok)) { ok = false; break; }    // the four warps of a quadrant leave together
+                // (a warp whose wait has failed keeps walking through the tiles with the others, so that
+                // the barriers of its quadrant stay balanced; every later wait returns at once)
                 tc::fence_after_sync();
 #pragma unroll
                 for (int hf = 0; hf < 2; ++hf) {       // 16 columns at a time, to stay within the registers
