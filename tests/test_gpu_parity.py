@@ -590,3 +590,24 @@ def test_calls_on_two_streams_with_their_own_workspaces_do_not_disturb_each_othe
         w, q, K, V, ws, nb, out = dev[name]
         assert max_err(out.cpu().numpy(), oracle.decode(w.q(), w.K(), w.V(), w.scale)) <= TOL, name
     assert all(np.array_equal(o, outs_small[0]) for o in outs_small)
+
+
+@pytest.mark.parametrize("gs", [17, 24, 32, 64])
+def test_rows_of_64_features_on_the_tensor_core_kernel(gs):
+    """Dense caches at d = 64 with 17..32 or 64 heads per K/V head: two cached rows are read as
+    one row of 128, a head takes two pseudo-heads (even rows / odd rows).  Even row counts only;
+    an odd count keeps the streaming kernels."""
+    hkv, B = 2, 2
+    for n in (2, 66, 130, 256, 1000, 5002):
+        q, K, V, s = make(4000 + 10 * gs + n, B, gs * hkv, hkv, n, 64, 64)
+        ref = oracle.decode(q, K, V, s)
+        assert max_err(gpu_decode(q, K, V, s, expect_path=moa.PATH_GROUPED), ref) <= TOL, (gs, n)
+        # the same call with a caller-owned workspace and no lengths
+        assert max_err(gpu_decode(q, K, V, s, seq_lens=np.full((B,), n, np.int32)), ref) <= TOL, (gs, n)
+    q, K, V, s = make(4100 + gs, B, gs * hkv, hkv, 999, 64, 64)
+    assert max_err(gpu_decode(q, K, V, s), oracle.decode(q, K, V, s)) <= TOL
+    assert moa.moa_last_path() != moa.PATH_GROUPED
+    # larger scores and a uniform V, several splits per unit
+    q, K, V, s = make(4200 + gs, 1, gs, 1, 20000, 64, 64, v_dist="uniform")
+    q, K = 2 * q, 2 * K
+    assert max_err(gpu_decode(q, K, V, s, expect_path=moa.PATH_GROUPED), oracle.decode(q, K, V, s)) <= TOL
