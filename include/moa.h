@@ -285,7 +285,12 @@ const char *moa_strerror(int code);
  *   MOA_OPT_GROUPED_HEADS : query heads per CTA of the tensor-core kernel (16, 32 or 64;
  *                        0 = automatic).  Larger groups are cut into neighbouring CTAs.
  *   MOA_OPT_DEPENDENT_LAUNCH : 1 (default) = the streaming kernels are launched with
- *                        programmatic stream serialisation, 0 = ordinary launches.
+ *                        programmatic stream serialisation, 0 = ordinary launches.  Every
+ *                        kernel of the library waits for its predecessor in the stream
+ *                        before its first access to global memory, so calls in one stream
+ *                        are ordered as usual; a kernel of the caller's that is itself
+ *                        launched with programmatic stream serialisation right after a
+ *                        library call has to do the same (cudaGridDependencySynchronize).
  *   MOA_OPT_GROUPED_OPERANDS : 0 (default) = groups of 17..64 heads may use the tensor-core kernel
  *                        that keeps the query and probability operands in tensor memory
  *                        (64 head lanes, smaller groups padded); 1 = only the kernel with

@@ -222,6 +222,12 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
     tc::fence_before_sync();
     __syncthreads();
     tc::fence_after_sync();
+    // Launched with programmatic stream serialisation, this kernel may start while its
+    // predecessor in the stream is still running (the streaming kernels let their successor go
+    // early).  With a tail-copy kernel in front, that kernel is the only one (it was launched
+    // after everything before it had completed) and only the tail tiles come from it; without
+    // one, wait here, before the first access to global memory.
+    if (a.tailK == nullptr) grid_dependency_wait();
     // The first ring-full of chunks needs nothing but the barriers: the producer starts those
     // loads now, so that they travel while the query operand is being built.
     ChunkSeq pseq(T);                              // the producer's position (warp 0, lane 0)

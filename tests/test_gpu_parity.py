@@ -611,3 +611,49 @@ def test_rows_of_64_features_on_the_tensor_core_kernel(gs):
     q, K, V, s = make(4200 + gs, 1, gs, 1, 20000, 64, 64, v_dist="uniform")
     q, K = 2 * q, 2 * K
     assert max_err(gpu_decode(q, K, V, s, expect_path=moa.PATH_GROUPED), oracle.decode(q, K, V, s)) <= TOL
+
+
+def test_back_to_back_calls_of_different_kernel_families_on_one_stream():
+    """Programmatic launches let a kernel start while its predecessor in the stream still runs;
+    every kernel therefore waits for that predecessor before its first global access.  A fused
+    step on the warp-MMA kernel appends a row; the next call (tensor-core kernel, 32 heads per
+    K/V head over the same cache, library workspace) must see that row and must not share the
+    workspace with a kernel still in flight.  The first call of each pair is held to 32 CTAs, so
+    that a successor released too early would find free SMs beside it."""
+    B, hkv, n, d = 1, 1, 65536, 128                 # the first call is held to 32 CTAs: a long kernel beside free SMs
+    w1 = mi.Workload("b2b1", 3400, B, 8, hkv, n, d, d)
+    w2 = mi.Workload("b2b2", 3401, B, 32, hkv, n, d, d)
+    K, V, q1, q2 = w1.K(), w1.V(), w1.q(), w2.q()
+    k_new, v_new = w1.k_new(0), w1.v_new(0) + 50.0      # a row whose absence or presence is visible in every output
+    pos = np.full((B,), n - 1, np.int32)
+    dK0, dV0 = torch.from_numpy(K).cuda(), torch.from_numpy(V).cuda()
+    dq1, dq2, dk, dv, dpos = (torch.from_numpy(x).cuda() for x in (q1, q2, k_new, v_new, pos))
+    nbytes = moa.moa_workspace_bytes(B, 8, hkv, n, d, d)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    out1, out2, out3, out4 = (torch.empty((B, h, d), device="cuda") for h in (8, 32, 8, 32))
+    oracle.kv_append(K, V, k_new, v_new, pos)
+    ref1, ref2 = oracle.decode(q1, K, V, w1.scale), oracle.decode(q2, K, V, w2.scale)
+    for rep in range(5):
+        dK, dV = dK0.clone(), dV0.clone()
+        torch.cuda.synchronize()
+        moa.moa_set_option(moa.OPT_NUM_CTAS, 32)
+        try:
+            moa.moa_append_decode(dq1, dK, dV, dk, dv, out1, dpos, B, 8, hkv, n, d, d, w1.scale, ws, nbytes)
+        finally:
+            moa.moa_set_option(moa.OPT_NUM_CTAS, 0)
+        assert moa.moa_last_path() == moa.PATH_MMA
+        moa.moa_decode_attn(dq2, dK, dV, out2, B, 32, hkv, n, d, d, w2.scale)
+        assert moa.moa_last_path() == moa.PATH_GROUPED
+        # the same pair once more, now both on the library's workspace
+        moa.moa_set_option(moa.OPT_NUM_CTAS, 32)
+        try:
+            moa.moa_decode_attn(dq1, dK, dV, out3, B, 8, hkv, n, d, d, w1.scale)
+        finally:
+            moa.moa_set_option(moa.OPT_NUM_CTAS, 0)
+        moa.moa_decode_attn(dq2, dK, dV, out4, B, 32, hkv, n, d, d, w2.scale)
+        torch.cuda.synchronize()
+        assert moa.moa_device_status() == 0
+        assert max_err(out1.cpu().numpy(), ref1) <= TOL, rep
+        assert max_err(out2.cpu().numpy(), ref2) <= TOL, rep
+        assert max_err(out3.cpu().numpy(), ref1) <= TOL, rep
+        assert max_err(out4.cpu().numpy(), ref2) <= TOL, rep
