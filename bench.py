@@ -170,10 +170,9 @@ EXTRA_WORKLOADS = {
     # 32 query heads on one K/V head at d = 64 (the shape of the paper's GQA/MQA traffic table), long cache
     "extra_mqa_d64": mi.Workload("extra_mqa_d64", 1105, 8, 32, 1, 131072, 64, 64),
 }
-# Workloads whose step is issued as two calls, moa_kv_append + moa_decode_attn: the tensor-core
-# path for rows of 64 features needs a dense cache of known length, which the fused call (lengths
-# on the device) cannot promise.
-TWO_CALL_STEP = {"extra_mqa_d64"}
+# Workloads whose step is issued as two calls, moa_kv_append + moa_decode_attn, instead of the
+# fused moa_append_decode (none at present; kept for A/B timing of the two forms).
+TWO_CALL_STEP = set()
 
 
 class DenseRun:

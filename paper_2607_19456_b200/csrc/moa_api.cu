@@ -564,7 +564,9 @@ static cudaError_t launch_generic(const DecodeArgs &a, cudaStream_t st)
 struct PairPlan {
     bool ok = false;
     int share = 1, gs = 0, splits = 1, tiles_per_split = 1;
-    size_t ws_bytes = 0;
+    size_t ws_bytes = 0;                 // dense: units x splits partial slots
+    size_t flat_bytes = 0, tail_bytes = 0;   // ragged: one partial slot per CTA, the tail copies
+    size_t ws_ragged() const { return (flat_bytes + 255) / 256 * 256 + tail_bytes; }
 };
 static PairPlan plan_grouped_pair(const DeviceState &s, int batch, int h_q, int h_kv, int n, int d_k, int d_v)
 {
@@ -583,12 +585,28 @@ static PairPlan plan_grouped_pair(const DeviceState &s, int batch, int h_q, int 
     p.splits = (int)splits;
     p.tiles_per_split = (tiles + p.splits - 1) / p.splits;
     p.ws_bytes = (size_t)vunits * p.splits * 64 * 132 * sizeof(float);
+    // ragged caches (one virtual head per stored one only): one partial per CTA, CTAs dealt by length
+    const size_t flat_slots = (size_t)(vunits > s.sm_count ? vunits : s.sm_count);
+    p.flat_bytes = flat_slots * 64 * 132 * sizeof(float);
+    p.tail_bytes = (size_t)batch * h_kv * 2 * 128 * 128 * sizeof(float);
     p.ok = true;
     return p;
 }
 
+struct FusedStep {                 // extra work folded into the decode launch(es)
+    float *Kw = nullptr, *Vw = nullptr;
+    const float *k_new = nullptr, *v_new = nullptr;
+    int32_t *lens_rw = nullptr;
+};
+
+// Rows of 64 features on the 64-lane kernel.  Dense caches: `seq_lens` null, one grid of
+// units x splits.  Ragged caches and the fused step (one virtual head per stored one): the
+// zero-padded copy of every unit's last tile first (which also stores the appended row), CTAs
+// dealt to the units by their lengths, then the merge and, for the step, the length advance.
 static cudaError_t launch_grouped_pair(const PairPlan &pp, const float *q, const float *K, const float *V, float *out,
-                                       float *ws, int batch, int h_q, int h_kv, int n, float scale, cudaStream_t st)
+                                       float *ws, int batch, int h_q, int h_kv, int n, float scale, cudaStream_t st,
+                                       const int32_t *seq_lens = nullptr, int len_bias = 0, const FusedStep *fused = nullptr,
+                                       int sm_count = 0)
 {
     const long long units = (long long)batch * h_kv;
     CUtensorMap mk, mv;
@@ -601,7 +619,7 @@ static cudaError_t launch_grouped_pair(const PairPlan &pp, const float *q, const
     ga.g_s = pp.gs; ga.h_kv_stored = h_kv; ga.share = pp.share;
     ga.splits = pp.splits; ga.tiles_per_split = pp.tiles_per_split;
     ga.qscale = scale * kLog2e;
-    ga.partial_out = nullptr; ga.seq_lens = nullptr; ga.len_bias = 0;
+    ga.partial_out = nullptr; ga.seq_lens = seq_lens; ga.len_bias = len_bias;
     ga.tailK = nullptr; ga.tailV = nullptr; ga.flat = 0;
     ga.pair = 1;
     using C = Grouped64Cfg;
@@ -614,10 +632,24 @@ static cudaError_t launch_grouped_pair(const PairPlan &pp, const float *q, const
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
+    CUtensorMap mkt = mk, mvt = mv;
+    int grid = (int)(units * pp.share * pp.splits);
+    if (seq_lens != nullptr) {
+        ga.tailK = reinterpret_cast<float *>(reinterpret_cast<unsigned char *>(ws) + (pp.flat_bytes + 255) / 256 * 256);
+        ga.tailV = ga.tailK + (size_t)units * 128 * 128;
+        if (!make_cache_map(&mkt, ga.tailK, units, 128, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
+            !make_cache_map(&mvt, ga.tailV, units, 128, 32, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B))
+            return cudaErrorInvalidValue;
+        grouped_tail_kernel<<<(int)units * 8, 256, 0, st>>>(ga, K, V, fused ? fused->Kw : nullptr, fused ? fused->Vw : nullptr,
+                                                            fused ? fused->k_new : nullptr, fused ? fused->v_new : nullptr);
+        count_launch();
+        if (cudaGetLastError() != cudaSuccess) return cudaErrorLaunchFailure;
+        grid = (int)(units > sm_count ? units : sm_count);
+        ga.flat = grid;
+    }
     {
         TimedLaunch t(st);
-        launch_dependent(grouped64_decode_kernel, (int)(units * pp.share * pp.splits), C::THREADS, C::SMEM_BYTES, st,
-                         mk, mv, mk, mv, ga);
+        launch_dependent(grouped64_decode_kernel, grid, C::THREADS, C::SMEM_BYTES, st, mk, mv, mkt, mvt, ga);
     }
     count_launch();
     cudaError_t e = cudaGetLastError();
@@ -625,17 +657,17 @@ static cudaError_t launch_grouped_pair(const PairPlan &pp, const float *q, const
     const long long rows = (long long)batch * h_q;
     launch_dependent(grouped_pair_combine_kernel, (int)((rows + 3) / 4), 128, 0, st, ga);
     count_launch();
-    return cudaGetLastError();
+    e = cudaGetLastError();
+    if (e == cudaSuccess && fused != nullptr && fused->lens_rw != nullptr) {
+        lens_add_kernel<<<(batch + 127) / 128, 128, 0, st>>>(fused->lens_rw, batch, 1, n);
+        count_launch();
+        e = cudaGetLastError();
+    }
+    return e;
 }
 
 // Shared implementation of the decode entry points.  `ws` may be null when the chosen
 // path needs none.
-struct FusedStep {                 // extra work folded into the streaming launch
-    float *Kw = nullptr, *Vw = nullptr;
-    const float *k_new = nullptr, *v_new = nullptr;
-    int32_t *lens_rw = nullptr;
-};
-
 static int decode_impl(const float *q, const float *K, const float *V, float *out, int batch,
                        int h_q, int h_kv, const int32_t *seq_lens, int len_bias, int n_max,
                        int d_k, int d_v, float scale, void *ws, size_t ws_bytes,
@@ -666,9 +698,23 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
             !make_rows_map(&probe, V, plan.D, n_max, h_kv, batch, lay.v))
             fast_ok = false;
     }
-    if (fast_ok && allow_grouped && lay.dense && seq_lens == nullptr && fused == nullptr && partial_out == nullptr) {
-        const PairPlan pp = plan_grouped_pair(*dev, batch, h_q, h_kv, n_max, d_k, d_v);
-        if (pp.ok && (library_ws || (ws && ws_bytes >= pp.ws_bytes))) {
+    // (ragged caches and the fused step: lengths on the device, scratch from the caller, one virtual head per stored one)
+    const bool pair_ragged = (seq_lens != nullptr) || (fused != nullptr);
+    if (fast_ok && allow_grouped && lay.dense && partial_out == nullptr &&
+        (!pair_ragged || (seq_lens != nullptr && !library_ws &&
+                          (fused == nullptr || (aligned(fused->k_new, 16) && aligned(fused->v_new, 16)))))) {
+        PairPlan pp = plan_grouped_pair(*dev, batch, h_q, h_kv, n_max, d_k, d_v);
+        if (pair_ragged && pp.share != 1) pp.ok = false;
+        if (pp.ok && pair_ragged) {
+            if (ws && ws_bytes >= pp.ws_ragged()) {
+                if (!aligned(ws, 256)) return MOA_ERR_ALIGN;
+                if (launch_grouped_pair(pp, q, K, V, out, static_cast<float *>(ws), batch, h_q, h_kv, n_max, scale, st,
+                                        seq_lens, len_bias, fused, dev->sm_count) != cudaSuccess)
+                    return MOA_ERR_CUDA;
+                g_last_path = MOA_PATH_GROUPED;
+                return MOA_OK;
+            }
+        } else if (pp.ok && (library_ws || (ws && ws_bytes >= pp.ws_bytes))) {
             if (library_ws) {
                 if (dev->ws_bytes < pp.ws_bytes) {
                     if (dev->ws) { cudaDeviceSynchronize(); cudaFree(dev->ws); dev->ws = nullptr; dev->ws_bytes = 0; }
@@ -938,6 +984,7 @@ size_t moa_workspace_bytes(int batch, int h_q, int h_kv, int n_max, int d_k, int
         if (gp.ok && gp.ws_ragged() > need) need = gp.ws_ragged();
         const PairPlan pp = plan_grouped_pair(*dev, batch, h_q, h_kv, n_max, d_k, d_v);
         if (pp.ok && pp.ws_bytes > need) need = pp.ws_bytes;
+        if (pp.ok && pp.share == 1 && pp.ws_ragged() > need) need = pp.ws_ragged();
     }
     return (need + 255) / 256 * 256;
 }

@@ -86,15 +86,24 @@ struct GroupedArgs {
     int flat;                  // 0, or the grid size: ragged caches, CTAs are dealt to the units in proportion
                                // to their lengths (see flat_share)
     int pair;                  // 64-lane kernel on rows of 64 features: two consecutive cached rows form one row of
-                               // 128 (n counts such pairs), a head takes two pseudo-heads (even rows, odd rows); dense only
+                               // 128 (n counts such pairs, lengths are given in cached rows), a head takes two
+                               // pseudo-heads (even rows, odd rows); ragged caches only with share == 1
 };
 
-// Rows of sequence b as this kernel family sees them; 0 for an out-of-range length.
+// Cached rows of sequence b (rows of 64 features in pair mode); 0 for an out-of-range length.
+__device__ __forceinline__ int grouped_len_rows(const GroupedArgs &a, int b)
+{
+    const int cap = a.pair ? 2 * a.n : a.n;
+    if (a.seq_lens == nullptr) return cap;
+    const int len = a.seq_lens[b] + a.len_bias;
+    return (len >= 1 && len <= cap) ? len : 0;
+}
+// Rows of sequence b as this kernel family sees them (pair mode: rows of 128 = pairs of cached
+// rows, the last one possibly half filled); 0 for an out-of-range length.
 __device__ __forceinline__ int grouped_len(const GroupedArgs &a, int b)
 {
-    if (a.seq_lens == nullptr) return a.n;
-    const int len = a.seq_lens[b] + a.len_bias;
-    return (len >= 1 && len <= a.n) ? len : 0;
+    const int rows = grouped_len_rows(a, b);
+    return a.pair ? (rows + 1) >> 1 : rows;
 }
 
 // Ragged caches, `flat` mode (share == 1): the grid's CTAs are dealt to the units in
@@ -156,12 +165,16 @@ __global__ void __launch_bounds__(256) grouped_tail_kernel(const GroupedArgs a, 
     launch_dependents();
     const int unit = blockIdx.x >> 3, part = blockIdx.x & 7, b = unit / a.h_kv_stored;
     const int len = grouped_len(a, b);
+    // pair mode: a row of 128 is two cached rows of 64; `halves` counts the cached rows of the tile
+    const int rows_real = grouped_len_rows(a, b);
     if (len == 0) {
         if (threadIdx.x == 0 && part == 0 && (unit % a.h_kv_stored) == 0)
             raise_status(MOA_STATUS_SEQLEN_RANGE | (k_new != nullptr ? MOA_STATUS_APPEND_RANGE : 0));
         return;
     }
     const int row0 = ((len - 1) / 128) * 128, valid = len - row0;
+    const int halves = a.pair ? rows_real - 2 * row0 : 2 * valid;     // 64-float half rows that hold data
+    const int new_half = halves - 1;                                  // pair mode: the appended cached row
     const float4 *srcK = reinterpret_cast<const float4 *>(K + ((size_t)unit * a.n + row0) * 128);
     const float4 *srcV = reinterpret_cast<const float4 *>(V + ((size_t)unit * a.n + row0) * 128);
     float4 *dstK = reinterpret_cast<float4 *>(a.tailK + (size_t)unit * 128 * 128);
@@ -169,11 +182,14 @@ __global__ void __launch_bounds__(256) grouped_tail_kernel(const GroupedArgs a, 
     const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int i = part * 512 + threadIdx.x; i < (part + 1) * 512; i += blockDim.x) {
         const int r = i >> 5, c = i & 31;
+        const int half = 2 * r + (c >> 4);
         float4 k = zero, v = zero;
-        if (r < valid) {
-            if (k_new != nullptr && r == valid - 1) {
-                k = reinterpret_cast<const float4 *>(k_new + (size_t)unit * 128)[c];
-                v = reinterpret_cast<const float4 *>(v_new + (size_t)unit * 128)[c];
+        if (half < halves) {
+            if (k_new != nullptr && (a.pair ? half == new_half : r == valid - 1)) {
+                k = a.pair ? reinterpret_cast<const float4 *>(k_new + (size_t)unit * 64)[c & 15]
+                           : reinterpret_cast<const float4 *>(k_new + (size_t)unit * 128)[c];
+                v = a.pair ? reinterpret_cast<const float4 *>(v_new + (size_t)unit * 64)[c & 15]
+                           : reinterpret_cast<const float4 *>(v_new + (size_t)unit * 128)[c];
                 reinterpret_cast<float4 *>(Kw + ((size_t)unit * a.n + row0) * 128)[i] = k;
                 reinterpret_cast<float4 *>(Vw + ((size_t)unit * a.n + row0) * 128)[i] = v;
             } else {
@@ -812,9 +828,22 @@ __global__ void __launch_bounds__(128) grouped_pair_combine_kernel(const Grouped
     if (wid >= (long long)a.batch * a.h_q) return;
     const int b = (int)(wid / a.h_q), gq = (int)(wid % a.h_q);
     const int vh = gq / a.g_s, j = gq % a.g_s;     // virtual kv head (a.h_kv of them per batch item), head inside it
-    const int tiles_total = (a.n + 127) / 128;
-    const int used = (tiles_total + a.tiles_per_split - 1) / a.tiles_per_split;     // non-empty splits
-    const float *base = a.ws + ((((size_t)b * a.h_kv + vh) * a.splits) * GH + 2 * j) * PS;
+    const int len_b = grouped_len(a, b);
+    if (len_b == 0) {                              // out-of-range length: report, leave out untouched
+        if (gq == 0 && lane == 0) raise_status(MOA_STATUS_SEQLEN_RANGE);
+        return;
+    }
+    const int tiles_total = (len_b + 127) / 128;
+    int splits_u = a.splits;
+    size_t first_slot = ((size_t)b * a.h_kv + vh) * a.splits;
+    if (a.flat) {                                  // ragged caches (share == 1): slots follow the CTAs
+        const FlatShare f = flat_share(a, a.flat, -1, b * a.h_kv + vh, lane);
+        splits_u = f.count;
+        first_slot = (size_t)f.first;
+    }
+    const int tiles_per_split = a.seq_lens ? (tiles_total + splits_u - 1) / splits_u : a.tiles_per_split;
+    const int used = (tiles_total + tiles_per_split - 1) / tiles_per_split;          // non-empty splits
+    const float *base = a.ws + (first_slot * GH + 2 * j) * PS;
     const size_t stride = (size_t)GH * PS;
     float M = -INFINITY;
     for (int i = lane; i < 2 * used; i += 32) M = fmaxf(M, base[(size_t)(i >> 1) * stride + (size_t)(i & 1) * PS + 128]);

@@ -194,6 +194,7 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
     const int b = a.pair ? sunit / a.h_kv : sunit / a.h_kv_stored;
     const int h = a.pair ? sunit % a.h_kv : sunit % a.h_kv_stored;  // (virtual) kv head inside the batch item
     const int len_b = grouped_len(a, b);           // 0: out-of-range length, the item is skipped
+    const int rows_b = grouped_len_rows(a, b);     // (pair mode: cached rows of 64 features)
     const int tiles_total = (len_b + C::TILE - 1) / C::TILE;
     const int tiles_per_split = a.seq_lens ? (tiles_total + splits_u - 1) / splits_u : a.tiles_per_split;
     const int tile0 = split * tiles_per_split;
@@ -263,6 +264,9 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
     const uint32_t lane_addr = (uint32_t)(qd * 32) << 16;
     const int head = 16 * qd + (lane & 15);
     const bool is_lo = (lane & 16) != 0;
+    // rows (of 128) this lane's head attends over: in pair mode pseudo-head 2j sees the even cached
+    // rows, pseudo-head 2j+1 the odd ones, so an odd length gives the latter one row less
+    const int len_m = a.pair ? (rows_b + 1 - (head & 1)) >> 1 : len_b;
     if (is_soft) {
         // Q operand: this lane's part (hi or lo) of (scale * log2 e) * q[head], columns = features
         // (a group of fewer than 64 heads is padded: the lanes of the missing heads hold zeros)
@@ -440,10 +444,10 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
             }
             float vmax = -INFINITY;
             const int rowc = row0 + (is_lo ? 16 : 0);
-            const bool full_tile = (row0 + 32 <= len_b);
+            const bool full_tile = (row0 + 32 <= len_m);
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
-                if (!full_tile && rowc + i >= len_b) sc[i] = -INFINITY;
+                if (!full_tile && rowc + i >= len_m) sc[i] = -INFINITY;
                 vmax = fmaxf(vmax, sc[i]);
             }
             vmax = fmaxf(vmax, __shfl_xor_sync(0xffffffffu, vmax, 16));
@@ -451,7 +455,9 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
             float *mxt = mx + (t & 1) * 256;
             if (!is_lo) mxt[sub * 64 + head] = vmax;
             named_sync(1 + qd, 128);
-            const float m_new = fmaxf(fmaxf(m_run, mxt[head]), fmaxf(fmaxf(mxt[64 + head], mxt[128 + head]), mxt[192 + head]));
+            // (never -inf: in pair mode a sequence of one row leaves the odd pseudo-heads without a score)
+            const float m_new = fmaxf(fmaxf(fmaxf(m_run, mxt[head]), fmaxf(fmaxf(mxt[64 + head], mxt[128 + head]), mxt[192 + head])),
+                                      -3.0e38f);
             const float alpha = exp2_diff(m_run, m_new);
             m_run = m_new;
             // probabilities of this lane's 16 columns, split: the lane keeps its own part (hi or lo)

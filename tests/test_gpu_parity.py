@@ -353,7 +353,7 @@ def test_append_out_of_range_position_is_skipped_and_reported():
 # ---------------------------------------------------------------------------------------
 @pytest.mark.parametrize("fused", [True, False])
 @pytest.mark.parametrize("D,hq,hkv", [(128, 8, 2), (64, 2, 1), (32, 8, 1), (16, 4, 4), (128, 8, 1), (64, 32, 2), ((128, 64), 8, 2),
-                                       ((64, 128), 4, 1), (128, 64, 1), (128, 64, 2)])
+                                       ((64, 128), 4, 1), (128, 64, 1), (128, 64, 2), (64, 64, 2), (64, 17, 1)])
 def test_multistep_small(fused, D, hq, hkv):
     D, Dv = D if isinstance(D, tuple) else (D, D)
     w = mi.Workload("ms", 950 + D + Dv, 4, hq, hkv, 80, D, Dv, steps=40, len_lo=1, len_hi=40)
@@ -390,7 +390,8 @@ def test_multistep_small(fused, D, hq, hkv):
 
 
 @pytest.mark.parametrize("ctas,misalign_new", [(0, 0), (4000, 0), (0, 1), (5, 0)])
-@pytest.mark.parametrize("D,hq,hkv", [(128, 32, 8), (64, 16, 1), (128, 6, 2), (32, 2, 2), (128, 16, 2), (128, 64, 1)])
+@pytest.mark.parametrize("D,hq,hkv", [(128, 32, 8), (64, 16, 1), (128, 6, 2), (32, 2, 2), (128, 16, 2), (128, 64, 1),
+                                      (64, 32, 1), (64, 48, 2)])
 def test_append_decode_single_call(ctas, misalign_new, D, hq, hkv):
     # one call appends at pos[b] and attends over pos[b]+1 rows; lengths are not modified.
     # ctas=4000 and a k_new that is only 4-byte aligned take the three-launch fallback.
@@ -657,3 +658,56 @@ def test_back_to_back_calls_of_different_kernel_families_on_one_stream():
         assert max_err(out2.cpu().numpy(), ref2) <= TOL, rep
         assert max_err(out3.cpu().numpy(), ref1) <= TOL, rep
         assert max_err(out4.cpu().numpy(), ref2) <= TOL, rep
+
+
+@pytest.mark.parametrize("gs", [17, 24, 32])
+def test_ragged_rows_of_64_features_on_the_tensor_core_kernel(gs):
+    """Ragged caches at d = 64 with 17..32 heads per K/V head (even capacity, scratch from the
+    caller): two cached rows are read as one row of 128, an odd length leaves the odd rows'
+    pseudo-heads one row short (none at all for a sequence of one row); rows past a length hold
+    NaNs and must not matter."""
+    hkv, n_max = 2, 1000
+    lens = np.array([1, 2, 3, 128, 129, 255, 256, 257, 999, 1000, 514, 77], np.int32)
+    B = len(lens)
+    q, K, V, s = make(4300 + gs, B, gs * hkv, hkv, n_max, 64, 64)
+    for b in range(B):
+        K[b, :, lens[b]:] = np.nan
+        V[b, :, lens[b]:] = np.nan
+    ref = oracle.decode_varlen(q, np.nan_to_num(K), np.nan_to_num(V), lens, s)
+    gq, gK, gV, glens = Guarded(q), Guarded(K), Guarded(V), Guarded(lens)
+    gout = Guarded(shape=(B, gs * hkv, 64))
+    gws, nbytes = workspace_for(B, gs * hkv, hkv, n_max, 64, 64)
+    moa.moa_decode_attn_varlen(gq.ptr, gK.ptr, gV.ptr, gout.ptr, B, gs * hkv, hkv, glens.ptr, n_max, 64, 64, s,
+                               gws.ptr, nbytes)
+    torch.cuda.synchronize()
+    assert moa.moa_last_path() == moa.PATH_GROUPED and moa.moa_device_status() == 0
+    assert max_err(gout.host(), ref) <= TOL
+    for g in (gq, gK, gV, glens, gout, gws):
+        assert g.guards_intact()
+    # an odd capacity keeps the streaming kernels
+    q, K, V, s = make(4350 + gs, 2, gs * hkv, hkv, 999, 64, 64)
+    l2 = np.array([999, 500], np.int32)
+    out = gpu_decode(q, K, V, s, seq_lens=l2)
+    assert moa.moa_last_path() != moa.PATH_GROUPED
+    assert max_err(out, oracle.decode_varlen(q, K, V, l2, s)) <= TOL
+
+
+def test_fused_step_at_capacity_on_rows_of_64_features():
+    B, hq, hkv, n_max, D = 2, 32, 1, 8, 64
+    q, K, V, s = make(961, B, hq, hkv, n_max, D, D)
+    lens = np.array([8, 3], np.int32)                       # item 0 is full
+    kn, vn = mi.normal(961, 4, (B, hkv, D)), mi.normal(961, 5, (B, hkv, D))
+    gq, gK, gV, gk, gv, glens = Guarded(q), Guarded(K), Guarded(V), Guarded(kn), Guarded(vn), Guarded(lens)
+    gout = Guarded(shape=(B, hq, D), fill=-7.0)
+    gws, nbytes = workspace_for(B, hq, hkv, n_max, D, D)
+    moa.moa_decode_step(gq.ptr, gK.ptr, gV.ptr, gk.ptr, gv.ptr, gout.ptr, glens.ptr, B, hq, hkv, n_max,
+                        D, D, s, gws.ptr, nbytes)
+    st = moa.moa_device_status()
+    assert moa.moa_last_path() == moa.PATH_GROUPED
+    assert st == (moa.STATUS_APPEND_RANGE | moa.STATUS_SEQLEN_RANGE)
+    assert list(glens.host()) == [8, 4]
+    assert np.all(gout.host()[0] == -7.0)
+    assert np.array_equal(gK.host()[0].view(np.uint32), K[0].view(np.uint32))
+    oracle.kv_append(K[1:], V[1:], kn[1:], vn[1:], lens[1:])
+    ref = oracle.decode_varlen(q[1:], K[1:], V[1:], np.array([4], np.int32), s)
+    assert max_err(gout.host()[1:], ref) <= TOL
