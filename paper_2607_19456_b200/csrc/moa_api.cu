@@ -655,7 +655,7 @@ static cudaError_t launch_grouped_pair(const PairPlan &pp, const float *q, const
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     const long long rows = (long long)batch * h_q;
-    launch_dependent(grouped_pair_combine_kernel, (int)((rows + 3) / 4), 128, 0, st, ga);
+    launch_dependent(grouped_pair_combine_kernel, (int)rows, 128, 0, st, ga);
     count_launch();
     e = cudaGetLastError();
     if (e == cudaSuccess && fused != nullptr && fused->lens_rw != nullptr) {

@@ -817,20 +817,22 @@ __global__ void __launch_bounds__(128) grouped_combine_kernel(const GroupedArgs 
 // Merge for the 64-lane kernel in pair mode (rows of 64 features): a head's result is spread over
 // two pseudo-heads, 2j (even cached rows: features 0..63 of its 128-wide partial are meaningful)
 // and 2j+1 (odd rows: features 64..127), each with a maximum and a sum of its own, times the
-// splits of the unit.  One warp per (batch, query head), partials in (split, parity) order,
-// compensated sums.
+// splits of the unit.  One block of four warps per (batch, query head), as in the kernel above:
+// warp w takes the partials w, w+4, ... in (split, parity) order against the global maximum,
+// the four compensated sums are added in warp order.
 __global__ void __launch_bounds__(128) grouped_pair_combine_kernel(const GroupedArgs a)
 {
     constexpr int PS = 132, GH = 64;
+    __shared__ float2 s_acc[4][32], s_accc[4][32];
+    __shared__ float s_l[4], s_lc[4];
     grid_dependency_wait();
-    const int lane = threadIdx.x & 31;
-    const long long wid = (long long)blockIdx.x * 4 + (threadIdx.x >> 5);
-    if (wid >= (long long)a.batch * a.h_q) return;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long wid = blockIdx.x;
     const int b = (int)(wid / a.h_q), gq = (int)(wid % a.h_q);
     const int vh = gq / a.g_s, j = gq % a.g_s;     // virtual kv head (a.h_kv of them per batch item), head inside it
     const int len_b = grouped_len(a, b);
     if (len_b == 0) {                              // out-of-range length: report, leave out untouched
-        if (gq == 0 && lane == 0) raise_status(MOA_STATUS_SEQLEN_RANGE);
+        if (gq == 0 && threadIdx.x == 0) raise_status(MOA_STATUS_SEQLEN_RANGE);
         return;
     }
     const int tiles_total = (len_b + 127) / 128;
@@ -851,13 +853,29 @@ __global__ void __launch_bounds__(128) grouped_pair_combine_kernel(const Grouped
     for (int off = 16; off >= 1; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
     float2 acc = make_float2(0.f, 0.f), accc = acc;
     float L = 0.f, Lc = 0.f;
-    for (int i = 0; i < 2 * used; ++i) {
+#pragma unroll 4
+    for (int i = warp; i < 2 * used; i += 4) {
         const float *row = base + (size_t)(i >> 1) * stride + (size_t)(i & 1) * PS;
         const float f = exp2_diff(row[128], M);
         comp_fma(L, Lc, row[129], f);
         const float2 t = *reinterpret_cast<const float2 *>(row + 64 * (i & 1) + 2 * lane);
         comp_fma(acc.x, accc.x, t.x, f);
         comp_fma(acc.y, accc.y, t.y, f);
+    }
+    s_acc[warp][lane] = acc; s_accc[warp][lane] = accc;
+    if (lane == 0) { s_l[warp] = L; s_lc[warp] = Lc; }
+    __syncthreads();
+    if (warp != 0) return;
+    acc = s_acc[0][lane]; accc = s_accc[0][lane];
+    L = s_l[0]; Lc = s_lc[0];
+#pragma unroll
+    for (int w = 1; w < 4; ++w) {
+        comp_fma(acc.x, accc.x, s_acc[w][lane].x, 1.0f);
+        comp_fma(acc.x, accc.x, s_accc[w][lane].x, -1.0f);
+        comp_fma(acc.y, accc.y, s_acc[w][lane].y, 1.0f);
+        comp_fma(acc.y, accc.y, s_accc[w][lane].y, -1.0f);
+        comp_fma(L, Lc, s_l[w], 1.0f);
+        comp_fma(L, Lc, s_lc[w], -1.0f);
     }
     const float inv = 1.0f / L;
     *reinterpret_cast<float2 *>(a.out + ((size_t)b * a.h_q + gq) * 64 + 2 * lane) = make_float2(acc.x * inv, acc.y * inv);
