@@ -62,3 +62,40 @@ def test_random_fused_steps(case):
     assert np.array_equal(gV.host().view(np.uint32), V.view(np.uint32))
     for g in (gK, gV, glens, gws, gout):
         assert g.guards_intact()
+
+
+@pytest.mark.parametrize("case", range(24))
+def test_random_large_groups_at_d64(case):
+    """17..32 and 64 heads per K/V head on rows of 64 features: even capacities take the 64-lane
+    tensor-core kernel two rows at a time (dense, ragged and fused step), odd ones the streaming
+    kernels; both against the oracle."""
+    r = np.random.default_rng(77000 + case)
+    gs = int(r.choice([17, 18, 23, 24, 31, 32, 64])); hkv = int(r.integers(1, 4)); B = int(r.integers(1, 6))
+    n = int(r.choice([2, 4, 16, 30, 128, 130, 254, 256, 258, 1000, 2050, 2 * int(r.integers(1, 2500)), int(r.integers(1, 3000))]))
+    hq = gs * hkv
+    q = mi.normal(77000 + case, 1, (B, hq, 64))
+    K = mi.normal(77000 + case, 2, (B, hkv, n, 64))
+    V = mi.normal(77000 + case, 3, (B, hkv, n, 64))
+    assert max_err(gpu_decode(q, K, V, 0.125), oracle.decode(q, K, V, 0.125)) <= TOL, (B, hq, hkv, n)
+    lens = r.integers(1, n + 1, size=B).astype(np.int32)
+    assert max_err(gpu_decode(q, K, V, 0.125, seq_lens=lens), oracle.decode_varlen(q, K, V, lens, 0.125)) <= TOL
+    n_max = n + 4
+    w = mi.Workload("fzp", 77000 + case, B, hq, hkv, n_max, 64, 64)
+    K, V = w.K(), w.V()
+    lens = r.integers(0, n_max - 3, size=B).astype(np.int32)
+    gK, gV, glens = Guarded(K), Guarded(V), Guarded(lens)
+    gws, nbytes = workspace_for(B, hq, hkv, n_max, 64, 64)
+    gout = Guarded(shape=(B, hq, 64))
+    for t in range(3):
+        kn, vn, qt = w.k_new(t), w.v_new(t), w.q_step(t)
+        gk, gv, gq = Guarded(kn), Guarded(vn), Guarded(qt)
+        moa.moa_decode_step(gq.ptr, gK.ptr, gV.ptr, gk.ptr, gv.ptr, gout.ptr, glens.ptr, B, hq, hkv, n_max, 64, 64,
+                            w.scale, gws.ptr, nbytes)
+        oracle.kv_append(K, V, kn, vn, lens)
+        lens = lens + 1
+        assert max_err(gout.host(), oracle.decode_varlen(qt, K, V, lens, w.scale)) <= TOL, (B, hq, hkv, n_max, t)
+    assert moa.moa_device_status() == 0
+    assert np.array_equal(gK.host().view(np.uint32), K.view(np.uint32))
+    assert np.array_equal(gV.host().view(np.uint32), V.view(np.uint32))
+    for g in (gK, gV, glens, gws, gout):
+        assert g.guards_intact()
