@@ -50,6 +50,7 @@ NCU_TRAFFIC = {
     "extra_group8_d128": {"bytes": 1075674112 + 735744, "sources": ["moa_mma.cuh", "moa_device.cuh"], "digest": "f33163d6964881e9"},
     "multi_step": {"bytes": 351759360 + 1064448, "sources": ["moa_stream.cuh", "moa_device.cuh"], "digest": "6fa6e4f72ab8ea40"},
     "mqa_long": {"bytes": 537187072 + 918528, "sources": ["moa_grouped64.cuh", "moa_grouped.cuh", "moa_tc.cuh"], "digest": "20558178161884c4"},
+    "extra_mqa_d64": {"bytes": 537044480 + 379904, "sources": ["moa_grouped64.cuh", "moa_grouped.cuh", "moa_tc.cuh"], "digest": "20558178161884c4"},
 }
 
 
