@@ -46,11 +46,11 @@ L2_BYTES_ASSUMED = 126 * 1024 * 1024
 # a digest of the kernel sources it was captured with; when those files have changed since,
 # the figure is stale and the line reports null instead.
 NCU_TRAFFIC = {
-    "gqa": {"bytes": 1074671872 + 495616, "sources": ["moa_stream.cuh", "moa_device.cuh"], "digest": "6fa6e4f72ab8ea40"},
-    "extra_group8_d128": {"bytes": 1075674112 + 735744, "sources": ["moa_mma.cuh", "moa_device.cuh"], "digest": "f33163d6964881e9"},
-    "multi_step": {"bytes": 351759360 + 1064448, "sources": ["moa_stream.cuh", "moa_device.cuh"], "digest": "6fa6e4f72ab8ea40"},
-    "mqa_long": {"bytes": 537187072 + 918528, "sources": ["moa_grouped64.cuh", "moa_grouped.cuh", "moa_tc.cuh"], "digest": "20558178161884c4"},
-    "extra_mqa_d64": {"bytes": 537044480 + 379904, "sources": ["moa_grouped64.cuh", "moa_grouped.cuh", "moa_tc.cuh"], "digest": "20558178161884c4"},
+    "gqa": {"bytes": 1074633984 + 712448, "sources": ["moa_stream.cuh", "moa_device.cuh"], "digest": "2059d7131252c205"},
+    "extra_group8_d128": {"bytes": 1075581184 + 977920, "sources": ["moa_mma.cuh", "moa_device.cuh"], "digest": "2bdcc5fb6d4fc6cd"},
+    "multi_step": {"bytes": 351770624 + 920064, "sources": ["moa_stream.cuh", "moa_device.cuh"], "digest": "2059d7131252c205"},
+    "mqa_long": {"bytes": 537107200 + 308480, "sources": ["moa_grouped64.cuh", "moa_grouped.cuh", "moa_tc.cuh"], "digest": "0b5aac4d04e08fcb"},
+    "extra_mqa_d64": {"bytes": 537044480 + 379904, "sources": ["moa_grouped64.cuh", "moa_grouped.cuh", "moa_tc.cuh"], "digest": "0b5aac4d04e08fcb"},
 }
 
 

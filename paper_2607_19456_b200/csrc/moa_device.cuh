@@ -89,8 +89,8 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
 
 // ---- bulk asynchronous copy global -> shared (TMA engine, 1-D) --------------------------
 // dst and src 16-byte aligned, bytes a positive multiple of 16.  Completion is signalled
-// on the mbarrier as `bytes` transaction bytes.  No multicast: every CTA fetches its own
-// tile.
+// on the mbarrier as `bytes` transaction bytes.  Every CTA fetches its own tile (plain
+// copies into the issuing CTA's shared memory only).
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes,
                                          uint32_t bar)
 {

@@ -192,7 +192,7 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
-// ---- tiled TMA loads (no multicast) ---------------------------------------------------------
+// ---- tiled TMA loads (into the issuing CTA's shared memory only) ----------------------------
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const void *tmap, int c0, int c1, int c2, uint32_t bar)
 {
     asm volatile(
