@@ -573,10 +573,10 @@ static PairPlan plan_grouped_pair(const DeviceState &s, int batch, int h_q, int 
     PairPlan p;
     const int g_s = h_q / h_kv;
     if (d_k != 64 || d_v != 64 || (n & 1) || n < 2) return p;
-    if (!((g_s > 16 && g_s <= 32) || g_s == 64)) return p;
+    if (g_s <= 16 || g_s > 64) return p;
     if (g_grouped_operands != 0 || (g_force_path != 0 && g_force_path != MOA_PATH_GROUPED)) return p;
-    p.share = g_s == 64 ? 2 : 1;
-    p.gs = g_s == 64 ? 32 : g_s;
+    p.share = g_s > 32 ? 2 : 1;                   // 33..64 heads: two virtual heads per stored one, the second possibly smaller
+    p.gs = g_s > 32 ? (g_s + 1) / 2 : g_s;
     const long long vunits = (long long)batch * h_kv * p.share;
     if (vunits > 0x7fffffffLL / 256) return p;
     const int tiles = (n / 2 + 127) / 128;
@@ -622,6 +622,7 @@ static cudaError_t launch_grouped_pair(const PairPlan &pp, const float *q, const
     ga.partial_out = nullptr; ga.seq_lens = seq_lens; ga.len_bias = len_bias;
     ga.tailK = nullptr; ga.tailV = nullptr; ga.flat = 0;
     ga.pair = 1;
+    ga.g_total = h_q / h_kv;
     using C = Grouped64Cfg;
     static bool attr_set[kMaxDevices] = {};
     int dev = 0;
@@ -792,6 +793,7 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
         ga.tailK = nullptr; ga.tailV = nullptr;
         ga.flat = 0;
             ga.pair = 0;
+        ga.g_total = 0;
         CUtensorMap mkt = mk, mvt = mv;
         if (ragged) {
             // the last, partly filled tile of every unit, zero-padded (and the appended row of

@@ -88,6 +88,8 @@ struct GroupedArgs {
     int pair;                  // 64-lane kernel on rows of 64 features: two consecutive cached rows form one row of
                                // 128 (n counts such pairs, lengths are given in cached rows), a head takes two
                                // pseudo-heads (even rows, odd rows); ragged caches only with share == 1
+    int g_total;               // pair mode: query heads per stored K/V head (<= share * g_s: the last virtual head
+                               // of a stored one may hold fewer than g_s)
 };
 
 // Cached rows of sequence b (rows of 64 features in pair mode); 0 for an out-of-range length.
@@ -829,7 +831,9 @@ __global__ void __launch_bounds__(128) grouped_pair_combine_kernel(const Grouped
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const long long wid = blockIdx.x;
     const int b = (int)(wid / a.h_q), gq = (int)(wid % a.h_q);
-    const int vh = gq / a.g_s, j = gq % a.g_s;     // virtual kv head (a.h_kv of them per batch item), head inside it
+    const int in_stored = gq % a.g_total;          // head inside its stored K/V head
+    const int vh = (gq / a.g_total) * a.share + in_stored / a.g_s;   // virtual kv head (a.h_kv of them per batch item)
+    const int j = in_stored % a.g_s;               // head inside the virtual head
     const int len_b = grouped_len(a, b);
     if (len_b == 0) {                              // out-of-range length: report, leave out untouched
         if (gq == 0 && threadIdx.x == 0) raise_status(MOA_STATUS_SEQLEN_RANGE);

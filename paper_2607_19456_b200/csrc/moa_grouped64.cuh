@@ -274,8 +274,10 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
         // q of head j in features 0..63 and zeros in 64..127 (it sees the even cached rows),
         // pseudo-head 2j+1 the other way round.
         const int qhead = a.pair ? head >> 1 : head;
-        const bool has_q = qhead < a.g_s && (!a.pair || (sub >> 1) == (head & 1));
-        const float *qb = a.pair ? a.q + ((size_t)b * a.h_q + (size_t)h * a.g_s + qhead) * 64 + 32 * (sub & 1)
+        // pair mode: head inside its stored K/V head (virtual head h % share of stored head h / share)
+        const int q_in_stored = a.pair ? (h % a.share) * a.g_s + qhead : 0;
+        const bool has_q = qhead < a.g_s && (!a.pair || ((sub >> 1) == (head & 1) && q_in_stored < a.g_total));
+        const float *qb = a.pair ? a.q + ((size_t)b * a.h_q + (size_t)(h / a.share) * a.g_total + q_in_stored) * 64 + 32 * (sub & 1)
                                  : a.q + ((size_t)b * a.h_q + (size_t)h * a.g_s + head) * 128 + col0;
         uint32_t v[32];
 #pragma unroll
@@ -518,7 +520,8 @@ grouped64_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_
             const float l_pair = l_run + __shfl_xor_sync(0xffffffffu, l_run, 16);   // each lane summed 16 of the 32 columns
             if (!is_lo) lx[sub * 64 + head] = l_pair;
             named_sync(1 + qd, 128);
-            const bool qhead_ok = (a.pair ? head >> 1 : head) < a.g_s;
+            const bool qhead_ok = a.pair ? ((head >> 1) < a.g_s && (h % a.share) * a.g_s + (head >> 1) < a.g_total)
+                                         : head < a.g_s;
             float *slot = (a.flat ? a.ws + ((size_t)blockIdx.x * GH) * PS
                                   : a.ws + ((((size_t)b * a.h_kv + h) * a.splits + split) * GH) * PS) + (size_t)head * PS;
 #pragma unroll

@@ -24,7 +24,7 @@ def run_dense_on_gpu(w):
     want = moa.PATH_STREAM
     if 17 <= w.group <= 64 and w.d_k == 128:
         want = moa.PATH_GROUPED
-    elif (17 <= w.group <= 32 or w.group == 64) and w.d_k == 64 and w.n % 2 == 0:
+    elif 17 <= w.group <= 64 and w.d_k == 64 and w.n % 2 == 0:
         want = moa.PATH_GROUPED              # rows of 64 features, taken in pairs
     elif w.group % 8 == 0 and w.d_k >= 64:
         want = moa.PATH_MMA

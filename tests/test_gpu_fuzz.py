@@ -66,11 +66,11 @@ def test_random_fused_steps(case):
 
 @pytest.mark.parametrize("case", range(24))
 def test_random_large_groups_at_d64(case):
-    """17..32 and 64 heads per K/V head on rows of 64 features: even capacities take the 64-lane
+    """17..64 heads per K/V head on rows of 64 features: even capacities take the 64-lane
     tensor-core kernel two rows at a time (dense, ragged and fused step), odd ones the streaming
     kernels; both against the oracle."""
     r = np.random.default_rng(77000 + case)
-    gs = int(r.choice([17, 18, 23, 24, 31, 32, 64])); hkv = int(r.integers(1, 4)); B = int(r.integers(1, 6))
+    gs = int(r.choice([17, 18, 23, 24, 31, 32, 33, 41, 48, 63, 64])); hkv = int(r.integers(1, 4)); B = int(r.integers(1, 6))
     n = int(r.choice([2, 4, 16, 30, 128, 130, 254, 256, 258, 1000, 2050, 2 * int(r.integers(1, 2500)), int(r.integers(1, 3000))]))
     hq = gs * hkv
     q = mi.normal(77000 + case, 1, (B, hq, 64))

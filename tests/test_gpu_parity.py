@@ -52,7 +52,7 @@ def automatic_path(D, gs, n=2):
     """The kernel family the library picks for a dense, aligned call."""
     if D == 128 and 17 <= gs <= 64:
         return moa.PATH_GROUPED              # 64 head lanes, missing heads padded
-    if D == 64 and (17 <= gs <= 32 or gs == 64) and n % 2 == 0:
+    if D == 64 and 17 <= gs <= 64 and n % 2 == 0:
         return moa.PATH_GROUPED              # the same kernel on pairs of rows
     if 8 < gs < 16 and D >= 64:
         return moa.PATH_MMA                  # one padded group of 16 heads
@@ -593,10 +593,11 @@ def test_calls_on_two_streams_with_their_own_workspaces_do_not_disturb_each_othe
     assert all(np.array_equal(o, outs_small[0]) for o in outs_small)
 
 
-@pytest.mark.parametrize("gs", [17, 24, 32, 64])
+@pytest.mark.parametrize("gs", [17, 24, 32, 33, 40, 47, 63, 64])
 def test_rows_of_64_features_on_the_tensor_core_kernel(gs):
-    """Dense caches at d = 64 with 17..32 or 64 heads per K/V head: two cached rows are read as
-    one row of 128, a head takes two pseudo-heads (even rows / odd rows).  Even row counts only;
+    """Dense caches at d = 64 with 17..64 heads per K/V head: two cached rows are read as
+    one row of 128, a head takes two pseudo-heads (even rows / odd rows); more than 32 heads
+    run as two virtual heads per stored one, the second possibly smaller.  Even row counts only;
     an odd count keeps the streaming kernels."""
     hkv, B = 2, 2
     for n in (2, 66, 130, 256, 1000, 5002):
