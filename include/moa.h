@@ -316,7 +316,8 @@ const char *moa_strerror(int code);
 #define MOA_PATH_GROUPED   3   /* tcgen05 tensor-core kernels: groups of 17..64 heads (16 when forced) at d = 128, dense layout;
                                   groups of 17..64 heads at d = 64 when the capacity is even (ragged caches and the
                                   fused step: 17..32) */
-#define MOA_PATH_MMA       4   /* streaming kernel with warp-level MMA, groups of 8 or 16 heads, d_k, d_v in {64,128} */
+#define MOA_PATH_MMA       4   /* streaming kernel with warp-level MMA, 8 or 16 heads per fetched row (larger groups in
+                                  several passes), d_k, d_v in {64,128} */
 int moa_set_option(int option, int value);
 int moa_last_path(void);
 

@@ -182,10 +182,8 @@ static int stream_group(int g_s, int *share)
         *share = 1;
         return G;
     }
-    int G = 8;                           // largest power of two <= 8 dividing g_s
-    while (g_s % G != 0) G >>= 1;
-    *share = g_s / G;
-    return G;
+    *share = (g_s + 7) / 8;              // virtual kv heads of 8 query heads; the last may hold fewer
+    return 8;
 }
 
 static int rows_per_block(int D, int G)
@@ -209,12 +207,11 @@ static StreamPlan plan_stream(int g_s, int d_k, int d_v, bool rows_contig = true
         // (a row stride larger than the row) need tiled copies, which only that kernel issues:
         // small groups are padded to 8 heads, which costs no extra memory traffic.
         if (!mma_allowed() || (d_k != 64 && d_k != 128) || (d_v != 64 && d_v != 128)) return p;
-        if (g_s > 8 && g_s % 8 != 0 && !(d_k == d_v && g_s < 16)) return p;
         p.D = d_v;
         p.G = 8;
-        p.share = g_s > 8 ? g_s / 8 : 1;
+        p.share = g_s > 8 ? (g_s + 7) / 8 : 1;   // (the last virtual head of a stored one may hold fewer than 8)
         if (d_k == d_v && g_s > 8 && g_s < 16) { p.G = 16; p.share = 1; }
-        else if (d_k == d_v && g_s % 16 == 0) { p.G = 16; p.share = g_s / 16; }
+        else if (d_k == d_v && g_s >= 16) { p.G = 16; p.share = (g_s + 15) / 16; }
         p.mma = true;
         p.R = 16;
         p.ok = true;
@@ -224,7 +221,7 @@ static StreamPlan plan_stream(int g_s, int d_k, int d_v, bool rows_contig = true
     p.D = d_k;
     p.G = stream_group(g_s, &p.share);
     p.mma = mma_allowed() && p.G == 8 && p.D >= 64;
-    if (p.mma && g_s % 16 == 0) { p.G = 16; p.share = g_s / 16; }   // two 8-head tiles per fetched row
+    if (p.mma && g_s >= 16) { p.G = 16; p.share = (g_s + 15) / 16; }   // two 8-head tiles per fetched row (the last virtual head may hold fewer)
     if (mma_allowed() && p.D >= 64 && g_s > 8 && g_s < 16) {         // 9..15 heads: one padded 16-head group
         p.G = 16; p.share = 1; p.mma = true;
     }
@@ -754,7 +751,7 @@ static int decode_impl(const float *q, const float *K, const float *V, float *ou
     DecodeArgs a;
     a.q = q; a.K = K; a.V = V; a.out = out; a.ws = nullptr;
     a.seq_lens = seq_lens; a.len_bias = len_bias;
-    a.batch = batch; a.h_q = h_q; a.h_kv = h_kv; a.g_s = g_s; a.kv_share = 1;
+    a.batch = batch; a.h_q = h_q; a.h_kv = h_kv; a.g_s = g_s; a.kv_share = 1; a.g_total = g_s;
     a.n_max = n_max; a.d_k = d_k; a.d_v = d_v;
     a.k_sb = lay.k.sb; a.k_sh = lay.k.sh; a.k_sr = lay.k.sr;
     a.v_sb = lay.v.sb; a.v_sh = lay.v.sh; a.v_sr = lay.v.sr;

@@ -178,6 +178,8 @@ struct DecodeArgs {
     int h_kv;                 // kv heads as the kernels count them (virtual heads, see kv_share)
     int g_s;                  // query heads per (virtual) kv head
     int kv_share;             // consecutive virtual kv heads that read the same stored K/V head
+    int g_total;              // query heads per stored K/V head (<= kv_share * g_s: the last virtual head of a
+                              // stored one may hold fewer than g_s)
     int n_max;                // row capacity of every (batch, kv head) slab
     int d_k, d_v;
     // Element strides of the caches: batch item, stored kv head, row.  The dense layout is
@@ -199,6 +201,14 @@ struct DecodeArgs {
     long long skip_copy_block;// test hook: the copies of this row block are announced but never
                               // issued, so the wait for them runs out (-1: off)
 };
+
+// Query head (inside its batch item) that is head g of virtual kv head h, or -1 if that slot is
+// padding.  The virtual heads of a stored K/V head take its g_total heads in runs of g_s.
+__device__ __forceinline__ int query_head(const DecodeArgs &a, int h, int g)
+{
+    const int in_stored = (h % a.kv_share) * a.g_s + g;
+    return (g < a.g_s && in_stored < a.g_total) ? (h / a.kv_share) * a.g_total + in_stored : -1;
+}
 
 // Final emission of one float4 column group of a (batch, query head) row: the normalised
 // output, or -- for a caller that merges several row ranges itself (sequence split across
@@ -447,7 +457,8 @@ __device__ __forceinline__ void merge_unit_partials(const DecodeArgs &a, float *
         const int idx = tid + it * nthreads;
         if (idx < G * LPR) {
             const int hg = idx / LPR, d4 = idx % LPR;
-            if (hg < a.g_s) emit_columns(a, (size_t)b * a.h_q + (size_t)h * a.g_s + hg, D, d4, acc[it], M[it], L[it]);
+            const int qh = query_head(a, h, hg);
+            if (qh >= 0) emit_columns(a, (size_t)b * a.h_q + qh, D, d4, acc[it], M[it], L[it]);
         }
     }
 }

@@ -277,7 +277,8 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
                     comp_fma(L, Lc, merge_ml[(v * 8 + h8) * 2 + 1], f);
                 }
                 if (complete) {
-                    if (hg < a.g_s) emit_columns(a, (size_t)cc.b * a.h_q + (size_t)cc.h * a.g_s + hg, D, d4, acc, M, L);
+                    const int qh = query_head(a, cc.h, hg);
+                    if (qh >= 0) emit_columns(a, (size_t)cc.b * a.h_q + qh, D, d4, acc, M, L);
                 } else {
                     const int slot = (seg_begin == c0) ? 0 : 1;
                     float *dst = a.ws + (((size_t)blockIdx.x * 2 + slot) * G + hg) * PS;
@@ -360,14 +361,14 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
     // State: Q^T fragments of head g (chunk t+4j of the scaled query row, split), running
     // maximum and this thread's share of the sum for heads 2t and 2t+1.
     auto score_begin = [&](ScoreState<NJ, NT> &st) {
-        const float *qb = a.q + ((size_t)cc.b * a.h_q + (size_t)cc.h * a.g_s) * DK;
+        const float *qb = a.q + (size_t)cc.b * a.h_q * DK;
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
-            const int hg = 8 * nt + g;
+            const int qh = query_head(a, cc.h, 8 * nt + g);
 #pragma unroll
             for (int j = 0; j < NJ; ++j) {
                 float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (hg < a.g_s) v = *reinterpret_cast<const float4 *>(qb + (size_t)hg * DK + (t + 4 * j) * 4);
+                if (qh >= 0) v = *reinterpret_cast<const float4 *>(qb + (size_t)qh * DK + (t + 4 * j) * 4);
                 const Split4 s = split4(make_float4(v.x * a.qscale, v.y * a.qscale, v.z * a.qscale, v.w * a.qscale));
 #pragma unroll
                 for (int i = 0; i < 4; ++i) { st.qh[nt][j][i] = s.h[i]; st.ql[nt][j][i] = s.l[i]; }

@@ -180,11 +180,12 @@ __global__ void __launch_bounds__(C::THREADS, 1) stream_decode_kernel(const Deco
     float4 o[G];
     float m_run, l_run;
     auto begin_unit = [&]() {
-        const float *qb = a.q + ((size_t)cc.b * a.h_q + (size_t)cc.h * a.g_s) * D;
+        const float *qb = a.q + (size_t)cc.b * a.h_q * D;
 #pragma unroll
         for (int g = 0; g < G; ++g) {
             float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (g < a.g_s) t = *reinterpret_cast<const float4 *>(qb + (size_t)g * D + (lane % LPR) * 4);
+            const int qh = query_head(a, cc.h, g);
+            if (qh >= 0) t = *reinterpret_cast<const float4 *>(qb + (size_t)qh * D + (lane % LPR) * 4);
             qreg[g] = make_float4(t.x * a.qscale, t.y * a.qscale, t.z * a.qscale, t.w * a.qscale);
             o[g] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
@@ -227,7 +228,8 @@ __global__ void __launch_bounds__(C::THREADS, 1) stream_decode_kernel(const Deco
                 comp_fma(L, Lc, merge_ml[(v * G + g) * 2 + 1], f);
             }
             if (complete) {
-                if (g < a.g_s) emit_columns(a, (size_t)cc.b * a.h_q + (size_t)cc.h * a.g_s + g, D, d4, acc, M, L);
+                const int qh = query_head(a, cc.h, g);
+                if (qh >= 0) emit_columns(a, (size_t)cc.b * a.h_q + qh, D, d4, acc, M, L);
             } else {
                 const int slot = (seg_begin == c0) ? 0 : 1;
                 float *dst = a.ws + (((size_t)blockIdx.x * 2 + slot) * G + g) * PS;
@@ -377,7 +379,8 @@ __global__ void __launch_bounds__(128) stream_combine_kernel(const DecodeArgs a,
     const long long wid = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (wid >= (long long)a.batch * a.h_q) return;
     const int b = (int)(wid / a.h_q), gq = (int)(wid % a.h_q);
-    const int h = gq / a.g_s, g = gq % a.g_s;
+    const int in_stored = gq % a.g_total;      // head inside its stored K/V head
+    const int h = (gq / a.g_total) * a.kv_share + in_stored / a.g_s, g = in_stored % a.g_s;
 
     const long long total = total_blocks<R>(a, lane);
     const long long bpc = (total + num_ctas - 1) / num_ctas;

@@ -56,19 +56,16 @@ def automatic_path(D, gs, n=2):
         return moa.PATH_GROUPED              # the same kernel on pairs of rows
     if 8 < gs < 16 and D >= 64:
         return moa.PATH_MMA                  # one padded group of 16 heads
+    G = 8                                    # larger groups: virtual heads of 8, the last one possibly smaller
     if gs <= 8:
         G = 1
         while G < gs:
             G *= 2
-    else:
-        G = 8
-        while gs % G:
-            G //= 2
     return moa.PATH_MMA if (G == 8 and D >= 64) else moa.PATH_STREAM
 
 
 @pytest.mark.parametrize("D", [32, 64, 128])
-@pytest.mark.parametrize("gs", [1, 2, 3, 4, 5, 8, 12, 16, 24, 40, 64])
+@pytest.mark.parametrize("gs", [1, 2, 3, 4, 5, 8, 12, 16, 19, 20, 24, 40, 43, 63, 64])
 def test_stream_kernel_group_sizes(D, gs):
     hkv = 2
     for n in (1, 7, 130, 1037):

@@ -98,7 +98,8 @@ def test_contiguous_rows_large_groups_run_on_the_mma_kernel(kind, D, gs):
 
 @pytest.mark.parametrize("kind", ["nhd", "nhd_pad"])
 @pytest.mark.parametrize("dk,dv,gs", [(128, 128, 1), (128, 128, 4), (128, 128, 8), (64, 64, 2), (64, 64, 16),
-                                      (128, 64, 4), (64, 128, 8), (128, 128, 12), (128, 128, 32)])
+                                      (128, 64, 4), (64, 128, 8), (128, 128, 12), (128, 128, 32), (128, 128, 21),
+                                      (64, 128, 19)])
 def test_heads_innermost_runs_on_the_mma_kernel(kind, dk, dv, gs):
     for n in (1, 16, 17, 333, 1500):
         run_strided(kind, dk + 3 * dv + gs + n, 2, 3 * gs, 3, n, dk, dv, expect=(moa.PATH_MMA,))
@@ -110,7 +111,8 @@ def test_layouts_without_a_fast_kernel_run_on_the_catch_all_kernel(kind):
     run_strided(kind, 6, 2, 4, 2, 77, 24, 40, expect=(moa.PATH_GENERIC,))
     if kind == "odd":
         run_strided(kind, 7, 2, 8, 2, 130, 128, 128, expect=(moa.PATH_GENERIC,))
-    run_strided(kind, 8, 2, 40, 2, 50, 128, 128, expect=(moa.PATH_GENERIC,))         # 20 heads per group
+    # 20 heads per group: virtual heads of 8, 8 and 4 on the warp-MMA kernel where tiled copies are possible
+    run_strided(kind, 8, 2, 40, 2, 50, 128, 128, expect=(moa.PATH_GENERIC if kind == "odd" else moa.PATH_MMA,))
 
 
 def test_shared_rows_for_every_batch_item_on_large_groups():
