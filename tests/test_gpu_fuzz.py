@@ -13,7 +13,7 @@ from gpu_util import TOL, Guarded, gpu_decode, max_err, workspace_for
 pytestmark = pytest.mark.gpu
 torch = pytest.importorskip("torch")
 
-GROUPS = [1, 2, 3, 4, 6, 8, 8, 12, 16, 16, 24, 32, 48, 64]
+GROUPS = [1, 2, 3, 4, 5, 6, 7, 8, 8, 9, 12, 16, 16, 19, 20, 24, 27, 32, 43, 48, 63, 64]
 
 
 def draw(case):
