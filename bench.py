@@ -46,11 +46,11 @@ L2_BYTES_ASSUMED = 126 * 1024 * 1024
 # a digest of the kernel sources it was captured with; when those files have changed since,
 # the figure is stale and the line reports null instead.
 NCU_TRAFFIC = {
-    "gqa": {"bytes": 1074633984 + 712448, "sources": ["moa_stream.cuh", "moa_device.cuh"], "digest": "2059d7131252c205"},
-    "extra_group8_d128": {"bytes": 1075581184 + 977920, "sources": ["moa_mma.cuh", "moa_device.cuh"], "digest": "2bdcc5fb6d4fc6cd"},
-    "multi_step": {"bytes": 351770624 + 920064, "sources": ["moa_stream.cuh", "moa_device.cuh"], "digest": "2059d7131252c205"},
-    "mqa_long": {"bytes": 537107200 + 308480, "sources": ["moa_grouped64.cuh", "moa_grouped.cuh", "moa_tc.cuh"], "digest": "0b5aac4d04e08fcb"},
-    "extra_mqa_d64": {"bytes": 537044480 + 379904, "sources": ["moa_grouped64.cuh", "moa_grouped.cuh", "moa_tc.cuh"], "digest": "0b5aac4d04e08fcb"},
+    "gqa": {"bytes": 1074633984 + 749568, "sources": ["moa_stream.cuh", "moa_device.cuh"], "digest": "833a325649c099ec"},
+    "extra_group8_d128": {"bytes": 1075635712 + 687616, "sources": ["moa_mma.cuh", "moa_device.cuh"], "digest": "2997f121ba054f53"},
+    "multi_step": {"bytes": 351778816 + 703488, "sources": ["moa_stream.cuh", "moa_device.cuh"], "digest": "833a325649c099ec"},
+    "mqa_long": {"bytes": 537101568 + 515584, "sources": ["moa_grouped64.cuh", "moa_grouped.cuh", "moa_tc.cuh"], "digest": "d68ab0582bbd0527"},
+    "extra_mqa_d64": {"bytes": 537046016 + 319744, "sources": ["moa_grouped64.cuh", "moa_grouped.cuh", "moa_tc.cuh"], "digest": "d68ab0582bbd0527"},
 }
 
 
