@@ -277,7 +277,7 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
                     comp_fma(L, Lc, merge_ml[(v * 8 + h8) * 2 + 1], f);
                 }
                 if (complete) {
-                    const int qh = query_head(a, cc.h, hg);
+                    const int qh = query_head<NT == 1>(a, cc.h, hg);
                     if (qh >= 0) emit_columns(a, (size_t)cc.b * a.h_q + qh, D, d4, acc, M, L);
                 } else {
                     const int slot = (seg_begin == c0) ? 0 : 1;
@@ -300,7 +300,7 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
             __syncthreads();
             if (s_last) {                          // uniform for the CTA
                 __threadfence();
-                merge_unit_partials<D>(a, merge_o, P * 8 * D, G, c_first, c_last, bpc, cc.first, cc.b, cc.h, tid,
+                merge_unit_partials<D, NT == 1>(a, merge_o, P * 8 * D, G, c_first, c_last, bpc, cc.first, cc.b, cc.h, tid,
                                        C::THREADS);
             }
         }
@@ -364,7 +364,7 @@ mma_decode_kernel(const __grid_constant__ CUtensorMap tmapK, const __grid_consta
         const float *qb = a.q + (size_t)cc.b * a.h_q * DK;
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
-            const int qh = query_head(a, cc.h, 8 * nt + g);
+            const int qh = query_head<NT == 1>(a, cc.h, 8 * nt + g);
 #pragma unroll
             for (int j = 0; j < NJ; ++j) {
                 float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
