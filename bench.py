@@ -46,11 +46,11 @@ L2_BYTES_ASSUMED = 126 * 1024 * 1024
 # a digest of the kernel sources it was captured with; when those files have changed since,
 # the figure is stale and the line reports null instead.
 NCU_TRAFFIC = {
-    "gqa": {"bytes": 1074633984 + 749568, "sources": ["moa_stream.cuh", "moa_device.cuh"], "digest": "833a325649c099ec"},
-    "extra_group8_d128": {"bytes": 1075635712 + 687616, "sources": ["moa_mma.cuh", "moa_device.cuh"], "digest": "2997f121ba054f53"},
-    "multi_step": {"bytes": 351778816 + 703488, "sources": ["moa_stream.cuh", "moa_device.cuh"], "digest": "833a325649c099ec"},
-    "mqa_long": {"bytes": 537101568 + 515584, "sources": ["moa_grouped64.cuh", "moa_grouped.cuh", "moa_tc.cuh"], "digest": "d68ab0582bbd0527"},
-    "extra_mqa_d64": {"bytes": 537046016 + 319744, "sources": ["moa_grouped64.cuh", "moa_grouped.cuh", "moa_tc.cuh"], "digest": "d68ab0582bbd0527"},
+    "gqa": {"bytes": 1074629632 + 1160704, "sources": ["moa_stream.cuh", "moa_device.cuh"], "digest": "5eab75429bf75dce"},
+    "extra_group8_d128": {"bytes": 1075606784 + 769792, "sources": ["moa_mma.cuh", "moa_device.cuh"], "digest": "7c7e6fb243ebb37f"},
+    "multi_step": {"bytes": 351830272 + 909056, "sources": ["moa_stream.cuh", "moa_device.cuh"], "digest": "5eab75429bf75dce"},
+    "mqa_long": {"bytes": 537116160 + 265472, "sources": ["moa_grouped64.cuh", "moa_grouped.cuh", "moa_tc.cuh"], "digest": "d68ab0582bbd0527"},
+    "extra_mqa_d64": {"bytes": 537045504 + 388608, "sources": ["moa_grouped64.cuh", "moa_grouped.cuh", "moa_tc.cuh"], "digest": "d68ab0582bbd0527"},
 }
 
 
