@@ -14,7 +14,9 @@ torch = pytest.importorskip("torch")
 
 
 @pytest.mark.parametrize("hq,hkv,d,want", [(8, 2, 128, moa.PATH_STREAM), (16, 2, 128, moa.PATH_MMA), (8, 1, 64, moa.PATH_MMA),
-                                           (64, 1, 128, moa.PATH_GROUPED), (40, 1, 128, moa.PATH_GROUPED)])
+                                           (64, 1, 128, moa.PATH_GROUPED), (40, 1, 128, moa.PATH_GROUPED),
+                                           (32, 1, 64, moa.PATH_GROUPED),      # rows of 64 features, two at a time
+                                           (38, 2, 64, moa.PATH_GROUPED)])     # 19 heads per K/V head, padded lanes
 def test_captured_steps_replay(hq, hkv, d, want):
     T, B, n_max = 6, 3, 400
     w = mi.Workload("gr", 5200 + hq + d, B, hq, hkv, n_max, d, d, steps=T, len_lo=1, len_hi=300)
